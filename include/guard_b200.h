@@ -1,0 +1,182 @@
+/*
+ * guard_b200.h -- C ABI of the straggler-scoring library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes the numerical core of Guard's online monitor (paper Section 4.2,
+ * "Online Monitoring Strategy") and the scoring half of its offline node sweep
+ * (Sections 5.2-5.4) over a fleet telemetry tensor T[step, rank, metric], float32,
+ * metric innermost, row-major.  The paper fixes the rules in words (peer-relative
+ * evaluation, several indicators, deviation sustained over evaluation windows, step time
+ * as the primary signal, response tiers at about 10 % and at 20 % or more, a node passes
+ * only if every part of its sweep passes) and names no statistic; the statistics below
+ * (median, raw median absolute deviation, the 0.6745-scaled robust z with a one-sided
+ * cut-off, k-of-W persistence, nearest-rank percentile) are the reading this library
+ * implements.
+ *
+ * Conventions
+ *   - Every pointer whose name starts with d_ is DEVICE memory owned by the caller; all
+ *     other pointers are HOST memory.  The library never allocates, frees or keeps device
+ *     memory of its own: the caller hands it one workspace (guard_workspace_bytes) that
+ *     holds the telemetry ring and all state, and must keep it alive and untouched until
+ *     guard_destroy.
+ *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it and no
+ *     call synchronises, except guard_sync_status.  Calls on one context must be issued
+ *     in order on streams that are ordered with respect to each other.
+ *   - Every function returns a status (GUARD_OK = 0, errors negative) and never throws,
+ *     aborts or traps.  Argument errors are detected on the host before anything is
+ *     enqueued.  Data-dependent errors (non-finite telemetry, a bounded wait that ran out)
+ *     are recorded in a sticky device status word that guard_sync_status reads back.
+ *   - Output pointers documented as "or NULL" may be NULL to skip that output.
+ *   - Order of values is the IEEE total order of finite float32 (so -0 < +0).  All
+ *     decisions (exceedance, flag, tier, percentile cut, top-k order) use single float32
+ *     subtract / multiply / fabs / compare only and are reproducible bit for bit;
+ *     reported scores use one extra float32 division.
+ */
+#ifndef GUARD_B200_H
+#define GUARD_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GUARD_MAX_METRICS 32
+#define GUARD_MAX_TOPK 1024
+#define GUARD_MAX_WINDOW 65535
+
+enum {
+    GUARD_OK = 0,
+    GUARD_ERR_ARG = -1,        /* invalid argument (see guard_last_error) */
+    GUARD_ERR_WORKSPACE = -2,  /* workspace NULL, misaligned (256 B) or too small */
+    GUARD_ERR_NOT_READY = -3,  /* guard_score before the first ingested step */
+    GUARD_ERR_NONFINITE = -4,  /* NaN or Inf seen in ingested telemetry (sticky) */
+    GUARD_ERR_TIMEOUT = -5,    /* a bounded on-device wait ran out (sticky) */
+    GUARD_ERR_CUDA = -6,       /* a CUDA runtime call failed */
+    GUARD_ERR_INTERNAL = -7    /* a device-side consistency check failed (sticky) */
+};
+
+typedef struct guard_ctx guard_ctx; /* host object; owns no device memory */
+
+/* Detector parameters; copied by guard_create / guard_sweep_qualify (host memory). */
+typedef struct {
+    int32_t primary;        /* index of the primary metric: training-step time (Sec. 4.2) */
+    int32_t min_signals;    /* metrics that must deviate persistently, "multiple" (Sec. 4.2); clipped to M */
+    int32_t n_consec;       /* consecutive evaluations required before a flag is raised (>= 1) */
+    int32_t ranks_per_node; /* 8 in the paper's cluster (Sec. 7.1); used by guard_node_verdict */
+    float tier_moderate;    /* relative slowdown of the moderate tier, 0.10 (Sec. 4.2) */
+    float tier_severe;      /* relative slowdown of the severe tier, 0.20 (Sec. 4.2) */
+    const int8_t *dir;      /* [M] +1: larger is worse (durations, temperature); -1: smaller is worse */
+    const float *thr;       /* [M] robust-z cut-off, e.g. 3.5 */
+    const float *floor_rel; /* [M] floor of the spread relative to |median|, e.g. 1e-4 */
+    const float *floor_abs; /* [M] absolute floor of the spread, e.g. 0 */
+} guard_thresholds;
+
+/* Bytes of device workspace needed by a context with these sizes (0 on invalid sizes).
+ * The ring holds capacity_steps steps; windows use the last min(W, seen) of them. */
+size_t guard_workspace_bytes(int ranks, int metrics, int W, int capacity_steps, int topk);
+
+/*
+ * Create a context for `ranks` peers and `metrics` (1..32) indicators, window W
+ * (1..65535 steps), persistence k (1..W): a metric is persistent for a rank when at
+ * least k of the last W steps exceeded the per-step peer baseline ("sustained deviation
+ * ... across consecutive evaluation windows", Sec. 4.2).  topk in 0..min(ranks, 1024).
+ * d_workspace: device memory, 256-byte aligned, >= guard_workspace_bytes(...); its state
+ * part is zeroed on `stream`.  Errors: GUARD_ERR_ARG, GUARD_ERR_WORKSPACE, GUARD_ERR_CUDA.
+ */
+int guard_create(guard_ctx **out, int ranks, int metrics, int W, int k, const guard_thresholds *th,
+                 int capacity_steps, int topk, void *d_workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Where the next `steps` steps of telemetry go inside the ring, for producers that write
+ * telemetry in place (a gather kernel, a host-to-device copy): *d_slot receives a device
+ * pointer to steps*ranks*metrics contiguous floats.  Fails with GUARD_ERR_ARG if that
+ * span would wrap around the end of the ring (choose capacity_steps as a multiple of the
+ * block size).  Passing the returned pointer to guard_ingest skips the copy into the ring.
+ */
+int guard_ring_reserve(guard_ctx *ctx, int steps, float **d_slot);
+
+/*
+ * Ingest B (1..capacity_steps) steps: d_block[B][ranks][metrics] float32.  Appends them
+ * to the ring (a device-to-device copy unless d_block came from guard_ring_reserve) and
+ * computes, for every step and metric, the cross-rank median and raw MAD -- the peer
+ * baseline of that step (Sec. 4.2, evaluation "relative to peer nodes") -- and the
+ * one-sided exceedance bit of every rank,
+ *     dir * (x - med) > (float)(thr / 0.6745) * max(mad, floor_rel * |med|, floor_abs),
+ * stored in the exceedance ring.  Even rank counts use the midpoint of the two middle
+ * values (one float32 add, one multiply by 0.5).
+ * d_step_med, d_step_mad: [B][metrics] float32 or NULL.
+ * Non-finite input sets the sticky GUARD_ERR_NONFINITE status; results are then
+ * unspecified until guard_reset.
+ */
+int guard_ingest(guard_ctx *ctx, const float *d_block, int B, float *d_step_med, float *d_step_mad, void *stream);
+
+/*
+ * One evaluation over the window of the last n = min(W, seen) steps (Sec. 4.2):
+ *   d_wmed[r][m]    windowed per-rank median (blind to isolated spikes)
+ *   d_fleet_med[m], d_fleet_mad[m]  cross-rank median / raw MAD of the windowed medians
+ *   d_scores[r][m]  0.6745 * dir * (wmed - fleet_med) / scale, 0 where wmed == fleet_med
+ *   d_counts[r][m]  exceedances among the window's steps (k-of-W persistence filter)
+ *   d_metric_mask[r] bit m set when the windowed median exceeds the cut-off AND count >= k
+ *   d_flags[r]      1 when the primary metric's bit is set, at least min_signals bits are
+ *                   set, and this held for n_consec consecutive evaluations
+ *   d_tier[r]       3: flagged and primary slowdown >= tier_severe * |fleet_med|;
+ *                   2: flagged and >= tier_moderate; 1: some bit set ("pending
+ *                   verification"); 0 otherwise
+ *   d_topk_idx[K], d_topk_score[K]  the K ranks with the largest dir * wmed of the primary
+ *                   metric (ties: lower rank first) and their primary scores
+ * Every output is "or NULL".  Updates the per-rank consecutive-evaluation counters.
+ * Errors: GUARD_ERR_NOT_READY before the first step.
+ */
+int guard_score(guard_ctx *ctx, float *d_wmed, float *d_fleet_med, float *d_fleet_mad, float *d_scores,
+                uint16_t *d_counts, uint32_t *d_metric_mask, uint8_t *d_flags, uint8_t *d_tier,
+                int32_t *d_topk_idx, float *d_topk_score, void *stream);
+
+/* Bytes of device workspace needed by guard_sweep_qualify (0 on invalid sizes). */
+size_t guard_sweep_workspace_bytes(int gpus, int reps, int metrics);
+
+/*
+ * Offline node-sweep qualification (Sec. 5.2-5.4): d_S[g][rep][metric] float32 holds the
+ * repeated benchmark results of GPU g = node * gpus_per_node + local index.  Per GPU and
+ * metric the median over the repetitions; per metric over all GPUs the median, raw MAD
+ * and the nearest-rank percentile cut of the bad tail (j = ceil(pct_ppm * G / 1e6)
+ * clipped to [1, G]; the j-th worst value).  Metric m fails GPU g when it is a robust-z
+ * outlier in the bad direction AND strictly beyond the cut.  A GPU passes when no metric
+ * fails; a node passes when all its GPUs pass ("nodes that pass both ... are returned to
+ * the healthy pool", Sec. 5.4).  th->dir/thr/floor_rel/floor_abs are used; the other
+ * fields are ignored.  Outputs ("or NULL"): d_gpu_med[G][M], d_fleet_med/mad/cut[M],
+ * d_fail_mask[G], d_gpu_pass[G], d_node_pass[nodes].  d_status: device uint32 or NULL,
+ * receives sticky status bits (1 = non-finite input, 2 = wait ran out, 4 = internal).
+ */
+int guard_sweep_qualify(const float *d_S, int nodes, int gpus_per_node, int reps, int metrics,
+                        const guard_thresholds *th, int32_t pct_ppm, void *d_workspace, size_t workspace_bytes,
+                        float *d_gpu_med, float *d_fleet_med, float *d_fleet_mad, float *d_fleet_cut,
+                        uint32_t *d_fail_mask, uint8_t *d_gpu_pass, uint8_t *d_node_pass, uint32_t *d_status,
+                        void *stream);
+
+/* Synchronises `stream` and returns the sticky device status of the context
+ * (GUARD_OK, GUARD_ERR_NONFINITE, GUARD_ERR_TIMEOUT, GUARD_ERR_INTERNAL, GUARD_ERR_CUDA). */
+int guard_sync_status(guard_ctx *ctx, void *stream);
+
+/* Clears the ring position, exceedance ring, consecutive counters and status. */
+int guard_reset(guard_ctx *ctx, void *stream);
+
+/* Steps ingested since creation or the last reset. */
+int64_t guard_steps_seen(const guard_ctx *ctx);
+
+/* Frees the host object (the workspace stays the caller's). NULL is allowed. */
+void guard_destroy(guard_ctx *ctx);
+
+/* Text of the last host-side error of this context (or of the last failed
+ * guard_create / guard_sweep_qualify when ctx is NULL).  Never NULL. */
+const char *guard_last_error(const guard_ctx *ctx);
+
+/* Host helper: the order-preserving float32 -> uint32 key the kernels select on
+ * (total order of finite floats equals unsigned order of keys), and its inverse. */
+uint32_t guard_key_from_float(float x);
+float guard_float_from_key(uint32_t key);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GUARD_B200_H */

@@ -1,0 +1,114 @@
+// Per-thread exact selection inside a strided shared-memory column, and the bulk-copy
+// (TMA) / mbarrier primitives used to stage the tiles those columns live in.
+#pragma once
+#include "common.cuh"
+
+namespace guard {
+
+// ---- selection ------------------------------------------------------------------------
+
+// k-th smallest (0-based) of col[0], col[stride], ..., col[(n-1)*stride] (uint32 keys).
+// Three-way partitioning around a median-of-three pivot; the column is permuted in
+// place (its multiset is preserved).  Each thread owns its column, so no barrier is
+// needed; with one column per lane and a row pitch that is a multiple of 32 words every
+// access of a warp is free of bank conflicts.
+__device__ __forceinline__ uint32_t col_select(uint32_t *col, int stride, int n, int k) {
+    int l = 0, r = n - 1;
+    while (l < r) {
+        const uint32_t a = col[(size_t)l * stride], b = col[(size_t)((l + r) >> 1) * stride],
+                       c = col[(size_t)r * stride];
+        const uint32_t p = max(min(a, b), min(max(a, b), c));
+        int store = l, ceq = 0;
+        for (int i = l; i <= r; ++i) {
+            const uint32_t v = col[(size_t)i * stride];
+            if (v < p) {
+                col[(size_t)i * stride] = col[(size_t)store * stride];
+                col[(size_t)store * stride] = v;
+                ++store;
+            }
+            ceq += (v == p);
+        }
+        if (k < store) {
+            r = store - 1;
+        } else if (k < store + ceq) {
+            return p;
+        } else {
+            int s2 = store;
+            for (int i = store; i <= r; ++i) {
+                const uint32_t v = col[(size_t)i * stride];
+                if (v == p) {
+                    col[(size_t)i * stride] = col[(size_t)s2 * stride];
+                    col[(size_t)s2 * stride] = v;
+                    ++s2;
+                }
+            }
+            l = s2;
+        }
+    }
+    return col[(size_t)l * stride];
+}
+
+// Given v = the key of 0-based rank k, the key of rank k + 1: v again if more than k + 1
+// keys are <= v, else the smallest key above v.
+__device__ __forceinline__ uint32_t col_next(const uint32_t *col, int stride, int n, int k, uint32_t v) {
+    int cle = 0;
+    uint32_t above = 0xFFFFFFFFu;
+    for (int i = 0; i < n; ++i) {
+        const uint32_t x = col[(size_t)i * stride];
+        cle += (x <= v);
+        if (x > v) above = min(above, x);
+    }
+    return (cle > k + 1) ? v : above;
+}
+
+// Median of a column of keys (midpoint rule for even n).
+__device__ __forceinline__ float col_median(uint32_t *col, int stride, int n) {
+    const int k = (n - 1) >> 1;
+    const uint32_t v1 = col_select(col, stride, n, k);
+    if (n & 1) return key2f(v1);
+    const uint32_t v2 = col_next(col, stride, n, k, v1);
+    return median_from_keys(v1, v2, true);
+}
+
+// ---- bulk async copy (TMA) + mbarrier ---------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Waits for the phase with a time limit (in clock cycles); false if it ran out.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, long long limit_cycles) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > limit_cycles) return false;
+    }
+    return true;
+}
+// 1-D bulk copy global -> shared, completion counted in bytes on the mbarrier.  Both
+// addresses and the size must be multiples of 16 bytes.
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+constexpr long long kWaitLimitCycles = 2000000000LL;  // about one second
+
+}  // namespace guard

@@ -1,0 +1,402 @@
+// C ABI of the library: context object, workspace carving, argument checks and the
+// stream-ordered kernel sequences behind guard_ingest / guard_score / guard_sweep_qualify.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/guard_b200.h"
+#include "kernels.h"
+
+using namespace guard;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+    size_t status, consec, ticket, fleet, wmed, stepstat, topk_cand, mask, ring, total;
+};
+
+// State and scratch first, the two rings last (the telemetry ring is by far the largest).
+Layout make_layout(int R, int M, int C, int K) {
+    Layout L{};
+    size_t off = 0;
+    L.status = off;    off = align_up(off + 64);
+    L.ticket = off;    off = align_up(off + 64);
+    L.fleet = off;     off = align_up(off + 3 * kMaxMetrics * sizeof(float));
+    L.consec = off;    off = align_up(off + (size_t)R);
+    L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
+    L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
+    L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
+    L.mask = off;      off = align_up(off + (size_t)C * R * (M <= 8 ? 1 : 4));
+    L.ring = off;      off = align_up(off + (size_t)C * R * M * sizeof(float));
+    L.total = off;
+    return L;
+}
+
+bool sizes_ok(int R, int M, int W, int C, int K) {
+    return R >= 1 && M >= 1 && M <= GUARD_MAX_METRICS && W >= 1 && W <= GUARD_MAX_WINDOW && C >= W && K >= 0 &&
+           K <= GUARD_MAX_TOPK && K <= R && (long long)R * M <= 0x7FFFFFFFLL;
+}
+
+thread_local char g_error[256] = "";
+
+void set_error(char *dst, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(dst, 256, fmt, ap);
+    va_end(ap);
+}
+
+// Copies and checks the per-metric parameters; returns nullptr or an error text.
+const char *fill_params(MetricParams &p, const guard_thresholds *th, int M, int k, bool online) {
+    if (!th || !th->dir || !th->thr || !th->floor_rel || !th->floor_abs) return "thresholds or one of its arrays is NULL";
+    memset(&p, 0, sizeof(p));
+    p.M = M;
+    p.k = k;
+    p.primary = th->primary;
+    p.min_signals = th->min_signals;
+    p.n_consec = th->n_consec;
+    p.tier_moderate = th->tier_moderate;
+    p.tier_severe = th->tier_severe;
+    if (online) {
+        if (th->primary < 0 || th->primary >= M) return "primary metric index out of range";
+        if (th->min_signals < 1) return "min_signals must be >= 1";
+        if (th->n_consec < 1 || th->n_consec > 255) return "n_consec must be in 1..255";
+        if (!(th->tier_moderate >= 0.0f) || !(th->tier_severe >= th->tier_moderate)) return "tier thresholds must satisfy 0 <= moderate <= severe";
+    }
+    for (int m = 0; m < M; ++m) {
+        if (th->dir[m] != 1 && th->dir[m] != -1) return "dir[m] must be +1 or -1";
+        if (!(th->thr[m] >= 0.0f) || !(th->thr[m] < 1e30f)) return "thr[m] must be finite and >= 0";
+        if (!(th->floor_rel[m] >= 0.0f) || !(th->floor_abs[m] >= 0.0f)) return "floors must be >= 0";
+        p.dir[m] = th->dir[m];
+        p.thrp[m] = (float)((double)th->thr[m] / 0.6745);
+        p.floor_rel[m] = th->floor_rel[m];
+        p.floor_abs[m] = th->floor_abs[m];
+    }
+    return nullptr;
+}
+
+int status_to_code(uint32_t s) {
+    if (s & kStatNonFinite) return GUARD_ERR_NONFINITE;
+    if (s & kStatTimeout) return GUARD_ERR_TIMEOUT;
+    if (s & kStatInternal) return GUARD_ERR_INTERNAL;
+    return GUARD_OK;
+}
+
+}  // namespace
+
+struct guard_ctx {
+    int R, M, W, k, C, K;
+    MetricParams p;
+    Layout L;
+    char *ws;
+    long long seen;
+    char error[256];
+
+    uint32_t *status() const { return (uint32_t *)(ws + L.status); }
+    unsigned int *ticket() const { return (unsigned int *)(ws + L.ticket); }
+    float *fleet_med() const { return (float *)(ws + L.fleet); }
+    float *fleet_mad() const { return fleet_med() + kMaxMetrics; }
+    uint8_t *consec() const { return (uint8_t *)(ws + L.consec); }
+    float *wmed() const { return (float *)(ws + L.wmed); }
+    float *step_med() const { return (float *)(ws + L.stepstat); }
+    float *step_mad() const { return step_med() + (size_t)C * M; }
+    unsigned long long *topk_cand() const { return (unsigned long long *)(ws + L.topk_cand); }
+    void *mask() const { return ws + L.mask; }
+    float *ring() const { return (float *)(ws + L.ring); }
+    int mask_bytes() const { return M <= 8 ? 1 : 4; }
+    int fail(int code, const char *fmt, ...) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(error, sizeof(error), fmt, ap);
+        va_end(ap);
+        return code;
+    }
+    int cuda_fail(cudaError_t e, const char *what) { return fail(GUARD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e)); }
+};
+
+extern "C" {
+
+size_t guard_workspace_bytes(int ranks, int metrics, int W, int capacity_steps, int topk) {
+    if (!sizes_ok(ranks, metrics, W, capacity_steps, topk)) return 0;
+    return make_layout(ranks, metrics, capacity_steps, topk).total;
+}
+
+int guard_create(guard_ctx **out, int ranks, int metrics, int W, int k, const guard_thresholds *th, int capacity_steps,
+                 int topk, void *d_workspace, size_t workspace_bytes, void *stream) {
+    if (!out) { set_error(g_error, "out is NULL"); return GUARD_ERR_ARG; }
+    *out = nullptr;
+    if (!sizes_ok(ranks, metrics, W, capacity_steps, topk)) {
+        set_error(g_error, "invalid sizes: need ranks >= 1, 1 <= metrics <= %d, 1 <= W <= %d, capacity >= W, 0 <= topk <= min(ranks, %d)",
+                  GUARD_MAX_METRICS, GUARD_MAX_WINDOW, GUARD_MAX_TOPK);
+        return GUARD_ERR_ARG;
+    }
+    if (k < 1 || k > W) { set_error(g_error, "k must be in 1..W"); return GUARD_ERR_ARG; }
+    MetricParams p;
+    if (const char *msg = fill_params(p, th, metrics, k, true)) { set_error(g_error, "%s", msg); return GUARD_ERR_ARG; }
+    const Layout L = make_layout(ranks, metrics, capacity_steps, topk);
+    if (!d_workspace || ((uintptr_t)d_workspace % kAlign) != 0 || workspace_bytes < L.total) {
+        set_error(g_error, "workspace must be non-NULL, 256-byte aligned and at least %zu bytes", L.total);
+        return GUARD_ERR_WORKSPACE;
+    }
+    guard_ctx *c = new (std::nothrow) guard_ctx();
+    if (!c) { set_error(g_error, "out of host memory"); return GUARD_ERR_ARG; }
+    c->R = ranks; c->M = metrics; c->W = W; c->k = k; c->C = capacity_steps; c->K = topk;
+    c->p = p; c->L = L; c->ws = (char *)d_workspace; c->seen = 0; c->error[0] = 0;
+    // state: status word, ticket, fleet statistics, consecutive counters
+    cudaError_t e = cudaMemsetAsync(c->ws, 0, L.wmed, (cudaStream_t)stream);
+    if (e != cudaSuccess) {
+        set_error(g_error, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+        delete c;
+        return GUARD_ERR_CUDA;
+    }
+    *out = c;
+    return GUARD_OK;
+}
+
+int guard_ring_reserve(guard_ctx *c, int steps, float **d_slot) {
+    if (!c) return GUARD_ERR_ARG;
+    if (!d_slot || steps < 1 || steps > c->C) return c->fail(GUARD_ERR_ARG, "steps must be in 1..capacity and d_slot non-NULL");
+    const int slot = (int)(c->seen % c->C);
+    if (slot + steps > c->C) return c->fail(GUARD_ERR_ARG, "reserved span would wrap around the ring (slot %d + %d > %d)", slot, steps, c->C);
+    *d_slot = c->ring() + (size_t)slot * c->R * c->M;
+    return GUARD_OK;
+}
+
+int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, float *d_step_mad, void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    if (!d_block) return c->fail(GUARD_ERR_ARG, "d_block is NULL");
+    if (B < 1 || B > c->C) return c->fail(GUARD_ERR_ARG, "B must be in 1..capacity_steps (%d)", c->C);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t row = (size_t)c->R * c->M;
+    const int slot = (int)(c->seen % c->C);
+    const bool in_place = (d_block == c->ring() + (size_t)slot * row) && (slot + B <= c->C);
+    if (!in_place) {
+        const int first = (slot + B <= c->C) ? B : (c->C - slot);
+        cudaError_t e = cudaMemcpyAsync(c->ring() + (size_t)slot * row, d_block, (size_t)first * row * sizeof(float),
+                                        cudaMemcpyDeviceToDevice, st);
+        if (e == cudaSuccess && first < B)
+            e = cudaMemcpyAsync(c->ring(), d_block + (size_t)first * row, (size_t)(B - first) * row * sizeof(float),
+                                cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) return c->cuda_fail(e, "cudaMemcpyAsync(ring)");
+    }
+    XrankArgs a{};
+    a.base = c->ring();
+    a.row_stride = (long long)row;
+    a.first_slot = slot;
+    a.capacity = c->C;
+    a.R = c->R;
+    a.M = c->M;
+    a.med = c->step_med();
+    a.mad = c->step_mad();
+    a.med_user = d_step_med;
+    a.mad_user = d_step_mad;
+    a.cut = nullptr;
+    a.mask_base = c->mask();
+    a.mask_bytes = c->mask_bytes();
+    a.check_finite = 1;
+    a.status = c->status();
+    cudaError_t e = launch_xrank_direct(a, c->p, B, st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "xrank launch");
+    c->seen += B;
+    return GUARD_OK;
+}
+
+int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_mad, float *d_scores, uint16_t *d_counts,
+                uint32_t *d_metric_mask, uint8_t *d_flags, uint8_t *d_tier, int32_t *d_topk_idx, float *d_topk_score,
+                void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    if (c->seen < 1) return c->fail(GUARD_ERR_NOT_READY, "guard_score before the first ingested step");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int n = (int)(c->seen < c->W ? c->seen : c->W);
+    const int last = (int)((c->seen - 1) % c->C);
+    const size_t row = (size_t)c->R * c->M;
+
+    WindowArgs w{};
+    w.ring = c->ring();
+    w.row_stride = (long long)row;
+    w.capacity = c->C;
+    w.last_slot = last;
+    w.n = n;
+    w.series = (int)row;
+    w.wmed = c->wmed();
+    w.wmed_user = d_wmed;
+    w.status = c->status();
+    cudaError_t e = launch_window_select(w, st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "window_select launch");
+
+    XrankArgs x{};
+    x.base = c->wmed();
+    x.row_stride = (long long)row;
+    x.first_slot = 0;
+    x.capacity = 1;
+    x.R = c->R;
+    x.M = c->M;
+    x.med = c->fleet_med();
+    x.mad = c->fleet_mad();
+    x.med_user = d_fleet_med;
+    x.mad_user = d_fleet_mad;
+    x.status = c->status();
+    e = launch_xrank_direct(x, c->p, 1, st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "fleet baseline launch");
+
+    ScoreArgs s{};
+    s.R = c->R;
+    s.M = c->M;
+    s.wmed = c->wmed();
+    s.fleet_med = c->fleet_med();
+    s.fleet_mad = c->fleet_mad();
+    s.mask_base = c->mask();
+    s.mask_bytes = c->mask_bytes();
+    s.capacity = c->C;
+    s.last_slot = last;
+    s.n = n;
+    s.consec = c->consec();
+    s.scores = d_scores;
+    s.counts = d_counts;
+    s.metric_mask = d_metric_mask;
+    s.flags = d_flags;
+    s.tier = d_tier;
+    e = launch_score_flag(s, c->p, st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
+
+    if (c->K > 0 && (d_topk_idx || d_topk_score)) {
+        TopkArgs t{};
+        t.R = c->R;
+        t.M = c->M;
+        t.K = c->K;
+        t.wmed = c->wmed();
+        t.fleet_med = c->fleet_med();
+        t.fleet_mad = c->fleet_mad();
+        t.cand = c->topk_cand();
+        t.ticket = c->ticket();
+        t.idx = d_topk_idx;
+        t.score = d_topk_score;
+        e = launch_topk(t, c->p, st);
+        if (e != cudaSuccess) return c->cuda_fail(e, "topk launch");
+    }
+    return GUARD_OK;
+}
+
+size_t guard_sweep_workspace_bytes(int gpus, int reps, int metrics) {
+    if (gpus < 1 || reps < 1 || reps > GUARD_MAX_WINDOW || metrics < 1 || metrics > GUARD_MAX_METRICS ||
+        (long long)gpus * metrics > 0x7FFFFFFFLL)
+        return 0;
+    return align_up(3 * kMaxMetrics * sizeof(float)) + align_up((size_t)gpus * metrics * sizeof(float));
+}
+
+int guard_sweep_qualify(const float *d_S, int nodes, int gpus_per_node, int reps, int metrics, const guard_thresholds *th,
+                        int32_t pct_ppm, void *d_workspace, size_t workspace_bytes, float *d_gpu_med, float *d_fleet_med,
+                        float *d_fleet_mad, float *d_fleet_cut, uint32_t *d_fail_mask, uint8_t *d_gpu_pass,
+                        uint8_t *d_node_pass, uint32_t *d_status, void *stream) {
+    if (!d_S || nodes < 1 || gpus_per_node < 1 || (long long)nodes * gpus_per_node > 0x7FFFFFFFLL) {
+        set_error(g_error, "d_S is NULL or nodes / gpus_per_node out of range");
+        return GUARD_ERR_ARG;
+    }
+    const int G = nodes * gpus_per_node;
+    const size_t need = guard_sweep_workspace_bytes(G, reps, metrics);
+    if (need == 0) { set_error(g_error, "invalid sweep sizes"); return GUARD_ERR_ARG; }
+    if (pct_ppm < 0 || pct_ppm > 1000000) { set_error(g_error, "pct_ppm must be in 0..1000000"); return GUARD_ERR_ARG; }
+    MetricParams p;
+    if (const char *msg = fill_params(p, th, metrics, 1, false)) { set_error(g_error, "%s", msg); return GUARD_ERR_ARG; }
+    if (!d_workspace || ((uintptr_t)d_workspace % kAlign) != 0 || workspace_bytes < need) {
+        set_error(g_error, "sweep workspace must be non-NULL, 256-byte aligned and at least %zu bytes", need);
+        return GUARD_ERR_WORKSPACE;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    float *fleet = (float *)d_workspace;
+    float *gmed = (float *)((char *)d_workspace + align_up(3 * kMaxMetrics * sizeof(float)));
+
+    SweepMedArgs sm{};
+    sm.S = d_S;
+    sm.G = G;
+    sm.reps = reps;
+    sm.M = metrics;
+    sm.gmed = gmed;
+    sm.gmed_user = d_gpu_med;
+    sm.status = d_status;
+    cudaError_t e = launch_sweep_medians(sm, st);
+    if (e != cudaSuccess) { set_error(g_error, "sweep medians launch: %s", cudaGetErrorString(e)); return GUARD_ERR_CUDA; }
+
+    // nearest-rank percentile of the bad tail: the j-th worst of G values
+    long long j = ((long long)pct_ppm * G + 999999) / 1000000;
+    if (j < 1) j = 1;
+    if (j > G) j = G;
+    XrankArgs x{};
+    x.base = gmed;
+    x.row_stride = (long long)G * metrics;
+    x.first_slot = 0;
+    x.capacity = 1;
+    x.R = G;
+    x.M = metrics;
+    x.med = fleet;
+    x.mad = fleet + kMaxMetrics;
+    x.cut = fleet + 2 * kMaxMetrics;
+    x.med_user = d_fleet_med;
+    x.mad_user = d_fleet_mad;
+    for (int m = 0; m < metrics; ++m) x.cut_rank[m] = p.dir[m] < 0 ? (int)(j - 1) : (int)(G - j);
+    x.status = d_status;
+    e = launch_xrank_direct(x, p, 1, st);
+    if (e != cudaSuccess) { set_error(g_error, "sweep fleet statistics launch: %s", cudaGetErrorString(e)); return GUARD_ERR_CUDA; }
+    if (d_fleet_cut) {
+        e = cudaMemcpyAsync(d_fleet_cut, fleet + 2 * kMaxMetrics, metrics * sizeof(float), cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) { set_error(g_error, "cudaMemcpyAsync: %s", cudaGetErrorString(e)); return GUARD_ERR_CUDA; }
+    }
+    SweepVerdictArgs v{};
+    v.nodes = nodes;
+    v.gpus_per_node = gpus_per_node;
+    v.M = metrics;
+    v.gmed = gmed;
+    v.fleet_med = fleet;
+    v.fleet_mad = fleet + kMaxMetrics;
+    v.fleet_cut = fleet + 2 * kMaxMetrics;
+    v.fail_mask = d_fail_mask;
+    v.gpu_pass = d_gpu_pass;
+    v.node_pass = d_node_pass;
+    e = launch_sweep_verdict(v, p, st);
+    if (e != cudaSuccess) { set_error(g_error, "sweep verdict launch: %s", cudaGetErrorString(e)); return GUARD_ERR_CUDA; }
+    return GUARD_OK;
+}
+
+int guard_sync_status(guard_ctx *c, void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    uint32_t s = 0;
+    cudaError_t e = cudaMemcpyAsync(&s, c->status(), sizeof(s), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_sync_status");
+    const int code = status_to_code(s);
+    if (code != GUARD_OK) c->fail(code, "device status word 0x%x", s);
+    return code;
+}
+
+int guard_reset(guard_ctx *c, void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    cudaError_t e = cudaMemsetAsync(c->ws, 0, c->L.wmed, (cudaStream_t)stream);
+    if (e != cudaSuccess) return c->cuda_fail(e, "cudaMemsetAsync");
+    c->seen = 0;
+    return GUARD_OK;
+}
+
+int64_t guard_steps_seen(const guard_ctx *c) { return c ? c->seen : 0; }
+
+void guard_destroy(guard_ctx *c) { delete c; }
+
+const char *guard_last_error(const guard_ctx *c) { return c ? c->error : g_error; }
+
+uint32_t guard_key_from_float(float x) {
+    uint32_t b;
+    memcpy(&b, &x, 4);
+    return key_of_bits(b);
+}
+
+float guard_float_from_key(uint32_t key) {
+    const uint32_t b = bits_of_key(key);
+    float x;
+    memcpy(&x, &b, 4);
+    return x;
+}
+
+}  // extern "C"

@@ -1,0 +1,96 @@
+// Host-side launchers of the scoring kernels (internal to the library).
+#pragma once
+#include "common.cuh"
+
+namespace guard {
+
+// Cross-rank statistics of S rows of a [rows][R][M] float32 array.  Row s of the launch
+// lives at base + ((first_slot + s) % capacity) * row_stride.
+struct XrankArgs {
+    const float *base;
+    long long row_stride;   // floats between consecutive rows (R * M)
+    int first_slot;
+    int capacity;
+    int R, M;
+    float *med;             // [S][M] cross-rank median (never NULL)
+    float *mad;             // [S][M] raw MAD about that median (never NULL)
+    float *med_user;        // [S][M] copy for the caller, or NULL
+    float *mad_user;        // [S][M] copy for the caller, or NULL
+    float *cut;             // [S][M] extra order statistic (0-based rank cut_rank[m]), or NULL
+    int cut_rank[kMaxMetrics];
+    void *mask_base;        // exceedance mask rows [capacity][R] of mask_bytes each, or NULL
+    int mask_bytes;         // 1 (M <= 8) or 4
+    int check_finite;       // flag NaN / Inf in the status word
+    uint32_t *status;
+};
+
+cudaError_t launch_xrank_direct(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st);
+
+// Windowed per-series median over the last n ring rows ending at slot `last_slot`.
+struct WindowArgs {
+    const float *ring;
+    long long row_stride;   // R * M
+    int capacity;
+    int last_slot;          // slot of the newest step
+    int n;                  // window length in steps
+    int series;             // R * M
+    float *wmed;            // [series] (never NULL)
+    float *wmed_user;       // or NULL
+    uint32_t *status;
+};
+cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st);
+
+// Fused k-of-W count, robust score, thresholds, multi-signal flag, tier, consecutive counter.
+struct ScoreArgs {
+    int R, M;
+    const float *wmed;       // [R][M]
+    const float *fleet_med;  // [M]
+    const float *fleet_mad;  // [M]
+    const void *mask_base;   // exceedance rows [capacity][R]
+    int mask_bytes;
+    int capacity;
+    int last_slot;
+    int n;                   // window length
+    uint8_t *consec;         // [R] state
+    float *scores;           // [R][M] or NULL
+    uint16_t *counts;        // [R][M] or NULL
+    uint32_t *metric_mask;   // [R] or NULL
+    uint8_t *flags;          // [R] or NULL
+    uint8_t *tier;           // [R] or NULL
+};
+cudaError_t launch_score_flag(const ScoreArgs &a, const MetricParams &p, cudaStream_t st);
+
+// Block-then-grid top-k of dir * wmed[:, primary].
+struct TopkArgs {
+    int R, M, K;
+    const float *wmed;
+    const float *fleet_med;
+    const float *fleet_mad;
+    unsigned long long *cand;   // scratch [topk_blocks(R)][K]
+    unsigned int *ticket;       // scratch, zero before first use (self-resetting)
+    int32_t *idx;               // [K] or NULL
+    float *score;               // [K] or NULL
+};
+int topk_blocks(int R);
+cudaError_t launch_topk(const TopkArgs &a, const MetricParams &p, cudaStream_t st);
+
+// Node sweep: per-GPU medians over repetitions, then the verdicts.
+struct SweepMedArgs {
+    const float *S;   // [G][reps][M]
+    int G, reps, M;
+    float *gmed;      // [G][M]
+    float *gmed_user; // or NULL
+    uint32_t *status; // or NULL
+};
+cudaError_t launch_sweep_medians(const SweepMedArgs &a, cudaStream_t st);
+
+struct SweepVerdictArgs {
+    int nodes, gpus_per_node, M;
+    const float *gmed, *fleet_med, *fleet_mad, *fleet_cut;
+    uint32_t *fail_mask;  // or NULL
+    uint8_t *gpu_pass;    // or NULL
+    uint8_t *node_pass;   // or NULL
+};
+cudaError_t launch_sweep_verdict(const SweepVerdictArgs &a, const MetricParams &p, cudaStream_t st);
+
+}  // namespace guard

@@ -1,0 +1,267 @@
+"""Thin ctypes binding of libguard_b200.so (the C ABI declared in include/guard_b200.h).
+
+Argument marshalling only: every step of the scoring path runs in the library's CUDA
+kernels.  PyTorch supplies device memory (the workspace and the output tensors) and the
+current CUDA stream.  There is no CPU fallback: if the library has not been built the
+import of this module's functions fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libguard_b200.so")
+
+GUARD_OK = 0
+ERR_NAMES = {0: "GUARD_OK", -1: "GUARD_ERR_ARG", -2: "GUARD_ERR_WORKSPACE", -3: "GUARD_ERR_NOT_READY",
+             -4: "GUARD_ERR_NONFINITE", -5: "GUARD_ERR_TIMEOUT", -6: "GUARD_ERR_CUDA", -7: "GUARD_ERR_INTERNAL"}
+MAX_METRICS, MAX_TOPK, MAX_WINDOW = 32, 1024, 65535
+
+
+class GuardError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__("%s (%d): %s" % (ERR_NAMES.get(code, "?"), code, text))
+        self.code = code
+
+
+class _Thresholds(C.Structure):
+    _fields_ = [("primary", C.c_int32), ("min_signals", C.c_int32), ("n_consec", C.c_int32),
+                ("ranks_per_node", C.c_int32), ("tier_moderate", C.c_float), ("tier_severe", C.c_float),
+                ("dir", C.POINTER(C.c_int8)), ("thr", C.POINTER(C.c_float)),
+                ("floor_rel", C.POINTER(C.c_float)), ("floor_abs", C.POINTER(C.c_float))]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libguard_b200.so is missing: build it with paper_2605_17879_b200.build.build_library() "
+                               "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, fp = C.c_void_p, C.c_void_p  # device pointers travel as integers
+        L.guard_workspace_bytes.restype = C.c_size_t
+        L.guard_workspace_bytes.argtypes = [C.c_int] * 5
+        L.guard_create.restype = C.c_int
+        L.guard_create.argtypes = [C.POINTER(vp), C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(_Thresholds),
+                                   C.c_int, C.c_int, vp, C.c_size_t, vp]
+        L.guard_ring_reserve.restype = C.c_int
+        L.guard_ring_reserve.argtypes = [vp, C.c_int, C.POINTER(vp)]
+        L.guard_ingest.restype = C.c_int
+        L.guard_ingest.argtypes = [vp, fp, C.c_int, fp, fp, vp]
+        L.guard_score.restype = C.c_int
+        L.guard_score.argtypes = [vp] + [fp] * 10 + [vp]
+        L.guard_sweep_workspace_bytes.restype = C.c_size_t
+        L.guard_sweep_workspace_bytes.argtypes = [C.c_int] * 3
+        L.guard_sweep_qualify.restype = C.c_int
+        L.guard_sweep_qualify.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(_Thresholds), C.c_int32,
+                                          vp, C.c_size_t] + [fp] * 8 + [vp]
+        L.guard_sync_status.restype = C.c_int
+        L.guard_sync_status.argtypes = [vp, vp]
+        L.guard_reset.restype = C.c_int
+        L.guard_reset.argtypes = [vp, vp]
+        L.guard_steps_seen.restype = C.c_int64
+        L.guard_steps_seen.argtypes = [vp]
+        L.guard_destroy.restype = None
+        L.guard_destroy.argtypes = [vp]
+        L.guard_last_error.restype = C.c_char_p
+        L.guard_last_error.argtypes = [vp]
+        L.guard_key_from_float.restype = C.c_uint32
+        L.guard_key_from_float.argtypes = [C.c_float]
+        L.guard_float_from_key.restype = C.c_float
+        L.guard_float_from_key.argtypes = [C.c_uint32]
+        _lib = L
+    return _lib
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, numel: Optional[int] = None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("expected dtype %s, got %s" % (dtype, t.dtype))
+    if numel is not None and t.numel() < numel:
+        raise ValueError("tensor too small: %d < %d elements" % (t.numel(), numel))
+    return t.data_ptr()
+
+
+class _Params:
+    """Host-side arrays behind a guard_thresholds struct (kept alive with it)."""
+
+    def __init__(self, metrics, dir, thr, floor_rel, floor_abs, primary=0, min_signals=2, n_consec=1,
+                 ranks_per_node=8, tier_moderate=0.10, tier_severe=0.20):
+        def bc(v, ctype):
+            vals = list(v) if isinstance(v, (list, tuple)) or hasattr(v, "__len__") else [v] * metrics
+            if len(vals) != metrics:
+                raise ValueError("expected %d per-metric values, got %d" % (metrics, len(vals)))
+            return (ctype * metrics)(*vals)
+        self.dir = bc([int(d) for d in dir], C.c_int8)
+        self.thr = bc(thr, C.c_float)
+        self.floor_rel = bc(floor_rel, C.c_float)
+        self.floor_abs = bc(floor_abs, C.c_float)
+        self.struct = _Thresholds(primary, min_signals, n_consec, ranks_per_node, tier_moderate, tier_severe,
+                                  self.dir, self.thr, self.floor_rel, self.floor_abs)
+
+
+def workspace_bytes(ranks: int, metrics: int, W: int, capacity: int, topk: int) -> int:
+    return int(lib().guard_workspace_bytes(ranks, metrics, W, capacity, topk))
+
+
+class Guard:
+    """Online scorer: `ingest` blocks of steps, `score` the current window."""
+
+    def __init__(self, ranks: int, metrics: int, W: int, k: int, *, dir: Sequence[int], thr=3.5, floor_rel=1e-4,
+                 floor_abs=0.0, primary: int = 0, min_signals: int = 2, n_consec: int = 1, ranks_per_node: int = 8,
+                 tier_moderate: float = 0.10, tier_severe: float = 0.20, capacity: Optional[int] = None, topk: int = 0,
+                 device="cuda", workspace: Optional[torch.Tensor] = None):
+        self.R, self.M, self.W, self.k, self.K = ranks, metrics, W, k, topk
+        self.C = capacity if capacity is not None else W
+        self.device = torch.device(device)
+        self._h = C.c_void_p()
+        self._params = _Params(metrics, dir, thr, floor_rel, floor_abs, primary, min_signals, n_consec,
+                               ranks_per_node, tier_moderate, tier_severe)
+        need = workspace_bytes(ranks, metrics, W, self.C, topk)
+        if need == 0:
+            raise GuardError(-1, "invalid sizes (ranks=%d metrics=%d W=%d capacity=%d topk=%d)" % (ranks, metrics, W, self.C, topk))
+        if workspace is None:
+            workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        self.workspace = workspace
+        with torch.cuda.device(self.device):
+            rc = lib().guard_create(C.byref(self._h), ranks, metrics, W, k, C.byref(self._params.struct), self.C, topk,
+                                    _ptr(workspace, torch.uint8), workspace.numel(), _stream())
+        if rc != GUARD_OK:
+            raise GuardError(rc, lib().guard_last_error(None).decode())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().guard_destroy(self._h)
+            self._h = C.c_void_p()
+
+    __del__ = close
+
+    def _check(self, rc: int):
+        if rc != GUARD_OK:
+            raise GuardError(rc, lib().guard_last_error(self._h).decode())
+
+    @property
+    def steps_seen(self) -> int:
+        return int(lib().guard_steps_seen(self._h))
+
+    def ring_reserve(self, steps: int) -> torch.Tensor:
+        """View [steps, ranks, metrics] of the ring slots the next `steps` steps occupy."""
+        p = C.c_void_p()
+        self._check(lib().guard_ring_reserve(self._h, steps, C.byref(p)))
+        off = p.value - self.workspace.data_ptr()
+        nbytes = steps * self.R * self.M * 4
+        return self.workspace[off:off + nbytes].view(torch.float32).view(steps, self.R, self.M)
+
+    def ingest(self, block: torch.Tensor, step_med: Optional[torch.Tensor] = None,
+               step_mad: Optional[torch.Tensor] = None) -> None:
+        if block.dim() != 3 or block.shape[1] != self.R or block.shape[2] != self.M:
+            raise ValueError("block must be [B, %d, %d]" % (self.R, self.M))
+        B = block.shape[0]
+        with torch.cuda.device(self.device):
+            self._check(lib().guard_ingest(self._h, _ptr(block, torch.float32), B,
+                                           _ptr(step_med, torch.float32, B * self.M),
+                                           _ptr(step_mad, torch.float32, B * self.M), _stream()))
+
+    def alloc_outputs(self) -> Dict[str, torch.Tensor]:
+        R, M, K, dev = self.R, self.M, self.K, self.device
+        return {
+            "wmed": torch.empty((R, M), dtype=torch.float32, device=dev),
+            "fleet_med": torch.empty(M, dtype=torch.float32, device=dev),
+            "fleet_mad": torch.empty(M, dtype=torch.float32, device=dev),
+            "scores": torch.empty((R, M), dtype=torch.float32, device=dev),
+            "counts": torch.empty((R, M), dtype=torch.uint16, device=dev),
+            "mask": torch.empty(R, dtype=torch.uint32, device=dev),
+            "flags": torch.empty(R, dtype=torch.uint8, device=dev),
+            "tier": torch.empty(R, dtype=torch.uint8, device=dev),
+            "topk_idx": torch.empty(K, dtype=torch.int32, device=dev),
+            "topk_score": torch.empty(K, dtype=torch.float32, device=dev),
+        }
+
+    def score(self, out: Optional[Dict[str, Optional[torch.Tensor]]] = None) -> Dict[str, Optional[torch.Tensor]]:
+        """One evaluation; `out` maps output names to tensors (missing / None entries are skipped)."""
+        if out is None:
+            out = self.alloc_outputs()
+        g = out.get
+        R, M, K = self.R, self.M, self.K
+        with torch.cuda.device(self.device):
+            self._check(lib().guard_score(
+                self._h, _ptr(g("wmed"), torch.float32, R * M), _ptr(g("fleet_med"), torch.float32, M),
+                _ptr(g("fleet_mad"), torch.float32, M), _ptr(g("scores"), torch.float32, R * M),
+                _ptr(g("counts"), torch.uint16, R * M), _ptr(g("mask"), torch.uint32, R),
+                _ptr(g("flags"), torch.uint8, R), _ptr(g("tier"), torch.uint8, R),
+                _ptr(g("topk_idx"), torch.int32, K) if K else None,
+                _ptr(g("topk_score"), torch.float32, K) if K else None, _stream()))
+        return out
+
+    def sync_status(self) -> int:
+        """Synchronises the current stream; raises GuardError on a sticky device error."""
+        with torch.cuda.device(self.device):
+            rc = lib().guard_sync_status(self._h, _stream())
+        self._check(rc)
+        return rc
+
+    def reset(self) -> None:
+        with torch.cuda.device(self.device):
+            self._check(lib().guard_reset(self._h, _stream()))
+
+
+def sweep_qualify(S: torch.Tensor, nodes: int, gpus_per_node: int, *, dir: Sequence[int], thr=3.5, floor_rel=1e-4,
+                  floor_abs=0.0, pct_ppm: int = 50_000, workspace: Optional[torch.Tensor] = None,
+                  out: Optional[Dict[str, Optional[torch.Tensor]]] = None) -> Dict[str, Optional[torch.Tensor]]:
+    """Node-sweep qualification of S[gpu, rep, metric]; returns the output tensors plus 'status'."""
+    if S.dim() != 3 or S.shape[0] != nodes * gpus_per_node:
+        raise ValueError("S must be [nodes * gpus_per_node, reps, metrics]")
+    G, reps, M = S.shape
+    dev = S.device
+    params = _Params(M, dir, thr, floor_rel, floor_abs)
+    need = int(lib().guard_sweep_workspace_bytes(G, reps, M))
+    if need == 0:
+        raise GuardError(-1, "invalid sweep sizes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    if out is None:
+        out = {
+            "gpu_med": torch.empty((G, M), dtype=torch.float32, device=dev),
+            "fleet_med": torch.empty(M, dtype=torch.float32, device=dev),
+            "fleet_mad": torch.empty(M, dtype=torch.float32, device=dev),
+            "fleet_cut": torch.empty(M, dtype=torch.float32, device=dev),
+            "fail_mask": torch.empty(G, dtype=torch.uint32, device=dev),
+            "gpu_pass": torch.empty(G, dtype=torch.uint8, device=dev),
+            "node_pass": torch.empty(nodes, dtype=torch.uint8, device=dev),
+            "status": torch.zeros(1, dtype=torch.uint32, device=dev),
+        }
+    g = out.get
+    with torch.cuda.device(dev):
+        rc = lib().guard_sweep_qualify(
+            _ptr(S, torch.float32), nodes, gpus_per_node, reps, M, C.byref(params.struct), pct_ppm,
+            _ptr(workspace, torch.uint8), workspace.numel(), _ptr(g("gpu_med"), torch.float32, G * M),
+            _ptr(g("fleet_med"), torch.float32, M), _ptr(g("fleet_mad"), torch.float32, M),
+            _ptr(g("fleet_cut"), torch.float32, M), _ptr(g("fail_mask"), torch.uint32, G),
+            _ptr(g("gpu_pass"), torch.uint8, G), _ptr(g("node_pass"), torch.uint8, nodes),
+            _ptr(g("status"), torch.uint32, 1), _stream())
+    if rc != GUARD_OK:
+        raise GuardError(rc, lib().guard_last_error(None).decode())
+    return out
+
+
+def key_from_float(x: float) -> int:
+    return int(lib().guard_key_from_float(C.c_float(x)))
+
+
+def float_from_key(k: int) -> float:
+    return float(lib().guard_float_from_key(C.c_uint32(k)))

@@ -1,0 +1,214 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, on the same
+seeded buffers, through the C ABI (via the ctypes binding)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import guard_oracle as go
+from paper_2605_17879_b200 import synth
+from parity_util import assert_bit_equal, compare_score, run_both, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2605_17879_b200 import build
+    build.build_library()
+
+
+def _rand_fleet(T, R, M, seed, quant=None, slow=True):
+    rng = np.random.default_rng(seed)
+    s = np.exp(0.03 * rng.normal(size=(T, R, 1)))
+    X = s * np.exp(0.015 * rng.normal(size=(T, R, M))) * (1.0 + np.arange(M))
+    dirs = [1 if m % 4 != 3 else -1 for m in range(M)]
+    for m in range(M):
+        if dirs[m] < 0:
+            X[..., m] = 100.0 / X[..., m]
+    if slow and R > 3:
+        for r in (1, R // 2):
+            f = 1.25
+            for m in range(M):
+                X[:, r, m] *= f if dirs[m] > 0 else 1 / f
+    if quant:
+        X = np.round(X * quant) / quant
+    return X.astype(np.float32), dirs
+
+
+@pytest.mark.parametrize("R,M,W,k,K,T,blocks,cap", [
+    (64, 4, 50, 30, 8, 200, [50], None),          # shape of the tiny configuration
+    (1, 1, 1, 1, 1, 5, [1], None),                # degenerate: one rank, one metric, window of one
+    (2, 3, 4, 2, 2, 9, [1, 2, 3], 5),             # ring wrap, metrics not a multiple of 4
+    (7, 5, 6, 3, 7, 20, [4], 9),                  # odd rank count, top-k of all ranks
+    (33, 8, 16, 9, 5, 40, [16, 7], 24),
+    (600, 2, 10, 6, 3, 25, [10], 16),             # more ranks than threads in a CTA
+    (130, 9, 12, 7, 4, 30, [5], 16),              # 32-bit exceedance masks (more than 8 metrics)
+    (40, 32, 8, 4, 0, 16, [8], None),             # maximum metric count, no top-k
+    (257, 8, 3, 2, 16, 12, [3], 6),
+])
+def test_small_fleets_match_oracle(R, M, W, k, K, T, blocks, cap):
+    X, dirs = _rand_fleet(T, R, M, seed=R * 1000 + M)
+    run_both(X, W, k, K, dirs, blocks, capacity=cap, min_signals=min(2, M))
+
+
+def test_ties_zero_mad_and_signed_zero():
+    # quantised telemetry: many equal values, MAD of zero, floors binding
+    X, dirs = _rand_fleet(60, 48, 4, seed=5, quant=20)
+    run_both(X, 20, 10, 6, dirs, [20], floor_rel=[0.0, 1e-4, 1e-2, 1e-4], floor_abs=[0.0, 0.0, 0.0, 0.5])
+    # values around zero with both signs and both zeros
+    rng = np.random.default_rng(6)
+    Y = rng.integers(-2, 3, (30, 17, 3)).astype(np.float32)
+    Y[Y == 0] = np.where(rng.random((Y == 0).sum()) < 0.5, 0.0, -0.0)
+    run_both(Y, 10, 5, 17, [1, -1, 1], [5], min_signals=1, floor_rel=0.0)
+    # constant fleet: nothing may be flagged and all scores are zero
+    Z = np.full((12, 16, 4), 1.25, np.float32)
+    last = run_both(Z, 6, 3, 4, [1, 1, 1, -1], [6])
+    assert not last["flags"].any() and not last["mask"].any()
+
+
+def test_wide_dynamic_range():
+    rng = np.random.default_rng(7)
+    X = (rng.standard_cauchy((24, 50, 4)) * 10.0 ** rng.integers(-30, 30, (24, 50, 4))).astype(np.float32)
+    X[~np.isfinite(X)] = 1.0
+    run_both(X, 8, 4, 10, [1, -1, 1, -1], [8], min_signals=1)
+
+
+def test_in_place_ingest_equals_copy_ingest():
+    X, dirs = _rand_fleet(48, 40, 4, seed=8)
+    a = run_both(X, 12, 6, 5, dirs, [12], capacity=24, in_place=True)
+    b = run_both(X, 12, 6, 5, dirs, [12], capacity=24, in_place=False)
+    for key in a:
+        assert np.array_equal(a[key], b[key])
+
+
+def test_long_window_paths():
+    # windows too long for a 128-column tile (64- and 32-column tiles), and the global-memory fallback
+    for W, R in ((500, 24), (1200, 8), (2000, 4)):
+        X, dirs = _rand_fleet(W + 7, R, 4, seed=W)
+        run_both(X, W, W // 2, 2, dirs, [W, 7], capacity=W + 16, score_every=1)
+
+
+def test_consecutive_evaluations_state():
+    X, dirs = _rand_fleet(80, 32, 4, seed=9)
+    run_both(X, 10, 6, 4, dirs, [10], n_consec=3)
+
+
+def test_tiny_configuration_full():
+    cfg = synth.paper_configs()["tiny"]
+    X = synth.fleet_tensor(cfg).numpy()
+    last = run_both(X, cfg.W, cfg.k, cfg.topk, synth.fleet_dir(cfg.metrics), [cfg.block])
+    truth = synth.fleet_truth(cfg)
+    assert sorted(np.nonzero(last["flags"])[0].tolist()) == sorted(truth["persistent"])
+
+
+def test_medium_configuration_full():
+    cfg = synth.paper_configs()["medium"]
+    X = synth.fleet_tensor(cfg, device="cuda").cpu().numpy()
+    last = run_both(X, cfg.W, cfg.k, cfg.topk, synth.fleet_dir(cfg.metrics), [cfg.block])
+    truth = synth.fleet_truth(cfg)
+    assert set(truth["persistent"]) <= set(np.nonzero(last["mask"])[0].tolist())
+
+
+def test_large_configuration_sampled_blocks():
+    """16 384 ranks x 8 metrics, W = 200: two of the hundred 200-step blocks, checked in full
+    (tumbling windows with one evaluation per block make every block independent)."""
+    cfg = synth.paper_configs()["large"]
+    for t0 in (0, 15_800):
+        X = synth.fleet_block(cfg, t0, t0 + cfg.block, device="cuda").cpu().numpy()
+        run_both(X, cfg.W, cfg.k, cfg.topk, synth.fleet_dir(cfg.metrics), [cfg.block], capacity=cfg.block, in_place=True)
+
+
+def test_streaming_configuration_prefix():
+    """32 768 ranks, one step per ingest into a 512-step ring; every step's cross-rank
+    statistics are compared, evaluations at a few steps (an oracle evaluation sorts 262 144
+    series)."""
+    from paper_2605_17879_b200 import guard
+    cfg = synth.paper_configs()["streaming"]
+    T = 230
+    X = synth.fleet_block(cfg, 0, T, device="cuda")
+    Xh = X.cpu().numpy()
+    dirs = synth.fleet_dir(cfg.metrics)
+    g = guard.Guard(cfg.ranks, cfg.metrics, cfg.W, cfg.k, dir=dirs, capacity=cfg.ring_capacity, topk=cfg.topk)
+    o = go.Oracle(cfg.ranks, cfg.metrics, cfg.W, cfg.k, cfg.topk, dir=dirs)
+    smed = torch.empty((T, cfg.metrics), dtype=torch.float32, device="cuda")
+    smad = torch.empty((T, cfg.metrics), dtype=torch.float32, device="cuda")
+    for t in range(T):
+        g.ingest(X[t:t + 1], smed[t:t + 1], smad[t:t + 1])
+        os_ = o.ingest(Xh[t:t + 1])
+        if t in (0, 3, 150, 229):
+            gout = g.score()
+            g.sync_status()
+            compare_score(gout, o.score(), "t=%d" % t)
+            assert_bit_equal(to_np(smed[t]), os_["step_med"][0], "step_med")
+            assert_bit_equal(to_np(smad[t]), os_["step_mad"][0], "step_mad")
+    g.close()
+
+
+def test_nonfinite_input_sets_sticky_status():
+    from paper_2605_17879_b200 import guard
+    X, dirs = _rand_fleet(4, 16, 4, seed=10)
+    X[2, 5, 1] = np.nan
+    g = guard.Guard(16, 4, 4, 2, dir=dirs, topk=2)
+    g.ingest(torch.from_numpy(X).cuda())
+    with pytest.raises(guard.GuardError) as ei:
+        g.sync_status()
+    assert ei.value.code == -4
+    g.reset()
+    X[2, 5, 1] = 1.0
+    g.ingest(torch.from_numpy(X).cuda())
+    g.score()
+    assert g.sync_status() == 0
+    g.close()
+
+
+def test_runtime_argument_errors():
+    from paper_2605_17879_b200 import guard
+    g = guard.Guard(8, 2, 4, 2, dir=[1, 1], capacity=6, topk=2)
+    with pytest.raises(guard.GuardError) as ei:
+        g.score()
+    assert ei.value.code == -3                       # nothing ingested yet
+    with pytest.raises(guard.GuardError):
+        g.ingest(torch.ones((7, 8, 2), device="cuda"))   # more steps than the ring holds
+    g.ingest(torch.ones((4, 8, 2), device="cuda"))
+    with pytest.raises(guard.GuardError):
+        g.ring_reserve(3)                            # would wrap: slot 4 + 3 > 6
+    assert g.ring_reserve(2).shape == (2, 8, 2)
+    assert g.steps_seen == 4
+    g.close()
+
+
+@pytest.mark.parametrize("nodes,gpn,N,M,seed", [(1, 1, 1, 1, 0), (3, 2, 5, 3, 1), (16, 8, 20, 6, 2), (5, 4, 33, 7, 3),
+                                               (2, 8, 600, 6, 4)])
+def test_sweep_small_matches_oracle(nodes, gpn, N, M, seed):
+    from paper_2605_17879_b200 import guard
+    rng = np.random.default_rng(300 + seed)
+    G = nodes * gpn
+    S = np.round((1.0 + 0.01 * rng.normal(size=(G, 1, M))) * np.exp(0.003 * rng.normal(size=(G, N, M))) * 500) / 500
+    S[0] *= 0.8
+    S = S.astype(np.float32)
+    dirs = [(-1 if m % 3 else 1) for m in range(M)]
+    kw = dict(dir=dirs, thr=[3.5] * M, floor_rel=[1e-4] * M, floor_abs=[0.0 if m % 2 else 0.002 for m in range(M)],
+              pct_ppm=100_000)
+    out = guard.sweep_qualify(torch.from_numpy(S).cuda(), nodes, gpn, **kw)
+    ref = go.sweep(S, nodes, gpn, **kw)
+    assert int(out["status"].cpu()[0]) == 0
+    for key in ref:
+        assert_bit_equal(to_np(out[key]), ref[key], key)
+
+
+def test_sweep_configuration_full():
+    from paper_2605_17879_b200 import guard
+    cfg = synth.SweepConfig()
+    S = synth.sweep_tensor(cfg, device="cuda")
+    kw = dict(dir=synth.sweep_dir(cfg.metrics), thr=3.5, floor_rel=1e-4, floor_abs=synth.sweep_floor_abs(cfg.metrics),
+              pct_ppm=cfg.pct_ppm)
+    out = guard.sweep_qualify(S, cfg.nodes, cfg.gpus_per_node, **kw)
+    ref = go.sweep(S.cpu().numpy(), cfg.nodes, cfg.gpus_per_node, **kw)
+    assert int(out["status"].cpu()[0]) == 0
+    for key in ref:
+        assert_bit_equal(to_np(out[key]), ref[key], key)
+    bad, which, amount = synth.sweep_tables(cfg)
+    failed = set(np.nonzero(ref["gpu_pass"] == 0)[0].tolist())
+    strong = set(np.nonzero((bad & (amount > 0.10)).numpy())[0].tolist())
+    assert strong <= failed                       # clearly degraded GPUs are caught
+    assert len(failed) < 0.05 * cfg.gpus          # and the healthy bulk passes

@@ -321,6 +321,12 @@ def test_consecutive_evaluations():
     assert [int(o["flags"][9]) for o in outs] == [0, 0, 1]
     outs = _run(X, n_consec=1)
     assert [int(o["flags"][9]) for o in outs] == [0, 1, 1]
+    # an interruption restarts the run: slow, healthy, slow never gives two in a row
+    Y = _fleet(R=64, T=200, seed=11)
+    Y[:50, 9] = _slow(Y, 9, 1.3)[:50, 9]
+    Y[100:150, 9] = _slow(Y, 9, 1.3)[100:150, 9]
+    assert [int(o["flags"][9]) for o in _run(Y, n_consec=2)] == [0, 0, 0, 0]
+    assert [int(o["flags"][9]) for o in _run(Y, n_consec=1)] == [1, 0, 1, 0]
 
 
 def test_nonfinite_rejected():
