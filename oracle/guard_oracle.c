@@ -73,7 +73,7 @@ static float median_sorted_copy(const float *v, long n, long stride, float *tmp)
     for (long i = 0; i < n; ++i) tmp[i] = v[i * stride];
     qsort(tmp, (size_t)n, sizeof(float), cmp_f32);
     if (n & 1) return tmp[(n - 1) / 2];
-    return tmp[n / 2];
+    return 0.5f * (tmp[n / 2 - 1] + tmp[n / 2]);
 }
 
 float oracle_median(const float *v, long n)
