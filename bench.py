@@ -1,0 +1,309 @@
+#!/usr/bin/env python
+"""Benchmark of the straggler-scoring hot path on B200.
+
+One "step" is one pass of the whole path over the large-fleet workload: 16 384 ranks x
+20 000 steps x 8 float32 metrics (10.49 GB), ingested in 100 blocks of 200 steps with one
+evaluation (windowed medians, fleet baseline, scores/flags/tiers, top-64) after each block.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line.  `value` is cells scored per second with the telemetry already
+resident in HBM (written in place into the library's ring before the timed region);
+`e2e` is the same metric with the telemetry in pinned HOST memory, copied block by block
+into the ring inside the timed region, and the flags / top-k read back to the host after
+every evaluation.  With N > 1 every rank runs an independent replica (the path does not
+shard: a cross-rank median needs all ranks of a step on one GPU).
+
+`--impl reference` times the CPU oracle (oracle/, single thread, as it stands) on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "rank-step-metric cells scored/s"
+UNIT = "cells/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0   # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+
+
+def measured_hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        try:
+            for ln in open(self.path):
+                p = [x.strip() for x in ln.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1]))
+                    mx.append(float(p[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def workload():
+    from paper_2605_17879_b200 import synth
+    return synth.paper_configs()["large"]
+
+
+def oracle_sample_rate(cfg, block_host, sample_steps):
+    """Cells per second of the CPU oracle on the first `sample_steps` steps of one block
+    (ingest + one evaluation), single thread."""
+    from oracle import guard_oracle as go
+    from paper_2605_17879_b200 import synth
+    o = go.Oracle(cfg.ranks, cfg.metrics, cfg.W, cfg.k, cfg.topk, dir=synth.fleet_dir(cfg.metrics))
+    x = block_host[:sample_steps]
+    t0 = time.perf_counter()
+    o.ingest(x)
+    o.score()
+    dt = time.perf_counter() - t0
+    return x.size / dt, dt
+
+
+def run_reference(args):
+    """The reference arm: the oracle as it stands, on the host cores."""
+    from paper_2605_17879_b200 import dist as gd, synth
+    rank, _, world = gd.env_world()
+    if rank != 0:
+        return 0
+    cfg = workload()
+    sample_steps = 40
+    block = synth.fleet_block(cfg, 0, sample_steps, device="cpu").numpy()
+    from oracle import guard_oracle as go
+    go.build()
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample_rate(cfg, block, 8)
+    times = []
+    for _ in range(args.steps):
+        rate, dt = oracle_sample_rate(cfg, block, sample_steps)
+        times.append(dt)
+    total = sum(times)
+    cells = block.size * args.steps
+    value = cells / total
+    sample = ("per step: ingest + one evaluation of the first %d steps of the workload at full width "
+              "(%d ranks x %d metrics), window = those %d steps" % (sample_steps, cfg.ranks, cfg.metrics, sample_steps))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "large fleet: 16384 ranks x 20000 steps x 8 metrics, W=200 k=120 top-64 (bounded sample)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="guard", choices=["guard", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2605_17879_b200 import dist as gd, guard, synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    guard.lib()   # fails loudly if the CUDA library is not built
+    rank, local_rank, world = gd.init("nccl")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    warm = max(3, args.warmup)
+
+    cfg = workload()
+    R, M, T, B = cfg.ranks, cfg.metrics, cfg.steps, cfg.block
+    n_blocks = T // B
+    dirs = synth.fleet_dir(M)
+    # the ring holds the whole tensor, so telemetry is written in place once and stays resident
+    g = guard.Guard(R, M, cfg.W, cfg.k, dir=dirs, capacity=T, topk=cfg.topk, device=dev)
+    ring = g.ring_reserve(T)
+    for t0 in range(0, T, B):
+        synth.fleet_block(cfg, t0, t0 + B, device=dev, out=ring[t0:t0 + B])
+    torch.cuda.synchronize()
+    out = g.alloc_outputs()
+    cells_per_step = R * M * T
+
+    ev_pairs = []
+
+    def one_pass(time_ingest=False):
+        g.reset()
+        for j in range(n_blocks):
+            blk = ring[j * B:(j + 1) * B]
+            if time_ingest:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                g.ingest(blk)
+                e1.record()
+                ev_pairs.append((e0, e1))
+            else:
+                g.ingest(blk)
+            g.score(out)
+
+    for _ in range(warm):
+        one_pass()
+    g.sync_status()
+    sampler = ClockSampler(local_rank)
+    launches0 = g.kernel_launches
+    gd.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        one_pass(time_ingest=True)
+    stop.record()
+    torch.cuda.synchronize()
+    gd.barrier()
+    clocks = sampler.stop()
+    g.sync_status()
+    launches = g.kernel_launches - launches0
+    secs = start.elapsed_time(stop) / 1e3
+    value, tmax = gd.aggregate_throughput(cells_per_step * args.steps, secs, device=dev)
+    flagged = int(out["flags"].sum().item())
+
+    # roofline of the dominant kernel: the cross-rank selection behind guard_ingest.  One
+    # launch reads a block of 200 steps once (4 B per cell) and writes one exceedance byte
+    # per (step, rank) (1/8 B per cell).
+    ingest_ms = [a.elapsed_time(b) for a, b in ev_pairs]
+    launch_s = statistics.fmean(ingest_ms) / 1e3
+    algo_bytes = B * R * M * 4 + B * R * 1
+    peak, peak_kind = measured_hbm_peak()
+    achieved = algo_bytes / launch_s / 1e9
+    roofline = {"bound": "hbm", "kernel": "xrank (cross-rank median/MAD/exceedance, one launch per ingested block)",
+                "achieved": achieved, "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": launch_s * 1e3,
+                "share_of_step": sum(ingest_ms) / 1e3 / secs,
+                "path_algorithmic_GBps": (8.125 * cells_per_step * args.steps) / secs / 1e9,
+                "path_frac_of_peak": (8.125 * cells_per_step * args.steps) / secs / 1e9 / peak}
+
+    # end to end: telemetry in pinned host memory, copied into the ring block by block,
+    # flags and top-k copied back after every evaluation
+    host = torch.empty((T, R, M), dtype=torch.float32, pin_memory=True)
+    host.copy_(ring)
+    h_flags = torch.empty(R, dtype=torch.uint8, pin_memory=True)
+    h_idx = torch.empty(cfg.topk, dtype=torch.int32, pin_memory=True)
+    h_sc = torch.empty(cfg.topk, dtype=torch.float32, pin_memory=True)
+    torch.cuda.synchronize()
+
+    def one_pass_e2e():
+        g.reset()
+        for j in range(n_blocks):
+            slot = g.ring_reserve(B)
+            slot.copy_(host[j * B:(j + 1) * B], non_blocking=True)
+            g.ingest(slot)
+            g.score(out)
+            h_flags.copy_(out["flags"], non_blocking=True)
+            h_idx.copy_(out["topk_idx"], non_blocking=True)
+            h_sc.copy_(out["topk_score"], non_blocking=True)
+
+    one_pass_e2e()
+    gd.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        one_pass_e2e()
+    torch.cuda.synchronize()
+    e2e_secs = time.perf_counter() - t0
+    gd.barrier()
+    e2e_value, _ = gd.aggregate_throughput(cells_per_step * args.e2e_steps, e2e_secs, device=dev)
+    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * R * M * 4,
+           "d2h_bytes_per_step": n_blocks * (R + 8 * cfg.topk), "steps": args.e2e_steps,
+           "ms_per_step": 1e3 * e2e_secs / args.e2e_steps}
+    g.sync_status()
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample_steps = B          # one whole block with its full window: the unit the workload repeats
+        blk = host[:sample_steps].numpy()
+        rate, dt = oracle_sample_rate(cfg, blk, sample_steps)
+        cpu_baseline = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
+                        "sample": "ingest + one evaluation of the first %d steps at full width (%d ranks x %d metrics)"
+                                  % (sample_steps, R, M)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
+            "ms_per_step": 1e3 * tmax / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "large fleet: 16384 ranks x 20000 steps x 8 metrics (10.49 GB), W=200 k=120 top-64, "
+                                   "100 blocks of 200 steps, one evaluation per block",
+                       "ingest": "in place (telemetry written into the ring before timing)",
+                       "l2": "inputs (10.49 GB) larger than L2", "parallelism": "replicas only",
+                       "flagged_last_evaluation": flagged},
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    g.close()
+    gd.finish()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

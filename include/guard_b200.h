@@ -164,6 +164,10 @@ int guard_reset(guard_ctx *ctx, void *stream);
 /* Steps ingested since creation or the last reset. */
 int64_t guard_steps_seen(const guard_ctx *ctx);
 
+/* Kernels this context has enqueued so far (host-side count; copies and memsets are not
+ * counted). */
+int64_t guard_kernel_launches(const guard_ctx *ctx);
+
 /* Frees the host object (the workspace stays the caller's). NULL is allowed. */
 void guard_destroy(guard_ctx *ctx);
 

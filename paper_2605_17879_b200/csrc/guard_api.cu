@@ -94,6 +94,7 @@ struct guard_ctx {
     Layout L;
     char *ws;
     long long seen;
+    long long launches;  // kernels enqueued by this context so far
     char error[256];
 
     uint32_t *status() const { return (uint32_t *)(ws + L.status); }
@@ -145,7 +146,7 @@ int guard_create(guard_ctx **out, int ranks, int metrics, int W, int k, const gu
     guard_ctx *c = new (std::nothrow) guard_ctx();
     if (!c) { set_error(g_error, "out of host memory"); return GUARD_ERR_ARG; }
     c->R = ranks; c->M = metrics; c->W = W; c->k = k; c->C = capacity_steps; c->K = topk;
-    c->p = p; c->L = L; c->ws = (char *)d_workspace; c->seen = 0; c->error[0] = 0;
+    c->p = p; c->L = L; c->ws = (char *)d_workspace; c->seen = 0; c->launches = 0; c->error[0] = 0;
     // state: status word, ticket, fleet statistics, consecutive counters
     cudaError_t e = cudaMemsetAsync(c->ws, 0, L.wmed, (cudaStream_t)stream);
     if (e != cudaSuccess) {
@@ -201,6 +202,7 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
     a.status = c->status();
     cudaError_t e = launch_xrank_direct(a, c->p, B, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "xrank launch");
+    c->launches += 1;
     c->seen += B;
     return GUARD_OK;
 }
@@ -262,6 +264,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     s.tier = d_tier;
     e = launch_score_flag(s, c->p, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
+    c->launches += 3;
 
     if (c->K > 0 && (d_topk_idx || d_topk_score)) {
         TopkArgs t{};
@@ -277,6 +280,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         t.score = d_topk_score;
         e = launch_topk(t, c->p, st);
         if (e != cudaSuccess) return c->cuda_fail(e, "topk launch");
+        c->launches += 1;
     }
     return GUARD_OK;
 }
@@ -381,6 +385,8 @@ int guard_reset(guard_ctx *c, void *stream) {
 }
 
 int64_t guard_steps_seen(const guard_ctx *c) { return c ? c->seen : 0; }
+
+int64_t guard_kernel_launches(const guard_ctx *c) { return c ? c->launches : 0; }
 
 void guard_destroy(guard_ctx *c) { delete c; }
 

@@ -69,6 +69,8 @@ def lib():
         L.guard_reset.argtypes = [vp, vp]
         L.guard_steps_seen.restype = C.c_int64
         L.guard_steps_seen.argtypes = [vp]
+        L.guard_kernel_launches.restype = C.c_int64
+        L.guard_kernel_launches.argtypes = [vp]
         L.guard_destroy.restype = None
         L.guard_destroy.argtypes = [vp]
         L.guard_last_error.restype = C.c_char_p
@@ -145,11 +147,15 @@ class Guard:
             raise GuardError(rc, lib().guard_last_error(None).decode())
 
     def close(self):
-        if getattr(self, "_h", None):
-            lib().guard_destroy(self._h)
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.guard_destroy(self._h)
             self._h = C.c_void_p()
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
     def _check(self, rc: int):
         if rc != GUARD_OK:
@@ -158,6 +164,10 @@ class Guard:
     @property
     def steps_seen(self) -> int:
         return int(lib().guard_steps_seen(self._h))
+
+    @property
+    def kernel_launches(self) -> int:
+        return int(lib().guard_kernel_launches(self._h))
 
     def ring_reserve(self, steps: int) -> torch.Tensor:
         """View [steps, ranks, metrics] of the ring slots the next `steps` steps occupy."""
