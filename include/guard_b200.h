@@ -154,6 +154,39 @@ int guard_sweep_qualify(const float *d_S, int nodes, int gpus_per_node, int reps
                         uint32_t *d_fail_mask, uint8_t *d_gpu_pass, uint8_t *d_node_pass, uint32_t *d_status,
                         void *stream);
 
+/*
+ * Top-k of an evaluation without any allocation.  (The paper has no counterpart: this
+ * entry point exists only for callers that cannot allocate device memory.)
+ *
+ * Some users of this library run as a telemetry sidecar next to a training job on the same
+ * GPU.  There the job's own allocator has usually claimed the device memory up front, and
+ * cudaMalloc / cudaFree synchronise the whole device, which would stall the job's streams;
+ * such a caller cannot size and hand over a workspace just to re-rank a result.  This call
+ * therefore takes its scratch from a fixed array inside the library image
+ * (64 * GUARD_TOPK_STATIC_MAX_K candidate entries plus one ticket line = 131 328 bytes,
+ * held by every GPU that loads the library until the process exits) and calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Inputs are the device arrays an evaluation produced (guard_score outputs or the
+ * caller's own): d_wmed[ranks][metrics], d_fleet_med[metrics], d_fleet_mad[metrics];
+ * th->primary, th->dir, th->floor_rel and th->floor_abs are used, the rest is ignored.
+ * Outputs (either may be NULL): d_topk_idx[topk], d_topk_score[topk], identical to what
+ * guard_score returns for the same inputs.
+ * Limits: 1 <= topk <= min(ranks, GUARD_TOPK_STATIC_MAX_K), ranks <=
+ * GUARD_TOPK_STATIC_MAX_RANKS; anything larger is rejected with GUARD_ERR_ARG and a text
+ * in guard_last_error(NULL).
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call before starting any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's contents
+ * (the call clears the ticket it needs at zero on `stream`): two calls whose kernels can
+ * overlap on the GPU -- different streams, no ordering between them -- race on it.  Issue
+ * them on one stream or order them with events.
+ */
+#define GUARD_TOPK_STATIC_MAX_K 256
+#define GUARD_TOPK_STATIC_MAX_RANKS (1 << 24)
+int guard_topk_static(const float *d_wmed, const float *d_fleet_med, const float *d_fleet_mad, int ranks, int metrics,
+                      const guard_thresholds *th, int topk, int32_t *d_topk_idx, float *d_topk_score, void *stream);
+
 /* Synchronises `stream` and returns the sticky device status of the context
  * (GUARD_OK, GUARD_ERR_NONFINITE, GUARD_ERR_TIMEOUT, GUARD_ERR_INTERNAL, GUARD_ERR_CUDA). */
 int guard_sync_status(guard_ctx *ctx, void *stream);

@@ -79,6 +79,14 @@ const char *fill_params(MetricParams &p, const guard_thresholds *th, int M, int 
     return nullptr;
 }
 
+}  // namespace
+
+namespace guard {
+void set_global_error(const char *text) { set_error(g_error, "%s", text); }
+}  // namespace guard
+
+namespace {
+
 int status_to_code(uint32_t s) {
     if (s & kStatNonFinite) return GUARD_ERR_NONFINITE;
     if (s & kStatTimeout) return GUARD_ERR_TIMEOUT;

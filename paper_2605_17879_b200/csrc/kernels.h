@@ -72,6 +72,8 @@ struct TopkArgs {
     float *score;               // [K] or NULL
 };
 int topk_blocks(int R);
+// Records the text guard_last_error(NULL) returns (defined next to the C ABI).
+void set_global_error(const char *text);
 cudaError_t launch_topk(const TopkArgs &a, const MetricParams &p, cudaStream_t st);
 
 // Node sweep: per-GPU medians over repetitions, then the verdicts.

@@ -1,6 +1,10 @@
 // Top-k slowest ranks, block then grid: every CTA keeps the best entries of its slice of
 // ranks with a shared-memory bitonic network, writes its K best to scratch, and the CTA
 // that takes the last ticket merges the per-CTA lists.  No CTA ever waits for another.
+#include <cstdio>
+#include <mutex>
+
+#include "../../include/guard_b200.h"
 #include "kernels.h"
 
 namespace guard {
@@ -103,3 +107,109 @@ cudaError_t launch_topk(const TopkArgs &a, const MetricParams &p, cudaStream_t s
 }
 
 }  // namespace guard
+
+// ---- top-k without any allocation ---------------------------------------------------------
+//
+// Scratch for guard_topk_static: the per-CTA candidate lists followed by the ticket word.
+// It lives in the library image, so every GPU that loads the library holds these bytes
+// until the process exits, and every call on a device shares them.
+namespace {
+constexpr int kStaticMaxBlocks = 64;   // topk_blocks() never exceeds this
+constexpr size_t kStaticCandEntries = (size_t)kStaticMaxBlocks * GUARD_TOPK_STATIC_MAX_K;
+constexpr size_t kStaticTicketEntries = 32;  // one 256-byte line for the ticket
+static __device__ __align__(256) unsigned long long g_topk_static_scratch[kStaticCandEntries + kStaticTicketEntries];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void *g_static_ptr[kMaxDevices] = {};
+}  // namespace
+
+extern "C" int guard_topk_static(const float *d_wmed, const float *d_fleet_med, const float *d_fleet_mad, int ranks,
+                                 int metrics, const guard_thresholds *th, int topk, int32_t *d_topk_idx,
+                                 float *d_topk_score, void *stream) {
+    using namespace guard;
+    char msg[200];
+    if (!d_wmed || !d_fleet_med || !d_fleet_mad || !th || !th->dir || !th->floor_rel || !th->floor_abs) {
+        set_global_error("guard_topk_static: a required pointer is NULL");
+        return GUARD_ERR_ARG;
+    }
+    if (ranks < 1 || ranks > GUARD_TOPK_STATIC_MAX_RANKS || metrics < 1 || metrics > GUARD_MAX_METRICS) {
+        snprintf(msg, sizeof(msg), "guard_topk_static: need 1 <= ranks <= %d and 1 <= metrics <= %d",
+                 GUARD_TOPK_STATIC_MAX_RANKS, GUARD_MAX_METRICS);
+        set_global_error(msg);
+        return GUARD_ERR_ARG;
+    }
+    if (topk < 1 || topk > GUARD_TOPK_STATIC_MAX_K || topk > ranks) {
+        snprintf(msg, sizeof(msg), "guard_topk_static: topk must be in 1..min(ranks, %d); the built-in scratch holds no more",
+                 GUARD_TOPK_STATIC_MAX_K);
+        set_global_error(msg);
+        return GUARD_ERR_ARG;
+    }
+    if (th->primary < 0 || th->primary >= metrics) {
+        set_global_error("guard_topk_static: primary metric index out of range");
+        return GUARD_ERR_ARG;
+    }
+    MetricParams p{};
+    p.M = metrics;
+    p.primary = th->primary;
+    for (int m = 0; m < metrics; ++m) {
+        if (th->dir[m] != 1 && th->dir[m] != -1) {
+            set_global_error("guard_topk_static: dir[m] must be +1 or -1");
+            return GUARD_ERR_ARG;
+        }
+        p.dir[m] = th->dir[m];
+        p.floor_rel[m] = th->floor_rel[m];
+        p.floor_abs[m] = th->floor_abs[m];
+    }
+    // Once per device: ask the runtime where the array lives on the current device.  In
+    // host code the array's name is only a handle, never a pointer a kernel could use.
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        set_global_error("guard_topk_static: cudaGetDevice failed or device index out of range");
+        return GUARD_ERR_CUDA;
+    }
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_ptr[dev]) {
+            void *ptr = nullptr;
+            e = cudaGetSymbolAddress((void **)&ptr, g_topk_static_scratch);
+            if (e != cudaSuccess || !ptr) {
+                snprintf(msg, sizeof(msg), "guard_topk_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+                set_global_error(msg);
+                return GUARD_ERR_CUDA;
+            }
+            g_static_ptr[dev] = ptr;
+        }
+        scratch = g_static_ptr[dev];
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned long long *cand = (unsigned long long *)scratch;
+    unsigned int *ticket = (unsigned int *)(cand + kStaticCandEntries);
+    // The array keeps whatever the previous call left; only the ticket has to start at zero.
+    e = cudaMemsetAsync(ticket, 0, kStaticTicketEntries * sizeof(unsigned long long), st);
+    if (e != cudaSuccess) {
+        snprintf(msg, sizeof(msg), "guard_topk_static: cudaMemsetAsync: %s", cudaGetErrorString(e));
+        set_global_error(msg);
+        return GUARD_ERR_CUDA;
+    }
+    TopkArgs t{};
+    t.R = ranks;
+    t.M = metrics;
+    t.K = topk;
+    t.wmed = d_wmed;
+    t.fleet_med = d_fleet_med;
+    t.fleet_mad = d_fleet_mad;
+    t.cand = cand;
+    t.ticket = ticket;
+    t.idx = d_topk_idx;
+    t.score = d_topk_score;
+    e = launch_topk(t, p, st);
+    if (e != cudaSuccess) {
+        snprintf(msg, sizeof(msg), "guard_topk_static: launch: %s", cudaGetErrorString(e));
+        set_global_error(msg);
+        return GUARD_ERR_CUDA;
+    }
+    return GUARD_OK;
+}

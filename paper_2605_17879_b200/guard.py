@@ -63,6 +63,8 @@ def lib():
         L.guard_sweep_qualify.restype = C.c_int
         L.guard_sweep_qualify.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(_Thresholds), C.c_int32,
                                           vp, C.c_size_t] + [fp] * 8 + [vp]
+        L.guard_topk_static.restype = C.c_int
+        L.guard_topk_static.argtypes = [fp, fp, fp, C.c_int, C.c_int, C.POINTER(_Thresholds), C.c_int, fp, fp, vp]
         L.guard_sync_status.restype = C.c_int
         L.guard_sync_status.argtypes = [vp, vp]
         L.guard_reset.restype = C.c_int
@@ -267,6 +269,29 @@ def sweep_qualify(S: torch.Tensor, nodes: int, gpus_per_node: int, *, dir: Seque
     if rc != GUARD_OK:
         raise GuardError(rc, lib().guard_last_error(None).decode())
     return out
+
+
+TOPK_STATIC_MAX_K = 256
+
+
+def topk_static(wmed: torch.Tensor, fleet_med: torch.Tensor, fleet_mad: torch.Tensor, topk: int, *,
+                dir: Sequence[int], floor_rel=1e-4, floor_abs=0.0, primary: int = 0,
+                out_idx: Optional[torch.Tensor] = None, out_score: Optional[torch.Tensor] = None) -> None:
+    """Top-k of an evaluation through guard_topk_static: the library allocates nothing, the
+    caller passes every input and output tensor (outputs may be None to skip them).  Meant
+    for a sidecar that shares a GPU with a training job and must not call the device
+    allocator; limited to topk <= TOPK_STATIC_MAX_K.  Calls on one device share a built-in
+    scratch array, so keep them on one stream."""
+    if wmed.dim() != 2:
+        raise ValueError("wmed must be [ranks, metrics]")
+    R, M = wmed.shape
+    params = _Params(M, dir, 0.0, floor_rel, floor_abs, primary=primary)
+    with torch.cuda.device(wmed.device):
+        rc = lib().guard_topk_static(_ptr(wmed, torch.float32), _ptr(fleet_med, torch.float32, M),
+                                     _ptr(fleet_mad, torch.float32, M), R, M, C.byref(params.struct), topk,
+                                     _ptr(out_idx, torch.int32, topk), _ptr(out_score, torch.float32, topk), _stream())
+    if rc != GUARD_OK:
+        raise GuardError(rc, lib().guard_last_error(None).decode())
 
 
 def key_from_float(x: float) -> int:
