@@ -245,8 +245,10 @@ def main():
 
     # end to end: telemetry in pinned host memory, copied into the ring block by block,
     # flags and top-k copied back after every evaluation
-    host = torch.empty((T, R, M), dtype=torch.float32, pin_memory=True)
-    host.copy_(ring)
+    need_host = args.e2e_steps > 0 or (rank == 0 and world == 1 and not args.no_cpu_baseline)
+    host = torch.empty((T if args.e2e_steps > 0 else B, R, M), dtype=torch.float32, pin_memory=True) if need_host else None
+    if need_host:
+        host.copy_(ring[:host.shape[0]])
     h_flags = torch.empty(R, dtype=torch.uint8, pin_memory=True)
     h_idx = torch.empty(cfg.topk, dtype=torch.int32, pin_memory=True)
     h_sc = torch.empty(cfg.topk, dtype=torch.float32, pin_memory=True)
@@ -263,19 +265,21 @@ def main():
             h_idx.copy_(out["topk_idx"], non_blocking=True)
             h_sc.copy_(out["topk_score"], non_blocking=True)
 
-    one_pass_e2e()
-    gd.barrier()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for _ in range(args.e2e_steps):
+    e2e = None
+    if args.e2e_steps > 0:
         one_pass_e2e()
-    torch.cuda.synchronize()
-    e2e_secs = time.perf_counter() - t0
-    gd.barrier()
-    e2e_value, _ = gd.aggregate_throughput(cells_per_step * args.e2e_steps, e2e_secs, device=dev)
-    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * R * M * 4,
-           "d2h_bytes_per_step": n_blocks * (R + 8 * cfg.topk), "steps": args.e2e_steps,
-           "ms_per_step": 1e3 * e2e_secs / args.e2e_steps}
+        gd.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            one_pass_e2e()
+        torch.cuda.synchronize()
+        e2e_secs = time.perf_counter() - t0
+        gd.barrier()
+        e2e_value, _ = gd.aggregate_throughput(cells_per_step * args.e2e_steps, e2e_secs, device=dev)
+        e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * R * M * 4,
+               "d2h_bytes_per_step": n_blocks * (R + 8 * cfg.topk), "steps": args.e2e_steps,
+               "ms_per_step": 1e3 * e2e_secs / args.e2e_steps}
     g.sync_status()
 
     cpu_baseline = None
