@@ -16,7 +16,8 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, ticket, fleet, wmed, stepstat, topk_cand, mask, ring, total;
+    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, xr_big, mask, ring, total;
+    int xr_steps;   // steps per launch of the bracketed cross-rank path (0: path not used)
 };
 
 // State and scratch first, the two rings last (the telemetry ring is by far the largest).
@@ -27,9 +28,12 @@ Layout make_layout(int R, int M, int C, int K) {
     L.ticket = off;    off = align_up(off + 64);
     L.fleet = off;     off = align_up(off + 3 * kMaxMetrics * sizeof(float));
     L.consec = off;    off = align_up(off + (size_t)R);
+    L.xr_steps = xrank_bracket_supported(R, M) ? xrank_scratch_steps(R, M, C) : 0;
+    L.xr_small = off;  off = align_up(off + (L.xr_steps ? xrank_scratch_small_bytes(M, L.xr_steps) : 0));
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
+    L.xr_big = off;    off = align_up(off + (L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps) : 0));
     L.mask = off;      off = align_up(off + (size_t)C * R * (M <= 8 ? 1 : 4));
     L.ring = off;      off = align_up(off + (size_t)C * R * M * sizeof(float));
     L.total = off;
@@ -117,6 +121,25 @@ struct guard_ctx {
     void *mask() const { return ws + L.mask; }
     float *ring() const { return (float *)(ws + L.ring); }
     int mask_bytes() const { return M <= 8 ? 1 : 4; }
+    // Cross-rank statistics of S rows: the bracketed path where it applies, else the direct one.
+    cudaError_t xrank(XrankArgs a, int S, cudaStream_t st) {
+        if (L.xr_steps == 0) { launches += 1; return launch_xrank_direct(a, p, S, st); }
+        const XrankScratch sc = carve_xrank_scratch(ws + L.xr_small, ws + L.xr_big, R, M, L.xr_steps);
+        const int first = a.first_slot;
+        for (int s0 = 0; s0 < S; s0 += L.xr_steps) {
+            const int n = (S - s0 < L.xr_steps) ? (S - s0) : L.xr_steps;
+            XrankArgs g = a;
+            g.first_slot = (int)(((long long)first + s0) % a.capacity);
+            g.med = a.med + (size_t)s0 * M;
+            g.mad = a.mad + (size_t)s0 * M;
+            if (a.med_user) g.med_user = a.med_user + (size_t)s0 * M;
+            if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
+            cudaError_t e = launch_xrank_bracketed(g, p, sc, n, st);
+            if (e != cudaSuccess) return e;
+            launches += 4;
+        }
+        return cudaSuccess;
+    }
     int fail(int code, const char *fmt, ...) {
         va_list ap;
         va_start(ap, fmt);
@@ -208,9 +231,8 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
     a.mask_bytes = c->mask_bytes();
     a.check_finite = 1;
     a.status = c->status();
-    cudaError_t e = launch_xrank_direct(a, c->p, B, st);
+    cudaError_t e = c->xrank(a, B, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "xrank launch");
-    c->launches += 1;
     c->seen += B;
     return GUARD_OK;
 }
@@ -250,7 +272,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     x.med_user = d_fleet_med;
     x.mad_user = d_fleet_mad;
     x.status = c->status();
-    e = launch_xrank_direct(x, c->p, 1, st);
+    e = c->xrank(x, 1, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "fleet baseline launch");
 
     ScoreArgs s{};
@@ -272,7 +294,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     s.tier = d_tier;
     e = launch_score_flag(s, c->p, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
-    c->launches += 3;
+    c->launches += 2;
 
     if (c->K > 0 && (d_topk_idx || d_topk_score)) {
         TopkArgs t{};

@@ -22,7 +22,31 @@ struct XrankArgs {
     int mask_bytes;         // 1 (M <= 8) or 4
     int check_finite;       // flag NaN / Inf in the status word
     uint32_t *status;
+    uint32_t *only_flagged; // [S] or NULL: direct kernel processes step s only if nonzero, then clears it
 };
+
+// Scratch of the bracketed path for up to S_max steps per launch.
+struct XrankScratch {
+    float *lo, *hi;          // [S_max][M] value interval holding the two middle elements
+    float *center;           // sample median the MAD interval was measured about
+    float *dlo, *dhi;        // interval holding the MAD
+    float *rhs_lo, *rhs_hi;  // range of the exceedance threshold over that interval
+    uint32_t *cnt_lt;        // [S_max][M] elements below the interval
+    uint32_t *ncand;         // [S_max][M] elements collected
+    uint32_t *ticket;        // [S_max]
+    uint32_t *flag;          // [S_max] step must be redone by the direct path
+    uint32_t *namb;          // [S_max] deferred exceedance decisions
+    uint32_t *cand;          // [S_max][M][cap] float bits of the collected elements
+    uint32_t *amb;           // [S_max][amb_cap] (rank << 5 | metric)
+    int cap, amb_cap, S_max;
+};
+bool xrank_bracket_supported(int R, int M);
+int xrank_scratch_steps(int R, int M, int want);
+size_t xrank_scratch_small_bytes(int M, int S_max);   // must be zero before first use
+size_t xrank_scratch_big_bytes(int R, int M, int S_max);
+XrankScratch carve_xrank_scratch(void *small_base, void *big_base, int R, int M, int S_max);
+cudaError_t launch_xrank_bracketed(const XrankArgs &a, const MetricParams &p, const XrankScratch &sc, int S,
+                                   cudaStream_t st);
 
 cudaError_t launch_xrank_direct(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st);
 

@@ -159,6 +159,7 @@ __global__ void __launch_bounds__(kXrThreads) xrank_direct_kernel(const XrankArg
     extern __shared__ uint32_t hist[];
     __shared__ XrShared sh;
     const int s = blockIdx.x, tid = threadIdx.x;
+    if (a.only_flagged && a.only_flagged[s] == 0) return;
     const int R = a.R, M = a.M;
     const int slot = (int)(((long long)a.first_slot + s) % a.capacity);
     const float *row = a.base + (size_t)slot * a.row_stride;
@@ -205,6 +206,7 @@ __global__ void __launch_bounds__(kXrThreads) xrank_direct_kernel(const XrankArg
         cta_select(row, R, M, false, [](float x, int) { return f2key(x); }, hist, sh, a.status);
         if (tid < M) a.cut[(size_t)s * M + tid] = key2f(sh.prefix[tid]);
     }
+    if (a.only_flagged && tid == 0) a.only_flagged[s] = 0;
 }
 
 }  // namespace

@@ -51,6 +51,31 @@ def test_small_fleets_match_oracle(R, M, W, k, K, T, blocks, cap):
     run_both(X, W, k, K, dirs, blocks, capacity=cap, min_signals=min(2, M))
 
 
+@pytest.mark.parametrize("R,M,W,T,quant", [
+    (4096, 8, 6, 12, None),        # smallest fleet on the bracketed cross-rank path
+    (5000, 4, 5, 10, None),        # ragged last chunk
+    (4100, 16, 4, 8, None),
+    (4096, 32, 3, 6, None),
+    (6001, 8, 4, 8, None),         # odd rank count: a single middle element
+    (4096, 8, 4, 8, 50),           # quantised: intervals collapse onto tied values, some steps fall back
+    (8192, 4, 4, 8, 4),            # very coarse: candidate lists overflow, every step falls back
+])
+def test_bracketed_cross_rank_path(R, M, W, T, quant):
+    X, dirs = _rand_fleet(T, R, M, seed=R + M, quant=quant)
+    run_both(X, W, max(1, W // 2), 16, dirs, [W, 1, 2], capacity=2 * W, min_signals=2)
+
+
+def test_bracketed_path_constant_and_two_valued_fleets():
+    # every element equal: nothing can be bracketed, the direct path must take over and
+    # later healthy steps must run on the fast path again with clean counters
+    X, dirs = _rand_fleet(9, 4096, 8, seed=77)
+    X[2] = 1.0
+    X[3, ::2] = 1.0
+    X[3, 1::2] = 2.0
+    X[5] = X[5, :1]
+    run_both(X, 4, 2, 8, dirs, [3], capacity=6)
+
+
 def test_ties_zero_mad_and_signed_zero():
     # quantised telemetry: many equal values, MAD of zero, floors binding
     X, dirs = _rand_fleet(60, 48, 4, seed=5, quant=20)
