@@ -224,6 +224,7 @@ def main():
     clocks = sampler.stop()
     g.sync_status()
     launches = g.kernel_launches - launches0
+    fallback_rows = g.fallback_steps()
     secs = start.elapsed_time(stop) / 1e3
     value, tmax = gd.aggregate_throughput(cells_per_step * args.steps, secs, device=dev)
     flagged = int(out["flags"].sum().item())
@@ -300,7 +301,7 @@ def main():
                                    "100 blocks of 200 steps, one evaluation per block",
                        "ingest": "in place (telemetry written into the ring before timing)",
                        "l2": "inputs (10.49 GB) larger than L2", "parallelism": "replicas only",
-                       "flagged_last_evaluation": flagged},
+                       "flagged_last_evaluation": flagged, "direct_path_fallback_rows_last_pass": fallback_rows},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)

@@ -201,6 +201,19 @@ int64_t guard_steps_seen(const guard_ctx *ctx);
  * counted). */
 int64_t guard_kernel_launches(const guard_ctx *ctx);
 
+/* Synchronises `stream` and returns how many cross-rank rows (ingested steps or fleet
+ * baselines) had to be recomputed by the slower direct selection since creation or the last
+ * reset, because the sampled interval of the fast path did not hold the middle elements or a
+ * candidate list overflowed.  Results are exact either way; this is a performance counter.
+ * Negative on error. */
+int64_t guard_fallback_steps(guard_ctx *ctx, void *stream);
+
+/* Diagnostic companion of guard_fallback_steps: synchronises `stream` and fills out[6] (HOST)
+ * with event counts since creation / reset: 0 a CTA's staged candidate list overflowed, 1 a
+ * step's candidate list overflowed, 2 the deferred-exceedance list overflowed, 3 the sampled
+ * interval missed the median, 4 candidate selection inconsistent, 5 the interval missed the MAD. */
+int guard_fallback_reasons(guard_ctx *ctx, uint32_t out[6], void *stream);
+
 /* Frees the host object (the workspace stays the caller's). NULL is allowed. */
 void guard_destroy(guard_ctx *ctx);
 

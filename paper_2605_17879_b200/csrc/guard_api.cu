@@ -124,11 +124,13 @@ struct guard_ctx {
     // Cross-rank statistics of S rows: the bracketed path where it applies, else the direct one.
     cudaError_t xrank(XrankArgs a, int S, cudaStream_t st) {
         if (L.xr_steps == 0) { launches += 1; return launch_xrank_direct(a, p, S, st); }
-        const XrankScratch sc = carve_xrank_scratch(ws + L.xr_small, ws + L.xr_big, R, M, L.xr_steps);
+        XrankScratch sc = carve_xrank_scratch(ws + L.xr_small, ws + L.xr_big, R, M, L.xr_steps);
+        sc.reasons = status() + 2;
         const int first = a.first_slot;
         for (int s0 = 0; s0 < S; s0 += L.xr_steps) {
             const int n = (S - s0 < L.xr_steps) ? (S - s0) : L.xr_steps;
             XrankArgs g = a;
+            g.fallbacks = status() + 1;
             g.first_slot = (int)(((long long)first + s0) % a.capacity);
             g.med = a.med + (size_t)s0 * M;
             g.mad = a.mad + (size_t)s0 * M;
@@ -417,6 +419,23 @@ int guard_reset(guard_ctx *c, void *stream) {
 int64_t guard_steps_seen(const guard_ctx *c) { return c ? c->seen : 0; }
 
 int64_t guard_kernel_launches(const guard_ctx *c) { return c ? c->launches : 0; }
+
+int guard_fallback_reasons(guard_ctx *c, uint32_t out[6], void *stream) {
+    if (!c || !out) return GUARD_ERR_ARG;
+    cudaError_t e = cudaMemcpyAsync(out, c->status() + 2, 6 * sizeof(uint32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_fallback_reasons");
+    return GUARD_OK;
+}
+
+int64_t guard_fallback_steps(guard_ctx *c, void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    uint32_t n = 0;
+    cudaError_t e = cudaMemcpyAsync(&n, c->status() + 1, sizeof(n), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_fallback_steps");
+    return (int64_t)n;
+}
 
 void guard_destroy(guard_ctx *c) { delete c; }
 

@@ -23,6 +23,7 @@ struct XrankArgs {
     int check_finite;       // flag NaN / Inf in the status word
     uint32_t *status;
     uint32_t *only_flagged; // [S] or NULL: direct kernel processes step s only if nonzero, then clears it
+    uint32_t *fallbacks;    // or NULL: counts the steps the direct kernel redid for the bracketed path
 };
 
 // Scratch of the bracketed path for up to S_max steps per launch.
@@ -38,8 +39,10 @@ struct XrankScratch {
     uint32_t *namb;          // [S_max] deferred exceedance decisions
     uint32_t *cand;          // [S_max][M][cap] float bits of the collected elements
     uint32_t *amb;           // [S_max][amb_cap] (rank << 5 | metric)
+    uint32_t *reasons;       // [8] why steps left the fast path (diagnostic counters) or NULL
     int cap, amb_cap, S_max;
 };
+enum { kWhyCtaList = 0, kWhyStepList = 1, kWhyAmbList = 2, kWhyMedianMiss = 3, kWhySelect = 4, kWhyMadMiss = 5 };
 bool xrank_bracket_supported(int R, int M);
 int xrank_scratch_steps(int R, int M, int want);
 size_t xrank_scratch_small_bytes(int M, int S_max);   // must be zero before first use

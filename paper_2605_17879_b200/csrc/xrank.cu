@@ -206,7 +206,10 @@ __global__ void __launch_bounds__(kXrThreads) xrank_direct_kernel(const XrankArg
         cta_select(row, R, M, false, [](float x, int) { return f2key(x); }, hist, sh, a.status);
         if (tid < M) a.cut[(size_t)s * M + tid] = key2f(sh.prefix[tid]);
     }
-    if (a.only_flagged && tid == 0) a.only_flagged[s] = 0;
+    if (a.only_flagged && tid == 0) {
+        a.only_flagged[s] = 0;
+        if (a.fallbacks) atomicAdd(a.fallbacks, 1u);
+    }
 }
 
 }  // namespace

@@ -362,19 +362,19 @@ __global__ void __launch_bounds__(kBrThreads) xrank_stream_kernel(const XrankArg
     // shared lists -> the step's global lists
     if (tid < M) {
         const uint32_t n = s_ncand[tid];
-        if (n > kCtaCand) s_overflow = 1;
+        if (n > kCtaCand) { s_overflow = 1; if (sc.reasons) atomicAdd(sc.reasons + kWhyCtaList, 1u); }
         if (s_cnt[tid]) atomicAdd(sc.cnt_lt + so + tid, s_cnt[tid]);
         uint32_t base = 0;
         if (n) base = atomicAdd(sc.ncand + so + tid, n);
         s_base[tid] = base;
-        if (base + n > (uint32_t)sc.cap) s_overflow = 1;
+        if (base + n > (uint32_t)sc.cap) { s_overflow = 1; if (sc.reasons) atomicAdd(sc.reasons + kWhyStepList, 1u); }
     }
     if (MODE == 1 && tid == 32) {
         const uint32_t n = min(s_namb, (uint32_t)kCtaAmb);
         uint32_t base = 0;
         if (n) base = atomicAdd(sc.namb + t, n);
         s_ambbase = base;
-        if (base + n > (uint32_t)sc.amb_cap) s_overflow = 1;
+        if (base + n > (uint32_t)sc.amb_cap || s_namb > (uint32_t)kCtaAmb) { s_overflow = 1; if (sc.reasons) atomicAdd(sc.reasons + kWhyAmbList, 1u); }
     }
     __syncthreads();
     if (!s_overflow) {
@@ -404,11 +404,19 @@ __global__ void __launch_bounds__(kBrThreads) xrank_stream_kernel(const XrankArg
     const uint32_t k1 = (uint32_t)((R - 1) / 2), k2 = (uint32_t)(R / 2);
     for (int m = 0; m < M && !fail; ++m) {
         const uint32_t clt = __ldcg(sc.cnt_lt + so + m), n = __ldcg(sc.ncand + so + m);
-        if (!(clt <= k1 && k2 < clt + n && n <= (uint32_t)sc.cap)) { fail = true; break; }
+        if (!(clt <= k1 && k2 < clt + n && n <= (uint32_t)sc.cap)) {
+            if (tid == 0 && sc.reasons) atomicAdd(sc.reasons + (MODE == 0 ? kWhyMedianMiss : kWhyMadMiss), 1u);
+            fail = true;
+            break;
+        }
         uint32_t v1, v2;
         bool ok;
         cta_select_list(sc.cand + (so + m) * (size_t)sc.cap, (int)n, k1 - clt, even, ls, v1, v2, ok);
-        if (!ok) { fail = true; break; }
+        if (!ok) {
+            if (tid == 0 && sc.reasons) atomicAdd(sc.reasons + kWhySelect, 1u);
+            fail = true;
+            break;
+        }
         if (tid == 0) s_val[m] = median_from_keys(v1, v2, even);
     }
     __syncthreads();
@@ -419,11 +427,12 @@ __global__ void __launch_bounds__(kBrThreads) xrank_stream_kernel(const XrankArg
                 const float med_m = s_val[m];
                 a.med[so + m] = med_m;
                 if (a.med_user) a.med_user[so + m] = med_m;
-                // move the sampled MAD interval from the sample's centre to the exact median
-                const float e = fabsf(med_m - sc.center[so + m]);
-                float dl = sc.dlo[so + m] - e;
+                // The MAD interval was measured about the sample's median.  Moving the centre
+                // to the exact median changes the count inside +-d only to second order (what
+                // one side gains the other loses), so the interval is kept, opened by one ulp.
+                float dl = sc.dlo[so + m];
                 dl = dl > 0.0f ? fdown(dl) : 0.0f;
-                float dh = sc.dhi[so + m] + e;
+                float dh = sc.dhi[so + m];
                 if (dh < CUDART_INF_F) dh = fup(dh);
                 sc.dlo[so + m] = dl;
                 sc.dhi[so + m] = dh;
@@ -551,7 +560,9 @@ cudaError_t launch_xrank_bracketed(const XrankArgs &a, const MetricParams &p, co
                                    cudaStream_t st) {
     if (S <= 0) return cudaSuccess;
     const int s = sample_size(a.R, a.M);
-    const int delta = (int)ceil(4.5 * 0.5 * sqrt((double)s));
+    // half-width of the sampled interval in sample ranks: 5.5 standard deviations of a sample
+    // quantile's rank (0.5 sqrt(s)), so that a miss (and the slow direct redo) is a ~1e-7 event
+    const int delta = (int)ceil(5.5 * 0.5 * sqrt((double)s));
     xrank_sample_kernel<<<S, kSampleThreads, (size_t)s * a.M * sizeof(uint32_t), st>>>(a, sc, s, delta);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

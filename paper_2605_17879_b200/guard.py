@@ -73,6 +73,10 @@ def lib():
         L.guard_steps_seen.argtypes = [vp]
         L.guard_kernel_launches.restype = C.c_int64
         L.guard_kernel_launches.argtypes = [vp]
+        L.guard_fallback_steps.restype = C.c_int64
+        L.guard_fallback_steps.argtypes = [vp, vp]
+        L.guard_fallback_reasons.restype = C.c_int
+        L.guard_fallback_reasons.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.guard_destroy.restype = None
         L.guard_destroy.argtypes = [vp]
         L.guard_last_error.restype = C.c_char_p
@@ -170,6 +174,22 @@ class Guard:
     @property
     def kernel_launches(self) -> int:
         return int(lib().guard_kernel_launches(self._h))
+
+    def fallback_steps(self) -> int:
+        """Rows the fast cross-rank path handed to the direct selection (synchronises)."""
+        with torch.cuda.device(self.device):
+            n = int(lib().guard_fallback_steps(self._h, _stream()))
+        if n < 0:
+            self._check(n)
+        return n
+
+    def fallback_reasons(self):
+        """Counts of the events that send rows to the direct selection (synchronises)."""
+        out = (C.c_uint32 * 6)()
+        with torch.cuda.device(self.device):
+            self._check(lib().guard_fallback_reasons(self._h, out, _stream()))
+        names = ("cta_list", "step_list", "deferred_list", "median_miss", "select", "mad_miss")
+        return dict(zip(names, [int(v) for v in out]))
 
     def ring_reserve(self, steps: int) -> torch.Tensor:
         """View [steps, ranks, metrics] of the ring slots the next `steps` steps occupy."""
