@@ -138,7 +138,7 @@ struct guard_ctx {
             if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
             cudaError_t e = launch_xrank_bracketed(g, p, sc, n, st);
             if (e != cudaSuccess) return e;
-            launches += 4;
+            launches += 6;
         }
         return cudaSuccess;
     }

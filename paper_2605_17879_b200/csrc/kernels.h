@@ -29,12 +29,10 @@ struct XrankArgs {
 // Scratch of the bracketed path for up to S_max steps per launch.
 struct XrankScratch {
     float *lo, *hi;          // [S_max][M] value interval holding the two middle elements
-    float *center;           // sample median the MAD interval was measured about
     float *dlo, *dhi;        // interval holding the MAD
     float *rhs_lo, *rhs_hi;  // range of the exceedance threshold over that interval
     uint32_t *cnt_lt;        // [S_max][M] elements below the interval
     uint32_t *ncand;         // [S_max][M] elements collected
-    uint32_t *ticket;        // [S_max]
     uint32_t *flag;          // [S_max] step must be redone by the direct path
     uint32_t *namb;          // [S_max] deferred exceedance decisions
     uint32_t *cand;          // [S_max][M][cap] float bits of the collected elements

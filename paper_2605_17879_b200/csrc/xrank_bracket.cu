@@ -5,26 +5,26 @@
 // nowhere near the middle.  This path brackets the wanted order statistic first and then
 // touches every element once per statistic:
 //
-//   1. sample kernel   one CTA per step sorts a strided sample of each column and derives
-//                      [lo, hi], a value interval that contains the column's two middle
-//                      elements with high probability, plus a first guess of the MAD interval;
-//   2. median kernel   many CTAs per step stream the row with 128-bit loads: every element
-//                      is counted if below lo and collected if inside [lo, hi]; the CTA that
-//                      draws the step's last ticket checks the counts (they prove whether
-//                      the interval really holds the middle elements) and selects the exact
-//                      median among the few collected candidates by radix select on
-//                      order-preserving keys;
-//   3. MAD kernel      the same for |x - med| against [dlo, dhi]; in the same sweep every
+//   1. sample kernel   one CTA per step; each warp sorts a strided sample of one column in
+//                      registers (bitonic network over shuffles) and derives [lo, hi], a value
+//                      interval that holds the column's two middle elements with high
+//                      probability, and [dlo, dhi], the same for the MAD;
+//   2. median sweep    many CTAs per step stream the row with 128-bit loads: every element is
+//                      counted if below lo and collected if inside [lo, hi];
+//   3. median select   one CTA per column checks the counts (they prove whether the interval
+//                      really holds the middle elements) and selects the exact median among the
+//                      collected elements: histogram of order-preserving keys over the
+//                      interval, refined until a bin is a single key;
+//   4. MAD sweep       the same for |x - med| against [dlo, dhi]; in the same sweep every
 //                      element's exceedance bit is decided when it is clear of the possible
 //                      range of the threshold and deferred to a short list when it is not;
-//                      the last CTA selects the exact MAD, fixes the threshold and settles the
-//                      deferred elements;
-//   4. any step whose interval failed (counts disagree, a list overflowed) is flagged and
+//   5. MAD select      exact MAD, then the threshold is fixed and the deferred elements settled;
+//   6. any step whose interval failed (counts disagree, a list overflowed) is flagged and
 //                      recomputed by the direct radix-select kernel, so results are always
-//                      exact; the brackets only decide how fast they arrive.
+//                      exact; the intervals only decide how fast they arrive.
 //
-// No CTA ever waits for another: cross-CTA combination uses atomic counters and a
-// last-ticket finaliser.
+// No CTA ever waits for another: cross-CTA combination uses atomic counters, and the kernel
+// boundary orders the phases.
 #include <math_constants.h>
 
 #include "kernels.h"
@@ -34,187 +34,108 @@ namespace guard {
 namespace {
 
 constexpr int kBrThreads = 256;
-constexpr int kRPT = 8;           // ranks per thread in the streaming kernels
+constexpr int kRPT = 8;              // ranks per thread in the streaming kernels
 constexpr int kCtaCandTotal = 5120;  // candidate slots staged in shared memory per CTA, shared out over the metrics
-constexpr int kCtaAmb = 512;      // deferred exceedance decisions staged per CTA
-constexpr int kSampleThreads = 1024;
+constexpr int kCtaAmb = 512;         // deferred exceedance decisions staged per CTA
+constexpr int kSelThreads = 256;
+constexpr int kSelBins = 2048;
 
 __device__ __forceinline__ float fdown(float x) { return __uint_as_float(f2key(x) == 0 ? __float_as_uint(x) : bits_of_key(f2key(x) - 1)); }
 __device__ __forceinline__ float fup(float x) { return __uint_as_float(bits_of_key(f2key(x) + 1)); }
 
 // ---------------------------------------------------------------------------------------
-// 1. sample kernel
+// 1. sample kernel: one warp per metric sorts 32 * EPL sampled keys in registers
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kSampleThreads) xrank_sample_kernel(const XrankArgs a, const XrankScratch sc, const int s,
-                                                                      const int delta) {
-    extern __shared__ uint32_t keys[];  // [M][s]
-    const int t = blockIdx.x, tid = threadIdx.x;
+template <int EPL>
+__device__ __forceinline__ void warp_bitonic_sort(uint32_t (&v)[EPL], const int lane) {
+    constexpr int N = 32 * EPL;
+#pragma unroll
+    for (int size = 2; size <= N; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            if (stride >= EPL) {   // partner element lives in lane ^ (stride / EPL), same register
+                const int lm = stride / EPL;
+                const bool upper = (lane & lm) != 0;
+#pragma unroll
+                for (int j = 0; j < EPL; ++j) {
+                    const bool asc = (((lane * EPL + j) & size) == 0);
+                    const uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, v[j], lm);
+                    v[j] = (asc != upper) ? min(v[j], o) : max(v[j], o);
+                }
+            } else {               // both elements in this lane
+#pragma unroll
+                for (int j = 0; j < EPL; ++j) {
+                    if ((j & stride) == 0) {
+                        const bool asc = (((lane * EPL + j) & size) == 0);
+                        const uint32_t x = v[j], y = v[j | stride];
+                        const uint32_t mn = min(x, y), mx = max(x, y);
+                        v[j] = asc ? mn : mx;
+                        v[j | stride] = asc ? mx : mn;
+                    }
+                }
+            }
+        }
+    }
+}
+
+template <int EPL>
+__global__ void __launch_bounds__(1024) xrank_sample_kernel(const XrankArgs a, const XrankScratch sc, const int delta) {
+    constexpr int s = 32 * EPL;
+    extern __shared__ uint32_t keys[];  // [M][s], sorted per metric
+    const int t = blockIdx.x, lane = lane_id(), m = warp_id();
     const int R = a.R, M = a.M;
     const int slot = (int)(((long long)a.first_slot + t) % a.capacity);
     const float *row = a.base + (size_t)slot * a.row_stride;
     const int stride = R / s;
-    for (int e = tid; e < s * M; e += blockDim.x) {
-        const int i = e / M, m = e - i * M;
-        const int r = i * stride + (stride >> 1);
-        keys[m * s + i] = f2key(row[(size_t)r * M + m]);
-    }
-    // bitonic sort of every metric's sample (ascending)
-    const int half = (s * M) >> 1;
-    for (int size = 2; size <= s; size <<= 1) {
-        for (int st = size >> 1; st > 0; st >>= 1) {
-            __syncthreads();
-            for (int e = tid; e < half; e += blockDim.x) {
-                const int m = e / (s >> 1), q = e - m * (s >> 1);
-                const int i = 2 * q - (q & (st - 1));
-                const int j = i + st;
-                uint32_t *k = keys + m * s;
-                const bool asc = ((i & size) == 0);
-                const uint32_t x = k[i], y = k[j];
-                if ((x > y) == asc) { k[i] = y; k[j] = x; }
-            }
-        }
-    }
-    __syncthreads();
-    // one warp per metric derives the intervals
-    const int warp = warp_id(), lane = lane_id(), nwarps = blockDim.x >> 5;
-    for (int m = warp; m < M; m += nwarps) {
-        const uint32_t *k = keys + m * s;
-        const int mid = s >> 1;
-        const int ilo = max(0, mid - delta), ihi = min(s - 1, mid + delta);
-        const float lo = key2f(k[ilo]), hi = key2f(k[ihi]);
-        const float c = key2f(k[mid]);
-        // interval of the MAD from the sample's deviations about its own median:
-        // f(d) = #{x : |x - c| <= d}; dlo = largest sampled deviation with f <= jlo,
-        // dhi = smallest with f >= jhi + 1.
-        const int jlo = max(0, mid - delta), jhi = min(s - 1, mid + delta);
-        float dlo = 0.0f, dhi = CUDART_INF_F;
-        for (int i = lane; i < s; i += 32) {
-            const float d = fabsf(key2f(k[i]) - c);
-            const uint32_t ka = f2key(c - d), kb = f2key(c + d);
-            int lb = 0, n = s;      // lb = #{key < ka}
-            while (n > 0) { const int h = n >> 1; if (k[lb + h] < ka) { lb += h + 1; n -= h + 1; } else n = h; }
-            int ub = 0; n = s;      // ub = #{key <= kb}
-            while (n > 0) { const int h = n >> 1; if (k[ub + h] <= kb) { ub += h + 1; n -= h + 1; } else n = h; }
-            const int f = ub - lb;
-            if (f <= jlo) dlo = fmaxf(dlo, d);
-            if (f >= jhi + 1) dhi = fminf(dhi, d);
-        }
+    uint32_t v[EPL];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            dlo = fmaxf(dlo, __shfl_xor_sync(0xFFFFFFFFu, dlo, o));
-            dhi = fminf(dhi, __shfl_xor_sync(0xFFFFFFFFu, dhi, o));
-        }
-        if (lane == 0) {
-            const size_t o = (size_t)t * M + m;
-            sc.lo[o] = lo;
-            sc.hi[o] = hi;
-            sc.center[o] = c;
-            sc.dlo[o] = dlo;
-            sc.dhi[o] = dhi;
-        }
+    for (int j = 0; j < EPL; ++j) {
+        const int r = (lane * EPL + j) * stride + (stride >> 1);
+        v[j] = f2key(__ldg(row + (size_t)r * M + m));
+    }
+    warp_bitonic_sort<EPL>(v, lane);
+    uint32_t *k = keys + m * s;
+#pragma unroll
+    for (int j = 0; j < EPL; ++j) k[lane * EPL + j] = v[j];
+    __syncwarp();
+    const int mid = s >> 1;
+    const int ilo = max(0, mid - delta), ihi = min(s - 1, mid + delta);
+    const float lo = key2f(k[ilo]), hi = key2f(k[ihi]);
+    const float c = key2f(k[mid]);
+    // interval of the MAD from the sample's deviations about its own median:
+    // f(d) = #{x : |x - c| <= d}; dlo = largest sampled deviation with f <= ilo,
+    // dhi = smallest with f >= ihi + 1.
+    float dlo = 0.0f, dhi = CUDART_INF_F;
+    for (int i = lane; i < s; i += 32) {
+        const float d = fabsf(key2f(k[i]) - c);
+        const uint32_t ka = f2key(c - d), kb = f2key(c + d);
+        int lb = 0, n = s;      // lb = #{key < ka}
+        while (n > 0) { const int h = n >> 1; if (k[lb + h] < ka) { lb += h + 1; n -= h + 1; } else n = h; }
+        int ub = 0; n = s;      // ub = #{key <= kb}
+        while (n > 0) { const int h = n >> 1; if (k[ub + h] <= kb) { ub += h + 1; n -= h + 1; } else n = h; }
+        const int f = ub - lb;
+        if (f <= ilo) dlo = fmaxf(dlo, d);
+        if (f >= ihi + 1) dhi = fminf(dhi, d);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        dlo = fmaxf(dlo, __shfl_xor_sync(0xFFFFFFFFu, dlo, o));
+        dhi = fminf(dhi, __shfl_xor_sync(0xFFFFFFFFu, dhi, o));
+    }
+    if (lane == 0) {
+        const size_t o = (size_t)t * M + m;
+        sc.lo[o] = lo;
+        sc.hi[o] = hi;
+        // The MAD interval was measured about the sample's median.  Moving the centre to the
+        // exact median changes the count inside +-d only to second order (what one side gains
+        // the other loses), so the interval is kept, opened by one ulp.
+        sc.dlo[o] = dlo > 0.0f ? fdown(dlo) : 0.0f;
+        sc.dhi[o] = dhi < CUDART_INF_F ? fup(dhi) : dhi;
     }
 }
 
 // ---------------------------------------------------------------------------------------
-// selection among the collected candidates (all threads of the CTA; list in global memory)
-// ---------------------------------------------------------------------------------------
-struct ListSel {
-    uint32_t hist[256];
-    uint32_t prefix, krem, ceq, v2, kand, kor;
-    int need;
-};
-
-// Finds the keys of 0-based ranks k and (if want_next) k + 1 in list[0..n) (raw float bits).
-__device__ void cta_select_list(const uint32_t *list, int n, uint32_t k, bool want_next, ListSel &ls, uint32_t &v1,
-                                uint32_t &v2, bool &ok) {
-    const int tid = threadIdx.x, lane = lane_id();
-    if (tid == 0) { ls.kand = 0xFFFFFFFFu; ls.kor = 0u; ls.prefix = 0; ls.krem = k; ls.ceq = (uint32_t)n; ls.v2 = 0xFFFFFFFFu; ls.need = 0; }
-    for (int i = tid; i < 256; i += blockDim.x) ls.hist[i] = 0;
-    __syncthreads();
-    uint32_t kand = 0xFFFFFFFFu, kor = 0u;
-    for (int i = tid; i < n; i += blockDim.x) {
-        const uint32_t key = key_of_bits(__ldcg(list + i));
-        kand &= key;
-        kor |= key;
-    }
-    kand = __reduce_and_sync(0xFFFFFFFFu, kand);
-    kor = __reduce_or_sync(0xFFFFFFFFu, kor);
-    if (lane == 0) { atomicAnd(&ls.kand, kand); atomicOr(&ls.kor, kor); }
-    __syncthreads();
-    const uint32_t diff = ls.kand ^ ls.kor;   // bits that vary among the candidates
-    ok = true;
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        if (((diff >> shift) & 255u) == 0) {   // this digit is the same for every candidate
-            if (tid == 0) ls.prefix |= ls.kor & (255u << shift);
-            __syncthreads();
-            continue;
-        }
-        const uint32_t prefix = ls.prefix;
-        const int nround = (n + blockDim.x - 1) / blockDim.x;
-        for (int it = 0; it < nround; ++it) {
-            const int i = it * blockDim.x + tid;
-            bool valid = i < n;
-            uint32_t key = 0;
-            if (valid) {
-                key = key_of_bits(__ldcg(list + i));
-                if (pass > 0) valid = ((key ^ prefix) >> (shift + 8)) == 0;
-            }
-            const uint32_t digit = (key >> shift) & 255u;
-            const unsigned peers = __match_any_sync(0xFFFFFFFFu, valid ? digit : (256u + lane));
-            if (valid && lane == __ffs(peers) - 1) atomicAdd(&ls.hist[digit], __popc(peers));
-        }
-        __syncthreads();
-        if (tid < 32) {
-            // find the bin holding rank krem
-            uint32_t loc[8], sum = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { loc[i] = ls.hist[lane * 8 + i]; sum += loc[i]; }
-            uint32_t incl = sum;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) { const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, incl, d); if (lane >= d) incl += u; }
-            const uint32_t excl = incl - sum, kk = ls.krem;
-            const bool mine = (kk >= excl) && (kk < incl);
-            const unsigned ball = __ballot_sync(0xFFFFFFFFu, mine);
-            __syncwarp();
-            for (int i = lane; i < 256; i += 32) ls.hist[i] = 0;
-            if (mine) {
-                uint32_t run = excl;
-                int b = 7; uint32_t bef = excl, c = 0;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) { if (kk >= run && kk < run + loc[i]) { b = i; bef = run; c = loc[i]; } run += loc[i]; }
-                ls.prefix |= (uint32_t)(lane * 8 + b) << shift;
-                ls.krem = kk - bef;
-                ls.ceq = c;
-            }
-            if (ball == 0 && lane == 0) ls.need = -1;   // rank not inside the list: caller flags the step
-        }
-        __syncthreads();
-    }
-    if (ls.need < 0) ok = false;
-    v1 = ls.prefix;
-    v2 = v1;
-    if (want_next && ok) {
-        // ceq counts the copies of the selected key (n if no digit varied at all)
-        const bool need = (ls.krem + 1 >= ls.ceq);
-        if (need) {
-            uint32_t cand = 0xFFFFFFFFu;
-            for (int i = tid; i < n; i += blockDim.x) {
-                const uint32_t key = key_of_bits(__ldcg(list + i));
-                if (key > v1) cand = min(cand, key);
-            }
-            cand = __reduce_min_sync(0xFFFFFFFFu, cand);
-            if (lane == 0 && cand != 0xFFFFFFFFu) atomicMin(&ls.v2, cand);
-            __syncthreads();
-            v2 = ls.v2;
-            if (v2 == 0xFFFFFFFFu) ok = false;
-        }
-    }
-    __syncthreads();
-}
-
-// ---------------------------------------------------------------------------------------
-// 2./3. streaming kernels
+// 2./4. streaming kernels
 // ---------------------------------------------------------------------------------------
 // Exclusive scan of `n` over the lanes of a warp that share the same quad index
 // (lanes q, q + NQ, q + 2 NQ, ...); returns the exclusive prefix and the group total.
@@ -241,7 +162,7 @@ __device__ __forceinline__ int group_sum(int v) {
 // MODE 0: median sweep.  MODE 1: MAD + exceedance sweep.
 template <int NQ, int MODE, typename MaskT>
 __global__ void __launch_bounds__(kBrThreads) xrank_stream_kernel(const XrankArgs a, const MetricParams p,
-                                                                 const XrankScratch sc, const int chunks) {
+                                                                 const XrankScratch sc) {
     constexpr int M = 4 * NQ;
     constexpr int LPI = kBrThreads / NQ;       // rank lanes per iteration
     constexpr int CHUNK = LPI * kRPT;          // ranks per CTA
@@ -250,12 +171,10 @@ __global__ void __launch_bounds__(kBrThreads) xrank_stream_kernel(const XrankArg
     __shared__ uint32_t s_cnt[M], s_ncand[M], s_base[M];
     __shared__ uint32_t s_amb[MODE == 1 ? kCtaAmb : 1];
     __shared__ uint32_t s_namb, s_ambbase;
-    __shared__ int s_overflow, s_last;
-    __shared__ float s_val[M], s_rhs[M];
-    __shared__ ListSel ls;
+    __shared__ int s_overflow;
 
     const int t = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x, lane = lane_id();
-    const bool skip = __ldcg(sc.flag + t) != 0;   // the step already goes to the direct path
+    if (__ldcg(sc.flag + t) != 0) return;   // the step already goes to the direct path
     const int R = a.R;
     const int slot = (int)(((long long)a.first_slot + t) % a.capacity);
     const float *row = a.base + (size_t)slot * a.row_stride;
@@ -266,7 +185,6 @@ __global__ void __launch_bounds__(kBrThreads) xrank_stream_kernel(const XrankArg
     if (tid == 0) { s_namb = 0; s_overflow = 0; }
     __syncthreads();
 
-    if (!skip) {
     float lo[4], hi[4], med[4], rlo[4], rhi[4];
     int dirv[4];
 #pragma unroll
@@ -391,112 +309,170 @@ __global__ void __launch_bounds__(kBrThreads) xrank_stream_kernel(const XrankArg
     } else if (tid == 0) {
         atomicExch(sc.flag + t, 1u);
     }
-    }  // !skip
-    // last ticket of the step finalises (a skipped step still needs its counters cleaned)
-    __threadfence();
+}
+
+// ---------------------------------------------------------------------------------------
+// 3./5. selection kernels: one CTA per (step, metric) column finishes the statistic
+// ---------------------------------------------------------------------------------------
+struct SelShared {
+    uint32_t hist[kSelBins];
+    uint32_t warp_tot[kSelThreads / 32];
+    uint32_t bin, before, cnt, vmin;
+    int found;
+};
+
+// Finds the bin of sh.hist that holds 0-based rank k (all threads; results in sh).
+__device__ __forceinline__ void cta_find_bin(SelShared &sh, uint32_t k) {
+    constexpr int BPT = kSelBins / kSelThreads;
+    const int tid = threadIdx.x, lane = lane_id(), warp = warp_id();
+    uint32_t loc[BPT], sum = 0;
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) { loc[i] = sh.hist[tid * BPT + i]; sum += loc[i]; }
+    uint32_t incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, incl, d); if (lane >= d) incl += u; }
+    if (lane == 31) sh.warp_tot[warp] = incl;
+    if (tid == 0) sh.found = 0;
     __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(sc.ticket + t, 1u) == (uint32_t)chunks - 1u);
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    bool fail = __ldcg(sc.flag + t) != 0;
-    const bool even = (R & 1) == 0;
-    const uint32_t k1 = (uint32_t)((R - 1) / 2), k2 = (uint32_t)(R / 2);
-    for (int m = 0; m < M && !fail; ++m) {
-        const uint32_t clt = __ldcg(sc.cnt_lt + so + m), n = __ldcg(sc.ncand + so + m);
-        if (!(clt <= k1 && k2 < clt + n && n <= (uint32_t)sc.cap)) {
-            if (tid == 0 && sc.reasons) atomicAdd(sc.reasons + (MODE == 0 ? kWhyMedianMiss : kWhyMadMiss), 1u);
-            fail = true;
-            break;
+    uint32_t off = 0;
+    for (int w = 0; w < warp; ++w) off += sh.warp_tot[w];
+    const uint32_t excl = off + incl - sum;
+    if (k >= excl && k < excl + sum) {
+        uint32_t run = excl;
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) {
+            if (k >= run && k < run + loc[i]) { sh.bin = (uint32_t)(tid * BPT + i); sh.before = run; sh.cnt = loc[i]; sh.found = 1; }
+            run += loc[i];
         }
-        uint32_t v1, v2;
-        bool ok;
-        cta_select_list(sc.cand + (so + m) * (size_t)sc.cap, (int)n, k1 - clt, even, ls, v1, v2, ok);
-        if (!ok) {
-            if (tid == 0 && sc.reasons) atomicAdd(sc.reasons + kWhySelect, 1u);
-            fail = true;
-            break;
-        }
-        if (tid == 0) s_val[m] = median_from_keys(v1, v2, even);
     }
     __syncthreads();
-    if (!fail) {
-        if (MODE == 0) {
-            if (tid < M) {
-                const int m = tid;
-                const float med_m = s_val[m];
-                a.med[so + m] = med_m;
-                if (a.med_user) a.med_user[so + m] = med_m;
-                // The MAD interval was measured about the sample's median.  Moving the centre
-                // to the exact median changes the count inside +-d only to second order (what
-                // one side gains the other loses), so the interval is kept, opened by one ulp.
-                float dl = sc.dlo[so + m];
-                dl = dl > 0.0f ? fdown(dl) : 0.0f;
-                float dh = sc.dhi[so + m];
-                if (dh < CUDART_INF_F) dh = fup(dh);
-                sc.dlo[so + m] = dl;
-                sc.dhi[so + m] = dh;
-                const float rel = __fmul_rn(p.floor_rel[m], fabsf(med_m));
-                sc.rhs_lo[so + m] = __fmul_rn(p.thrp[m], fmaxf(fmaxf(dl, rel), p.floor_abs[m]));
-                sc.rhs_hi[so + m] = __fmul_rn(p.thrp[m], fmaxf(fmaxf(dh, rel), p.floor_abs[m]));
-            }
-        } else {
-            if (tid < M) {
-                const int m = tid;
-                const float mad = s_val[m];
-                a.mad[so + m] = mad;
-                if (a.mad_user) a.mad_user[so + m] = mad;
-                s_rhs[m] = __fmul_rn(p.thrp[m], scale_of(mad, a.med[so + m], p.floor_rel[m], p.floor_abs[m]));
+}
+
+// MODE 0: median of the column from the elements collected inside [lo, hi].
+// MODE 1: MAD from those inside [dlo, dhi], then the deferred exceedance decisions.
+template <int MODE, typename MaskT>
+__global__ void __launch_bounds__(kSelThreads) xrank_select_kernel(const XrankArgs a, const MetricParams p, const XrankScratch sc) {
+    __shared__ SelShared sh;
+    const int m = blockIdx.x, t = blockIdx.y, tid = threadIdx.x, lane = lane_id();
+    const int R = a.R, M = a.M;
+    const size_t so = (size_t)t * M, col = so + m;
+    const uint32_t clt = __ldcg(sc.cnt_lt + col), n = __ldcg(sc.ncand + col);
+    __syncthreads();
+    // leave the counters clean for the next sweep / launch (every thread has read them)
+    if (tid == 0) {
+        sc.cnt_lt[col] = 0;
+        sc.ncand[col] = 0;
+        if (MODE == 0 && m == 0) sc.namb[t] = 0;
+    }
+    if (__ldcg(sc.flag + t) != 0) return;
+    const bool even = (R & 1) == 0;
+    const uint32_t k1 = (uint32_t)((R - 1) / 2), k2 = (uint32_t)(R / 2);
+    int why = -1;
+    if (!(clt <= k1 && k2 < clt + n && n <= (uint32_t)sc.cap)) why = (MODE == 0 ? kWhyMedianMiss : kWhyMadMiss);
+    uint32_t v1 = 0, v2 = 0;
+    if (why < 0) {
+        const uint32_t *list = sc.cand + col * (size_t)sc.cap;
+        const float flo = (MODE == 0 ? sc.lo : sc.dlo)[col], fhi = (MODE == 0 ? sc.hi : sc.dhi)[col];
+        // key range of the collected elements (a float compare accepts both zeros)
+        uint32_t base = f2key(flo == 0.0f ? -0.0f : flo);
+        uint32_t width = f2key(fhi == 0.0f ? 0.0f : fhi) - base;
+        uint32_t krem = k1 - clt, ceq = 0;
+        for (;;) {
+            const int bits = 32 - __clz(width);
+            const int shv = bits > 11 ? bits - 11 : 0;
+            for (int i = tid; i < kSelBins; i += kSelThreads) sh.hist[i] = 0;
+            __syncthreads();
+            for (uint32_t i = tid; i < n; i += kSelThreads) {
+                const uint32_t off = key_of_bits(__ldcg(list + i)) - base;
+                if (off <= width) atomicAdd(&sh.hist[off >> shv], 1u);
             }
             __syncthreads();
-            if (a.mask_base) {
-                const uint32_t n = __ldcg(sc.namb + t);
-                for (uint32_t i = tid; i < n; i += kBrThreads) {
-                    const uint32_t e = __ldcg(sc.amb + (size_t)t * sc.amb_cap + i);
-                    const uint32_t r = e >> 5, m = e & 31u;
-                    if (exceeds(row[(size_t)r * M + m], a.med[so + m], p.dir[m], s_rhs[m])) {
-                        const size_t idx = (size_t)slot * R + r;
-                        if (sizeof(MaskT) == 1) {
-                            unsigned int *w = reinterpret_cast<unsigned int *>(reinterpret_cast<uintptr_t>(a.mask_base) + (idx & ~(size_t)3));
-                            atomicOr(w, (1u << m) << (8 * (idx & 3)));
-                        } else {
-                            atomicOr(reinterpret_cast<unsigned int *>(a.mask_base) + idx, 1u << m);
-                        }
+            cta_find_bin(sh, krem);
+            if (!sh.found) { why = kWhySelect; break; }
+            krem -= sh.before;
+            if (shv == 0) { v1 = base + sh.bin; ceq = sh.cnt; break; }
+            base += sh.bin << shv;
+            width = (1u << shv) - 1u;
+            __syncthreads();
+        }
+        v2 = v1;
+        if (why < 0 && even && krem + 1 >= ceq) {   // next order statistic: smallest key above v1
+            if (tid == 0) sh.vmin = 0xFFFFFFFFu;
+            __syncthreads();
+            uint32_t cand = 0xFFFFFFFFu;
+            for (uint32_t i = tid; i < n; i += kSelThreads) {
+                const uint32_t key = key_of_bits(__ldcg(list + i));
+                if (key > v1) cand = min(cand, key);
+            }
+            cand = __reduce_min_sync(0xFFFFFFFFu, cand);
+            if (lane == 0 && cand != 0xFFFFFFFFu) atomicMin(&sh.vmin, cand);
+            __syncthreads();
+            v2 = sh.vmin;
+            if (v2 == 0xFFFFFFFFu) why = kWhySelect;
+        }
+    }
+    if (why >= 0) {
+        if (tid == 0) {
+            if (sc.reasons) atomicAdd(sc.reasons + why, 1u);
+            atomicExch(sc.flag + t, 1u);
+        }
+        return;
+    }
+    const float val = median_from_keys(v1, v2, even);
+    if (MODE == 0) {
+        if (tid == 0) {
+            a.med[col] = val;
+            if (a.med_user) a.med_user[col] = val;
+            // range of the exceedance threshold over the MAD interval
+            const float rel = __fmul_rn(p.floor_rel[m], fabsf(val));
+            sc.rhs_lo[col] = __fmul_rn(p.thrp[m], fmaxf(fmaxf(sc.dlo[col], rel), p.floor_abs[m]));
+            sc.rhs_hi[col] = __fmul_rn(p.thrp[m], fmaxf(fmaxf(sc.dhi[col], rel), p.floor_abs[m]));
+        }
+    } else {
+        const float med = a.med[col];
+        if (tid == 0) {
+            a.mad[col] = val;
+            if (a.mad_user) a.mad_user[col] = val;
+        }
+        if (a.mask_base) {
+            // settle the elements whose exceedance depended on the exact MAD
+            const float rhs = __fmul_rn(p.thrp[m], scale_of(val, med, p.floor_rel[m], p.floor_abs[m]));
+            const int slot = (int)(((long long)a.first_slot + t) % a.capacity);
+            const float *row = a.base + (size_t)slot * a.row_stride;
+            const uint32_t na = __ldcg(sc.namb + t);
+            for (uint32_t i = tid; i < na; i += kSelThreads) {
+                const uint32_t e = __ldcg(sc.amb + (size_t)t * sc.amb_cap + i);
+                if ((int)(e & 31u) != m) continue;
+                const uint32_t r = e >> 5;
+                if (exceeds(row[(size_t)r * M + m], med, p.dir[m], rhs)) {
+                    const size_t idx = (size_t)slot * R + r;
+                    if (sizeof(MaskT) == 1) {
+                        unsigned int *w = reinterpret_cast<unsigned int *>(reinterpret_cast<uintptr_t>(a.mask_base) + (idx & ~(size_t)3));
+                        atomicOr(w, (1u << m) << (8 * (idx & 3)));
+                    } else {
+                        atomicOr(reinterpret_cast<unsigned int *>(a.mask_base) + idx, 1u << m);
                     }
                 }
             }
         }
-    } else if (tid == 0) {
-        atomicExch(sc.flag + t, 1u);
     }
-    // leave the counters clean for the next sweep / launch
-    if (tid < M) { sc.cnt_lt[so + tid] = 0; sc.ncand[so + tid] = 0; }
-    if (tid == 0) { sc.ticket[t] = 0; sc.namb[t] = 0; }
-}
-
-template <int NQ, int MODE>
-cudaError_t launch_stream(const XrankArgs &a, const MetricParams &p, const XrankScratch &sc, int S, cudaStream_t st) {
-    constexpr int CHUNK = (kBrThreads / NQ) * kRPT;
-    const int chunks = (a.R + CHUNK - 1) / CHUNK;
-    dim3 grid(chunks, S);
-    if (a.mask_bytes == 4)
-        xrank_stream_kernel<NQ, MODE, uint32_t><<<grid, kBrThreads, 0, st>>>(a, p, sc, chunks);
-    else
-        xrank_stream_kernel<NQ, MODE, uint8_t><<<grid, kBrThreads, 0, st>>>(a, p, sc, chunks);
-    return cudaGetLastError();
 }
 
 template <int NQ>
-cudaError_t launch_both(const XrankArgs &a, const MetricParams &p, const XrankScratch &sc, int S, cudaStream_t st) {
-    cudaError_t e = launch_stream<NQ, 0>(a, p, sc, S, st);
-    if (e != cudaSuccess) return e;
-    return launch_stream<NQ, 1>(a, p, sc, S, st);
-}
-
-int sample_size(int R, int M) {
-    int s = 1024;
-    while (s > 64 && (s * M > 8192 || s * 4 > R)) s >>= 1;
-    return s;
+cudaError_t launch_phases(const XrankArgs &a, const MetricParams &p, const XrankScratch &sc, int S, cudaStream_t st) {
+    constexpr int CHUNK = (kBrThreads / NQ) * kRPT;
+    const int chunks = (a.R + CHUNK - 1) / CHUNK;
+    const dim3 sgrid(chunks, S), cgrid(a.M, S);
+    const bool wide = a.mask_bytes == 4;
+    if (wide) xrank_stream_kernel<NQ, 0, uint32_t><<<sgrid, kBrThreads, 0, st>>>(a, p, sc);
+    else xrank_stream_kernel<NQ, 0, uint8_t><<<sgrid, kBrThreads, 0, st>>>(a, p, sc);
+    if (wide) xrank_select_kernel<0, uint32_t><<<cgrid, kSelThreads, 0, st>>>(a, p, sc);
+    else xrank_select_kernel<0, uint8_t><<<cgrid, kSelThreads, 0, st>>>(a, p, sc);
+    if (wide) xrank_stream_kernel<NQ, 1, uint32_t><<<sgrid, kBrThreads, 0, st>>>(a, p, sc);
+    else xrank_stream_kernel<NQ, 1, uint8_t><<<sgrid, kBrThreads, 0, st>>>(a, p, sc);
+    if (wide) xrank_select_kernel<1, uint32_t><<<cgrid, kSelThreads, 0, st>>>(a, p, sc);
+    else xrank_select_kernel<1, uint8_t><<<cgrid, kSelThreads, 0, st>>>(a, p, sc);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -522,11 +498,11 @@ int xrank_scratch_steps(int R, int M, int want) {
 }
 
 size_t xrank_scratch_small_bytes(int M, int S_max) {
-    return (size_t)S_max * (2 * M + 3) * sizeof(uint32_t);
+    return (size_t)S_max * (2 * M + 2) * sizeof(uint32_t);
 }
 
 size_t xrank_scratch_big_bytes(int R, int M, int S_max) {
-    return (size_t)S_max * M * 7 * sizeof(float) + (size_t)S_max * M * xrank_cand_cap(R) * 4 +
+    return (size_t)S_max * M * 6 * sizeof(float) + (size_t)S_max * M * xrank_cand_cap(R) * 4 +
            (size_t)S_max * xrank_amb_cap(R, M) * 4;
 }
 
@@ -538,13 +514,11 @@ XrankScratch carve_xrank_scratch(void *small_base, void *big_base, int R, int M,
     uint32_t *u = (uint32_t *)small_base;   // zero-initialised state
     sc.cnt_lt = u; u += (size_t)S_max * M;
     sc.ncand = u;  u += (size_t)S_max * M;
-    sc.ticket = u; u += S_max;
     sc.flag = u;   u += S_max;
     sc.namb = u;
     float *f = (float *)big_base;
     sc.lo = f;     f += (size_t)S_max * M;
     sc.hi = f;     f += (size_t)S_max * M;
-    sc.center = f; f += (size_t)S_max * M;
     sc.dlo = f;    f += (size_t)S_max * M;
     sc.dhi = f;    f += (size_t)S_max * M;
     sc.rhs_lo = f; f += (size_t)S_max * M;
@@ -554,23 +528,28 @@ XrankScratch carve_xrank_scratch(void *small_base, void *big_base, int R, int M,
     return sc;
 }
 
-// Runs the bracketed path on S <= scratch.S_max steps, then the direct kernel on the
-// steps it flagged.  a.med / a.mad must hold S * M floats.
+// Runs the bracketed path on S <= scratch.S_max steps (sample, then one streaming sweep and
+// one per-column selection for the median and again for the MAD), then the direct kernel on
+// the steps it flagged.  a.med / a.mad must hold S * M floats.  Six launches.
 cudaError_t launch_xrank_bracketed(const XrankArgs &a, const MetricParams &p, const XrankScratch &sc, int S,
                                    cudaStream_t st) {
     if (S <= 0) return cudaSuccess;
-    const int s = sample_size(a.R, a.M);
+    const int epl = a.M <= 8 ? 32 : (a.M == 16 ? 16 : 8);
+    const int s = 32 * epl;
     // half-width of the sampled interval in sample ranks: 5.5 standard deviations of a sample
     // quantile's rank (0.5 sqrt(s)), so that a miss (and the slow direct redo) is a ~1e-7 event
     const int delta = (int)ceil(5.5 * 0.5 * sqrt((double)s));
-    xrank_sample_kernel<<<S, kSampleThreads, (size_t)s * a.M * sizeof(uint32_t), st>>>(a, sc, s, delta);
+    const size_t smem = (size_t)s * a.M * sizeof(uint32_t);
+    if (epl == 32) xrank_sample_kernel<32><<<S, 32 * a.M, smem, st>>>(a, sc, delta);
+    else if (epl == 16) xrank_sample_kernel<16><<<S, 32 * a.M, smem, st>>>(a, sc, delta);
+    else xrank_sample_kernel<8><<<S, 32 * a.M, smem, st>>>(a, sc, delta);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     switch (a.M) {
-        case 4: e = launch_both<1>(a, p, sc, S, st); break;
-        case 8: e = launch_both<2>(a, p, sc, S, st); break;
-        case 16: e = launch_both<4>(a, p, sc, S, st); break;
-        case 32: e = launch_both<8>(a, p, sc, S, st); break;
+        case 4: e = launch_phases<1>(a, p, sc, S, st); break;
+        case 8: e = launch_phases<2>(a, p, sc, S, st); break;
+        case 16: e = launch_phases<4>(a, p, sc, S, st); break;
+        case 32: e = launch_phases<8>(a, p, sc, S, st); break;
         default: return cudaErrorInvalidValue;
     }
     if (e != cudaSuccess) return e;
