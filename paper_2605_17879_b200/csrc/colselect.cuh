@@ -11,26 +11,40 @@ namespace guard {
 // Three-way partitioning around a median-of-three pivot; the column is permuted in
 // place (its multiset is preserved).  Each thread owns its column, so no barrier is
 // needed; with one column per lane and a row pitch that is a multiple of 32 words every
-// access of a warp is free of bank conflicts.
-__device__ __forceinline__ uint32_t col_select(uint32_t *col, int stride, int n, int k) {
+// access of a warp is free of bank conflicts.  Loads are issued in batches of eight before
+// the dependent compare / swap work, so that a thread keeps several shared-memory loads in
+// flight (few warps fit next to the tiles, latency has to be hidden inside the thread).
+// On return *below_end is the first position not known to hold a key < the result: every
+// position before it holds a key <= the result.
+constexpr int kSelBatch = 8;
+
+__device__ __forceinline__ uint32_t col_select(uint32_t *col, int stride, int n, int k, int *below_end) {
     int l = 0, r = n - 1;
     while (l < r) {
         const uint32_t a = col[(size_t)l * stride], b = col[(size_t)((l + r) >> 1) * stride],
                        c = col[(size_t)r * stride];
         const uint32_t p = max(min(a, b), min(max(a, b), c));
         int store = l, ceq = 0;
-        for (int i = l; i <= r; ++i) {
-            const uint32_t v = col[(size_t)i * stride];
-            if (v < p) {
-                col[(size_t)i * stride] = col[(size_t)store * stride];
-                col[(size_t)store * stride] = v;
-                ++store;
+        for (int i = l; i <= r; i += kSelBatch) {
+            uint32_t v[kSelBatch];
+#pragma unroll
+            for (int u = 0; u < kSelBatch; ++u) v[u] = (i + u <= r) ? col[(size_t)(i + u) * stride] : 0xFFFFFFFFu;
+#pragma unroll
+            for (int u = 0; u < kSelBatch; ++u) {
+                if (i + u <= r) {
+                    if (v[u] < p) {   // earlier swaps of this batch never touch position i + u
+                        col[(size_t)(i + u) * stride] = col[(size_t)store * stride];
+                        col[(size_t)store * stride] = v[u];
+                        ++store;
+                    }
+                    ceq += (v[u] == p);
+                }
             }
-            ceq += (v == p);
         }
         if (k < store) {
             r = store - 1;
         } else if (k < store + ceq) {
+            *below_end = store;
             return p;
         } else {
             int s2 = store;
@@ -45,28 +59,32 @@ __device__ __forceinline__ uint32_t col_select(uint32_t *col, int stride, int n,
             l = s2;
         }
     }
+    *below_end = l;
     return col[(size_t)l * stride];
 }
 
-// Given v = the key of 0-based rank k, the key of rank k + 1: v again if more than k + 1
-// keys are <= v, else the smallest key above v.
-__device__ __forceinline__ uint32_t col_next(const uint32_t *col, int stride, int n, int k, uint32_t v) {
-    int cle = 0;
-    uint32_t above = 0xFFFFFFFFu;
-    for (int i = 0; i < n; ++i) {
-        const uint32_t x = col[(size_t)i * stride];
-        cle += (x <= v);
-        if (x > v) above = min(above, x);
-    }
-    return (cle > k + 1) ? v : above;
-}
-
-// Median of a column of keys (midpoint rule for even n).
+// Median of a column of keys (midpoint rule for even n).  For even n the upper middle
+// element (rank n/2) is selected; the lower middle one is then the largest key among the
+// positions the partitioning left before it.
 __device__ __forceinline__ float col_median(uint32_t *col, int stride, int n) {
-    const int k = (n - 1) >> 1;
-    const uint32_t v1 = col_select(col, stride, n, k);
-    if (n & 1) return key2f(v1);
-    const uint32_t v2 = col_next(col, stride, n, k, v1);
+    int below_end;
+    const int k = n >> 1;   // n odd: the middle; n even: the upper middle
+    const uint32_t v2 = col_select(col, stride, n, k, &below_end);
+    if (n & 1) return key2f(v2);
+    // rank k - 1: equal to v2 if a further copy of it sits at or before position k - 1,
+    // i.e. if fewer than k keys are strictly below v2; otherwise the maximum of the keys
+    // strictly below v2, all of which lie in positions [0, below_end).
+    uint32_t v1 = v2;
+    if (below_end >= k) {
+        v1 = 0;
+        for (int i = 0; i < below_end; i += kSelBatch) {
+            uint32_t v[kSelBatch];
+#pragma unroll
+            for (int u = 0; u < kSelBatch; ++u) v[u] = (i + u < below_end) ? col[(size_t)(i + u) * stride] : 0u;
+#pragma unroll
+            for (int u = 0; u < kSelBatch; ++u) v1 = max(v1, v[u]);
+        }
+    }
     return median_from_keys(v1, v2, true);
 }
 

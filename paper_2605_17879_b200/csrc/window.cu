@@ -47,10 +47,165 @@ __global__ void __launch_bounds__(TC) window_select_kernel(const WindowArgs a, c
     }
     if (tid >= ncols) return;
     uint32_t *col = tile + tid;
-    for (int j = 0; j < n; ++j) col[(size_t)j * TC] = key_of_bits(col[(size_t)j * TC]);
+    for (int j = 0; j < n; j += kSelBatch) {   // raw bits -> order-preserving keys, loads batched
+        uint32_t v[kSelBatch];
+#pragma unroll
+        for (int u = 0; u < kSelBatch; ++u) v[u] = (j + u < n) ? col[(size_t)(j + u) * TC] : 0u;
+#pragma unroll
+        for (int u = 0; u < kSelBatch; ++u)
+            if (j + u < n) col[(size_t)(j + u) * TC] = key_of_bits(v[u]);
+    }
     const float med = col_median(col, TC, n);
     a.wmed[col0 + tid] = med;
     if (a.wmed_user) a.wmed_user[col0 + tid] = med;
+}
+
+// ---------------------------------------------------------------------------------------
+// Warp-per-series path for windows of up to 256 steps: the window of one series lives in
+// the registers of one warp (VPL keys per lane), so no shared-memory column limits the
+// number of resident warps.  A CTA of 32 warps handles a tile of 32 adjacent series; tiles
+// are staged with cp.async into a padded (pitch 33) double buffer so that both the row-wise
+// fill and the column-wise read are free of bank conflicts.
+// Selection: every lane sorts its own keys (odd-even merge network), then the warp narrows
+// [lo, hi] around the wanted rank: the lane with the longest still-active run proposes its
+// middle key as pivot, every lane counts its keys below / not above the pivot, one
+// __reduce_add_sync gives the pivot's global rank.  The pivot is always a key that is still
+// active and leaves the active set, so the loop ends after at most n rounds (about seven in
+// practice for n = 200).
+// ---------------------------------------------------------------------------------------
+constexpr int kWarpTileCols = 32;
+constexpr int kWarpPitch = 33;
+
+template <int VPL>
+__device__ __forceinline__ void lane_sort(uint32_t (&v)[VPL]) {
+#pragma unroll
+    for (int p = 1; p < VPL; p <<= 1)
+#pragma unroll
+        for (int k = p; k >= 1; k >>= 1)
+#pragma unroll
+            for (int j = k % p; j + k < VPL; j += 2 * k)
+#pragma unroll
+                for (int i = 0; i < k; ++i)
+                    if ((i + j) / (2 * p) == (i + j + k) / (2 * p)) {
+                        const uint32_t x = v[i + j], y = v[i + j + k];
+                        v[i + j] = min(x, y);
+                        v[i + j + k] = max(x, y);
+                    }
+}
+
+template <int VPL>
+__device__ __forceinline__ uint32_t lane_pick(const uint32_t (&v)[VPL], int idx) {
+    uint32_t r = v[0];
+#pragma unroll
+    for (int i = 1; i < VPL; ++i) r = (idx == i) ? v[i] : r;
+    return r;
+}
+
+__device__ __forceinline__ void cp_async4(void *dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int VPL>
+__global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a, const int ntiles) {
+    extern __shared__ __align__(16) uint32_t wbuf[];   // 2 x [n][kWarpPitch]
+    const int tid = threadIdx.x, lane = lane_id(), w = warp_id();
+    const int n = a.n;
+    const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;
+    const int bufwords = n * kWarpPitch;
+    const int kq = n >> 1;   // n odd: the middle; n even: the upper middle
+
+    auto stage = [&](int tile, uint32_t *buf) {
+        const int col0 = tile * kWarpTileCols;
+        for (int e = tid; e < n * kWarpTileCols; e += 1024) {
+            const int row = e >> 5, c = e & 31;
+            int slot = first + row;
+            if (slot >= a.capacity) slot -= a.capacity;
+            if (col0 + c < a.series) cp_async4(buf + row * kWarpPitch + c, a.ring + (size_t)slot * a.row_stride + col0 + c);
+        }
+        cp_async_commit();
+    };
+
+    int cur = 0;
+    if ((int)blockIdx.x < ntiles) stage(blockIdx.x, wbuf);
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int next = tile + gridDim.x;
+        if (next < ntiles) {
+            stage(next, wbuf + (cur ^ 1) * bufwords);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const uint32_t *buf = wbuf + cur * bufwords;
+        const int series = tile * kWarpTileCols + w;
+        if (series < a.series) {
+            uint32_t kv[VPL];
+            int nreal = 0;
+#pragma unroll
+            for (int i = 0; i < VPL; ++i) {
+                const int row = lane + 32 * i;
+                const bool real = row < n;
+                kv[i] = real ? key_of_bits(buf[row * kWarpPitch + w]) : 0xFFFFFFFFu;
+                nreal += real;
+            }
+            lane_sort<VPL>(kv);
+            int lo_i = 0, hi_i = nreal;   // this lane's active run [lo_i, hi_i)
+            uint32_t v2 = 0, v1 = 0;
+            bool found = false;
+            for (int round = 0; round < 320; ++round) {
+                const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, ((uint32_t)(hi_i - lo_i) << 5) | (uint32_t)lane);
+                if ((best >> 5) == 0) break;
+                const uint32_t prop = lane_pick<VPL>(kv, (lo_i + hi_i) >> 1);
+                const uint32_t p = __shfl_sync(0xFFFFFFFFu, prop, best & 31u);
+                int clt = 0, cle = 0;
+#pragma unroll
+                for (int i = 0; i < VPL; ++i) {
+                    clt += (kv[i] < p);
+                    cle += (kv[i] <= p);
+                }
+                const uint32_t tot = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)clt | ((uint32_t)cle << 16));
+                const int tlt = (int)(tot & 0xFFFFu), tle = (int)(tot >> 16);
+                if (kq < tlt) {
+                    hi_i = clt;
+                } else if (kq >= tle) {
+                    lo_i = cle;
+                } else {
+                    v2 = p;
+                    v1 = p;
+                    if (!(n & 1) && tlt == kq) {   // lower middle: the largest key below the pivot
+                        const uint32_t below = clt > 0 ? lane_pick<VPL>(kv, clt - 1) : 0u;
+                        v1 = __reduce_max_sync(0xFFFFFFFFu, below);
+                    }
+                    found = true;
+                    break;
+                }
+            }
+            if (lane == 0) {
+                if (!found) atomicOr(a.status, kStatInternal);
+                const float med = median_from_keys(v1, v2, !(n & 1));
+                a.wmed[series] = med;
+                if (a.wmed_user) a.wmed_user[series] = med;
+            }
+        }
+        __syncthreads();
+        cur ^= 1;
+    }
+}
+
+template <int VPL>
+cudaError_t launch_warp_path(const WindowArgs &a, cudaStream_t st) {
+    const size_t smem = 2 * (size_t)a.n * kWarpPitch * 4;
+    cudaError_t e = cudaFuncSetAttribute(window_warp_kernel<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int ntiles = (a.series + kWarpTileCols - 1) / kWarpTileCols;
+    const int grid = ntiles < 2 * sms ? ntiles : 2 * sms;
+    window_warp_kernel<VPL><<<grid, 1024, smem, st>>>(a, ntiles);
+    return cudaGetLastError();
 }
 
 // Fallback for windows too long to stage: one thread per series, bit-by-bit counting
@@ -112,6 +267,9 @@ cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st) {
     // bulk copies need 16-byte aligned sources and sizes
     const int use_bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
     const size_t n = (size_t)a.n;
+    if (n <= 64) return launch_warp_path<2>(a, st);
+    if (n <= 128) return launch_warp_path<4>(a, st);
+    if (n <= 256) return launch_warp_path<8>(a, st);
     if (n * 128 * 4 <= kMaxTile) return launch_staged<128>(a, use_bulk, st);
     if (n * 64 * 4 <= kMaxTile) return launch_staged<64>(a, use_bulk, st);
     if (n * 32 * 4 <= kMaxTile) return launch_staged<32>(a, use_bulk, st);

@@ -107,8 +107,9 @@ def test_in_place_ingest_equals_copy_ingest():
 
 
 def test_long_window_paths():
-    # windows too long for a 128-column tile (64- and 32-column tiles), and the global-memory fallback
-    for W, R in ((500, 24), (1200, 8), (2000, 4)):
+    # windows too long for the warp-per-series path: 128-, 64- and 32-column staged tiles, and the
+    # global-memory fallback
+    for W, R in ((300, 40), (500, 24), (1200, 8), (2000, 4)):
         X, dirs = _rand_fleet(W + 7, R, 4, seed=W)
         run_both(X, W, W // 2, 2, dirs, [W, 7], capacity=W + 16, score_every=1)
 

@@ -39,16 +39,18 @@ def test_static_scratch_topk_matches_score_twice_in_a_row():
     assert not torch.equal(ref_a["topk_idx"], ref_b["topk_idx"])
     idx = torch.empty(K, dtype=torch.int32, device="cuda")
     sc = torch.empty(K, dtype=torch.float32, device="cuda")
-    before = torch.cuda.memory_allocated()
     for ref in (ref_a, ref_b, ref_a):
         idx.fill_(-1)
         sc.fill_(float("nan"))
+        torch.cuda.synchronize()
+        before = torch.cuda.memory_stats()["allocation.all.allocated"]
         guard.topk_static(ref["wmed"], ref["fleet_med"], ref["fleet_mad"], K, dir=dirs, out_idx=idx, out_score=sc)
         torch.cuda.synchronize()
+        # the call itself went nowhere near torch's device allocator either
+        assert torch.cuda.memory_stats()["allocation.all.allocated"] == before
         assert torch.equal(idx, ref["topk_idx"])
         got, want = sc.cpu().numpy().astype(np.float64), ref["topk_score"].cpu().numpy().astype(np.float64)
         assert np.allclose(got, want, rtol=1e-6, atol=1e-30)
-    assert torch.cuda.memory_allocated() == before      # torch's allocator was not touched either
 
 
 def test_static_scratch_limits_are_rejected():
