@@ -64,17 +64,23 @@ __global__ void __launch_bounds__(TC) window_select_kernel(const WindowArgs a, c
 // Warp-per-series path for windows of up to 256 steps: the window of one series lives in
 // the registers of one warp (VPL keys per lane), so no shared-memory column limits the
 // number of resident warps.  A CTA of 32 warps handles a tile of 32 adjacent series; tiles
-// are staged with cp.async into a padded (pitch 33) double buffer so that both the row-wise
-// fill and the column-wise read are free of bank conflicts.
-// Selection: every lane sorts its own keys (odd-even merge network), then the warp narrows
-// [lo, hi] around the wanted rank: the lane with the longest still-active run proposes its
-// middle key as pivot, every lane counts its keys below / not above the pivot, one
-// __reduce_add_sync gives the pivot's global rank.  The pivot is always a key that is still
-// active and leaves the active set, so the loop ends after at most n rounds (about seven in
-// practice for n = 200).
+// are staged into a double buffer with one bulk asynchronous copy (TMA) per ring row onto
+// an mbarrier per buffer (plain cp.async when rows are not 16-byte aligned).  Rows are
+// pitched 36 words apart: 16-byte aligned for the bulk copy, and a column read then costs
+// four shared-memory wavefronts instead of thirty-two.
+//
+// Selection: every lane sorts its own keys (odd-even merge network).  The median of the
+// lanes' middle keys (a 32-key bitonic sort over shuffles) is a pivot within a few ranks of
+// the wanted one; every lane counts its keys below / not above the pivot and one
+// __reduce_add_sync gives the pivot's global rank.  From there the warp walks rank by rank
+// (each lane offers its next key, __reduce_min/max_sync picks the winner) until it passes
+// the wanted rank; if the pivot turns out to be far off, further pivot rounds (middle key of
+// the longest still-active run) narrow the distance first.  Every round removes at least its
+// pivot from the active set, so the loop is bounded by the window length.
 // ---------------------------------------------------------------------------------------
 constexpr int kWarpTileCols = 32;
-constexpr int kWarpPitch = 33;
+constexpr int kWarpPitch = 36;
+constexpr int kWalkMax = 24;     // walk when the wanted rank is at most this far from the pivot
 
 template <int VPL>
 __device__ __forceinline__ void lane_sort(uint32_t (&v)[VPL]) {
@@ -101,6 +107,20 @@ __device__ __forceinline__ uint32_t lane_pick(const uint32_t (&v)[VPL], int idx)
     return r;
 }
 
+// Ascending sort of one key per lane; returns the key of sorted position `pos`.
+__device__ __forceinline__ uint32_t warp_sorted_at(uint32_t x, int pos) {
+    const int lane = lane_id();
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1)
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, x, stride);
+            const bool asc = (lane & size) == 0, upper = (lane & stride) != 0;
+            x = (asc != upper) ? min(x, o) : max(x, o);
+        }
+    return __shfl_sync(0xFFFFFFFFu, x, pos);
+}
+
 __device__ __forceinline__ void cp_async4(void *dst, const void *src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
@@ -108,37 +128,140 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// Median of the n keys held by the warp (kv sorted ascending per lane, padded with
+// 0xFFFFFFFF; nreal real keys in this lane).  Returns false if the loop bound was hit.
 template <int VPL>
-__global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a, const int ntiles) {
-    extern __shared__ __align__(16) uint32_t wbuf[];   // 2 x [n][kWarpPitch]
+__device__ __forceinline__ bool warp_median(const uint32_t (&kv)[VPL], const int nreal, const int n, float &med) {
+    const int lane = lane_id();
+    const bool even = !(n & 1);
+    const int kq = n >> 1;             // upper middle rank (the middle for odd n)
+    int lo_i = 0, hi_i = nreal;        // this lane's active run [lo_i, hi_i)
+    uint32_t v1 = 0, v2 = 0;
+    // first pivot: median of the lanes' middle keys
+    const unsigned have = __ballot_sync(0xFFFFFFFFu, nreal > 0);
+    uint32_t p = warp_sorted_at(nreal > 0 ? lane_pick<VPL>(kv, nreal >> 1) : 0xFFFFFFFFu, __popc(have) >> 1);
+    for (int round = 0; round < 300; ++round) {
+        int clt = 0, cle = 0;
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) {
+            clt += (kv[i] < p);
+            cle += (kv[i] <= p);
+        }
+        const uint32_t tot = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)clt | ((uint32_t)cle << 16));
+        const int tlt = (int)(tot & 0xFFFFu), tle = (int)(tot >> 16);   // ranks [tlt, tle) hold p
+        if (kq >= tlt && kq < tle) {
+            v2 = p;
+            v1 = p;
+            if (even && kq == tlt) {   // lower middle: the largest key below the pivot
+                v1 = __reduce_max_sync(0xFFFFFFFFu, clt > 0 ? lane_pick<VPL>(kv, clt - 1) : 0u);
+            }
+            med = median_from_keys(v1, v2, even);
+            return true;
+        }
+        if (kq >= tle) {
+            lo_i = cle;
+            if (kq - tle < kWalkMax) {   // walk upwards: ranks tle, tle + 1, ...
+                int cur = tle, nxt = cle;
+                v1 = p;                  // rank kq - 1 if it is still inside the pivot's run
+                for (int step = 0; step <= kWalkMax; ++step) {
+                    const uint32_t prop = nxt < nreal ? lane_pick<VPL>(kv, nxt) : 0xFFFFFFFFu;
+                    const uint32_t m = __reduce_min_sync(0xFFFFFFFFu, prop);
+                    const bool is = (prop == m) && (nxt < nreal);
+                    const int c = __popc(__ballot_sync(0xFFFFFFFFu, is));
+                    if (kq - 1 >= cur && kq - 1 < cur + c) v1 = m;
+                    if (kq < cur + c) {
+                        med = even ? median_from_keys(v1, m, true) : key2f(m);
+                        return true;
+                    }
+                    nxt += is;
+                    cur += c;
+                }
+                return false;
+            }
+        } else {
+            hi_i = clt;
+            if (tlt - kq <= kWalkMax) {  // walk downwards: ranks tlt - 1, tlt - 2, ...
+                int cur = tlt, nxt = clt;   // ranks [.., cur) are still below; this lane's next is kv[nxt - 1]
+                for (int step = 0; step <= kWalkMax + 1; ++step) {
+                    const uint32_t prop = nxt > 0 ? lane_pick<VPL>(kv, nxt - 1) : 0u;
+                    const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, prop);
+                    const bool is = (prop == m) && (nxt > 0);
+                    const int c = __popc(__ballot_sync(0xFFFFFFFFu, is));
+                    if (c == 0) return false;
+                    // ranks [cur - c, cur) hold m
+                    if (kq >= cur - c && kq < cur) v2 = m;
+                    if (kq - 1 >= cur - c) {     // rank kq - 1 (or, for odd n, rank kq) reached
+                        if (!even) { med = key2f(v2); return true; }
+                        med = median_from_keys(m, v2, true);
+                        return true;
+                    }
+                    nxt -= is;
+                    cur -= c;
+                }
+                return false;
+            }
+        }
+        // far off: next pivot is the middle key of the longest still-active run
+        const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, ((uint32_t)(hi_i - lo_i) << 5) | (uint32_t)lane);
+        if ((best >> 5) == 0) return false;
+        p = __shfl_sync(0xFFFFFFFFu, lane_pick<VPL>(kv, (lo_i + hi_i) >> 1), best & 31u);
+    }
+    return false;
+}
+
+template <int VPL>
+__global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a, const int ntiles, const int use_bulk) {
+    extern __shared__ __align__(128) uint32_t wbuf[];   // 2 x [n][kWarpPitch]
+    __shared__ __align__(8) uint64_t bar[2];
     const int tid = threadIdx.x, lane = lane_id(), w = warp_id();
     const int n = a.n;
     const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;
     const int bufwords = n * kWarpPitch;
-    const int kq = n >> 1;   // n odd: the middle; n even: the upper middle
 
-    auto stage = [&](int tile, uint32_t *buf) {
+    auto stage = [&](int tile, int b) {
+        uint32_t *buf = wbuf + b * bufwords;
         const int col0 = tile * kWarpTileCols;
-        for (int e = tid; e < n * kWarpTileCols; e += 1024) {
-            const int row = e >> 5, c = e & 31;
-            int slot = first + row;
-            if (slot >= a.capacity) slot -= a.capacity;
-            if (col0 + c < a.series) cp_async4(buf + row * kWarpPitch + c, a.ring + (size_t)slot * a.row_stride + col0 + c);
+        const int ncols = min(kWarpTileCols, a.series - col0);
+        if (use_bulk) {
+            if (tid == 0) mbar_arrive_expect_tx(&bar[b], (uint32_t)n * (uint32_t)ncols * 4u);
+            __syncthreads();   // the expectation is registered before any copy can complete
+            for (int row = tid; row < n; row += 1024) {
+                int slot = first + row;
+                if (slot >= a.capacity) slot -= a.capacity;
+                bulk_g2s(buf + row * kWarpPitch, a.ring + (size_t)slot * a.row_stride + col0, (uint32_t)ncols * 4u, &bar[b]);
+            }
+        } else {
+            for (int e = tid; e < n * kWarpTileCols; e += 1024) {
+                const int row = e >> 5, c = e & 31;
+                int slot = first + row;
+                if (slot >= a.capacity) slot -= a.capacity;
+                if (c < ncols) cp_async4(buf + row * kWarpPitch + c, a.ring + (size_t)slot * a.row_stride + col0 + c);
+            }
+            cp_async_commit();
         }
-        cp_async_commit();
     };
 
-    int cur = 0;
-    if ((int)blockIdx.x < ntiles) stage(blockIdx.x, wbuf);
-    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    if (use_bulk && tid == 0) {
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
+    }
+    __syncthreads();
+    int cur = 0, it = 0;
+    if ((int)blockIdx.x < ntiles) stage(blockIdx.x, 0);
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
         const int next = tile + gridDim.x;
-        if (next < ntiles) {
-            stage(next, wbuf + (cur ^ 1) * bufwords);
-            cp_async_wait<1>();
+        if (next < ntiles) stage(next, cur ^ 1);
+        if (use_bulk) {
+            if (!mbar_wait_bounded(&bar[cur], (uint32_t)((it >> 1) & 1), kWaitLimitCycles)) {
+                atomicOr(a.status, kStatTimeout);
+                mbar_wait_bounded(&bar[cur], (uint32_t)((it >> 1) & 1), kWaitLimitCycles);   // let copies in flight land
+                if (next < ntiles) mbar_wait_bounded(&bar[cur ^ 1], (uint32_t)(((it + 1) >> 1) & 1), kWaitLimitCycles);
+                return;
+            }
         } else {
-            cp_async_wait<0>();
+            if (next < ntiles) cp_async_wait<1>(); else cp_async_wait<0>();
+            __syncthreads();
         }
-        __syncthreads();
         const uint32_t *buf = wbuf + cur * bufwords;
         const int series = tile * kWarpTileCols + w;
         if (series < a.series) {
@@ -152,51 +275,21 @@ __global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a
                 nreal += real;
             }
             lane_sort<VPL>(kv);
-            int lo_i = 0, hi_i = nreal;   // this lane's active run [lo_i, hi_i)
-            uint32_t v2 = 0, v1 = 0;
-            bool found = false;
-            for (int round = 0; round < 320; ++round) {
-                const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, ((uint32_t)(hi_i - lo_i) << 5) | (uint32_t)lane);
-                if ((best >> 5) == 0) break;
-                const uint32_t prop = lane_pick<VPL>(kv, (lo_i + hi_i) >> 1);
-                const uint32_t p = __shfl_sync(0xFFFFFFFFu, prop, best & 31u);
-                int clt = 0, cle = 0;
-#pragma unroll
-                for (int i = 0; i < VPL; ++i) {
-                    clt += (kv[i] < p);
-                    cle += (kv[i] <= p);
-                }
-                const uint32_t tot = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)clt | ((uint32_t)cle << 16));
-                const int tlt = (int)(tot & 0xFFFFu), tle = (int)(tot >> 16);
-                if (kq < tlt) {
-                    hi_i = clt;
-                } else if (kq >= tle) {
-                    lo_i = cle;
-                } else {
-                    v2 = p;
-                    v1 = p;
-                    if (!(n & 1) && tlt == kq) {   // lower middle: the largest key below the pivot
-                        const uint32_t below = clt > 0 ? lane_pick<VPL>(kv, clt - 1) : 0u;
-                        v1 = __reduce_max_sync(0xFFFFFFFFu, below);
-                    }
-                    found = true;
-                    break;
-                }
-            }
+            float med = 0.0f;
+            const bool ok = warp_median<VPL>(kv, nreal, n, med);
             if (lane == 0) {
-                if (!found) atomicOr(a.status, kStatInternal);
-                const float med = median_from_keys(v1, v2, !(n & 1));
+                if (!ok) atomicOr(a.status, kStatInternal);
                 a.wmed[series] = med;
                 if (a.wmed_user) a.wmed_user[series] = med;
             }
         }
-        __syncthreads();
+        __syncthreads();   // every warp is done with this buffer before it is refilled
         cur ^= 1;
     }
 }
 
 template <int VPL>
-cudaError_t launch_warp_path(const WindowArgs &a, cudaStream_t st) {
+cudaError_t launch_warp_path(const WindowArgs &a, int use_bulk, cudaStream_t st) {
     const size_t smem = 2 * (size_t)a.n * kWarpPitch * 4;
     cudaError_t e = cudaFuncSetAttribute(window_warp_kernel<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -204,7 +297,7 @@ cudaError_t launch_warp_path(const WindowArgs &a, cudaStream_t st) {
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int ntiles = (a.series + kWarpTileCols - 1) / kWarpTileCols;
     const int grid = ntiles < 2 * sms ? ntiles : 2 * sms;
-    window_warp_kernel<VPL><<<grid, 1024, smem, st>>>(a, ntiles);
+    window_warp_kernel<VPL><<<grid, 1024, smem, st>>>(a, ntiles, use_bulk);
     return cudaGetLastError();
 }
 
@@ -267,9 +360,9 @@ cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st) {
     // bulk copies need 16-byte aligned sources and sizes
     const int use_bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
     const size_t n = (size_t)a.n;
-    if (n <= 64) return launch_warp_path<2>(a, st);
-    if (n <= 128) return launch_warp_path<4>(a, st);
-    if (n <= 256) return launch_warp_path<8>(a, st);
+    if (n <= 64) return launch_warp_path<2>(a, use_bulk, st);
+    if (n <= 128) return launch_warp_path<4>(a, use_bulk, st);
+    if (n <= 256) return launch_warp_path<8>(a, use_bulk, st);
     if (n * 128 * 4 <= kMaxTile) return launch_staged<128>(a, use_bulk, st);
     if (n * 64 * 4 <= kMaxTile) return launch_staged<64>(a, use_bulk, st);
     if (n * 32 * 4 <= kMaxTile) return launch_staged<32>(a, use_bulk, st);

@@ -45,6 +45,10 @@ def _rand_fleet(T, R, M, seed, quant=None, slow=True):
     (130, 9, 12, 7, 4, 30, [5], 16),              # 32-bit exceedance masks (more than 8 metrics)
     (40, 32, 8, 4, 0, 16, [8], None),             # maximum metric count, no top-k
     (257, 8, 3, 2, 16, 12, [3], 6),
+    (96, 4, 33, 17, 8, 70, [33, 2], 40),          # odd window, 2 keys per lane
+    (80, 8, 101, 51, 8, 210, [101, 4], 128),      # odd window, 4 keys per lane
+    (70, 4, 255, 128, 8, 300, [255, 3], 256),     # odd window, 8 keys per lane, ring wrap
+    (50, 3, 77, 40, 5, 160, [77, 1], 90),         # rows not 16-byte aligned: cp.async staging
 ])
 def test_small_fleets_match_oracle(R, M, W, k, K, T, blocks, cap):
     X, dirs = _rand_fleet(T, R, M, seed=R * 1000 + M)
