@@ -17,7 +17,8 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
     size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, xr_big, mask, ring, total;
-    int xr_steps;   // steps per launch of the bracketed cross-rank path (0: path not used)
+    int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
+    int xr_fused;   // the single-launch fused cross-rank path applies
 };
 
 // State and scratch first, the two rings last (the telemetry ring is by far the largest).
@@ -28,7 +29,8 @@ Layout make_layout(int R, int M, int C, int K) {
     L.ticket = off;    off = align_up(off + 64);
     L.fleet = off;     off = align_up(off + 3 * kMaxMetrics * sizeof(float));
     L.consec = off;    off = align_up(off + (size_t)R);
-    L.xr_steps = xrank_bracket_supported(R, M) ? xrank_scratch_steps(R, M, C) : 0;
+    L.xr_fused = xrank_fused_supported(R, M) ? 1 : 0;
+    L.xr_steps = (!L.xr_fused && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
     L.xr_small = off;  off = align_up(off + (L.xr_steps ? xrank_scratch_small_bytes(M, L.xr_steps) : 0));
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
@@ -123,6 +125,11 @@ struct guard_ctx {
     int mask_bytes() const { return M <= 8 ? 1 : 4; }
     // Cross-rank statistics of S rows: the bracketed path where it applies, else the direct one.
     cudaError_t xrank(XrankArgs a, int S, cudaStream_t st) {
+        if (L.xr_fused) {
+            a.fallbacks = status() + 1;
+            launches += 1;
+            return launch_xrank_fused(a, p, S, status() + 2, st);
+        }
         if (L.xr_steps == 0) { launches += 1; return launch_xrank_direct(a, p, S, st); }
         XrankScratch sc = carve_xrank_scratch(ws + L.xr_small, ws + L.xr_big, R, M, L.xr_steps);
         sc.reasons = status() + 2;

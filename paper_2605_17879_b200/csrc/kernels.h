@@ -41,6 +41,8 @@ struct XrankScratch {
     int cap, amb_cap, S_max;
 };
 enum { kWhyCtaList = 0, kWhyStepList = 1, kWhyAmbList = 2, kWhyMedianMiss = 3, kWhySelect = 4, kWhyMadMiss = 5 };
+bool xrank_fused_supported(int R, int M);
+cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, cudaStream_t st);
 bool xrank_bracket_supported(int R, int M);
 int xrank_scratch_steps(int R, int M, int want);
 size_t xrank_scratch_small_bytes(int M, int S_max);   // must be zero before first use

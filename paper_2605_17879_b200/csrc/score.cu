@@ -71,12 +71,119 @@ __global__ void __launch_bounds__(kScoreThreads) score_flag_kernel(const ScoreAr
     if (a.tier) a.tier[r] = (uint8_t)t;
 }
 
+
+// Byte-wide exceedance masks (at most 8 metrics): a CTA scores 128 ranks.  The recount over
+// the window is split over the CTA's eight warps (warp w takes steps w, w + 8, ...); every
+// thread loads the mask bytes of four adjacent ranks as one 32-bit word and accumulates
+// metric m of all four in the byte lanes of one register ((word >> m) & 0x01010101), so a
+// window step costs one coalesced 128-byte load per warp.  Partial counts meet in shared
+// memory, then one thread per rank does the scoring.
+constexpr int kFastRanks = 128;
+constexpr int kFastWarps = 8;
+
+__global__ void __launch_bounds__(kFastWarps * 32) score_flag_bytes_kernel(const ScoreArgs a, const MetricParams p) {
+    __shared__ float s_B[8], s_rhs[8], s_Ds[8];
+    const int M = a.M, tid = threadIdx.x, lane = lane_id(), w = warp_id();
+    if (tid < M) {
+        const float B = a.fleet_med[tid];
+        const float Ds = scale_of(a.fleet_mad[tid], B, p.floor_rel[tid], p.floor_abs[tid]);
+        s_B[tid] = B;
+        s_Ds[tid] = Ds;
+        s_rhs[tid] = __fmul_rn(p.thrp[tid], Ds);
+    }
+    const int r0 = blockIdx.x * kFastRanks;
+    const uint8_t *mask_base = (const uint8_t *)a.mask_base;
+    const int first = ((a.last_slot - (a.n - 1)) % a.capacity + a.capacity) % a.capacity;
+    const int rq = r0 + 4 * lane;                 // this lane's four ranks
+    const bool word_ok = (rq + 3 < a.R) && ((a.R & 3) == 0);
+    uint32_t acc[8];
+#pragma unroll
+    for (int m = 0; m < 8; ++m) acc[m] = 0;
+    uint32_t sums[4][8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int m = 0; m < 8; ++m) sums[q][m] = 0;
+    int pending = 0;
+    for (int j = w; j < a.n; j += kFastWarps) {
+        int slot = first + j;
+        if (slot >= a.capacity) slot -= a.capacity;
+        const uint8_t *rowp = mask_base + (size_t)slot * a.R;
+        uint32_t word = 0;
+        if (word_ok) {
+            word = *reinterpret_cast<const uint32_t *>(rowp + rq);
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (rq + q < a.R) word |= (uint32_t)rowp[rq + q] << (8 * q);
+        }
+#pragma unroll
+        for (int m = 0; m < 8; ++m) acc[m] += (word >> m) & 0x01010101u;
+        if (++pending == 255) {   // byte lanes are about to overflow: spill into the wide sums
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int m = 0; m < 8; ++m) sums[q][m] += (acc[m] >> (8 * q)) & 255u;
+#pragma unroll
+            for (int m = 0; m < 8; ++m) acc[m] = 0;
+            pending = 0;
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int m = 0; m < 8; ++m) sums[q][m] += (acc[m] >> (8 * q)) & 255u;
+    // the eight warps' partial counts meet in shared memory
+    __shared__ uint32_t s_cnt[kFastRanks][8];
+    for (int i = tid; i < kFastRanks * 8; i += blockDim.x) (&s_cnt[0][0])[i] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int m = 0; m < 8; ++m)
+            if (sums[q][m]) atomicAdd(&s_cnt[4 * lane + q][m], sums[q][m]);
+    __syncthreads();
+    if (tid >= kFastRanks) return;
+    const int r = r0 + tid;
+    if (r >= a.R) return;
+    uint32_t mask = 0;
+    const float *wv = a.wmed + (size_t)r * M;
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+        if (m < M) {
+            const int cnt = (int)s_cnt[tid][m];
+            float dev = __fsub_rn(wv[m], s_B[m]);
+            if (p.dir[m] < 0) dev = -dev;
+            if (dev > s_rhs[m] && cnt >= p.k) mask |= 1u << m;
+            if (a.counts) a.counts[(size_t)r * M + m] = (uint16_t)cnt;
+            if (a.scores) a.scores[(size_t)r * M + m] = (dev == 0.0f) ? 0.0f : __fdiv_rn(__fmul_rn(0.6745f, dev), s_Ds[m]);
+        }
+    }
+    const int need = min(p.min_signals, M);
+    const bool cand = ((mask >> p.primary) & 1u) && (__popc(mask) >= need);
+    int c = a.consec[r];
+    c = cand ? min(c + 1, 255) : 0;
+    a.consec[r] = (uint8_t)c;
+    const bool flag = cand && (c >= p.n_consec);
+    const int pm = p.primary;
+    float devp = __fsub_rn(wv[pm], s_B[pm]);
+    if (p.dir[pm] < 0) devp = -devp;
+    const float absB = fabsf(s_B[pm]);
+    int t = 0;
+    if (flag && devp >= __fmul_rn(p.tier_severe, absB)) t = 3;
+    else if (flag && devp >= __fmul_rn(p.tier_moderate, absB)) t = 2;
+    else if (mask != 0) t = 1;
+    if (a.metric_mask) a.metric_mask[r] = mask;
+    if (a.flags) a.flags[r] = (uint8_t)flag;
+    if (a.tier) a.tier[r] = (uint8_t)t;
+}
+
 }  // namespace
 
 cudaError_t launch_score_flag(const ScoreArgs &a, const MetricParams &p, cudaStream_t st) {
     const int grid = (a.R + kScoreThreads - 1) / kScoreThreads;
     if (a.mask_bytes == 1)
-        score_flag_kernel<uint8_t, 8><<<grid, kScoreThreads, 0, st>>>(a, p);
+        score_flag_bytes_kernel<<<(a.R + kFastRanks - 1) / kFastRanks, kFastWarps * 32, 0, st>>>(a, p);
     else
         score_flag_kernel<uint32_t, 32><<<grid, kScoreThreads, 0, st>>>(a, p);
     return cudaGetLastError();

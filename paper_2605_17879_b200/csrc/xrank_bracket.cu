@@ -25,9 +25,8 @@
 //
 // No CTA ever waits for another: cross-CTA combination uses atomic counters, and the kernel
 // boundary orders the phases.
-#include <math_constants.h>
-
 #include "kernels.h"
+#include "xrank_common.cuh"
 
 namespace guard {
 
@@ -40,44 +39,9 @@ constexpr int kCtaAmb = 512;         // deferred exceedance decisions staged per
 constexpr int kSelThreads = 256;
 constexpr int kSelBins = 2048;
 
-__device__ __forceinline__ float fdown(float x) { return __uint_as_float(f2key(x) == 0 ? __float_as_uint(x) : bits_of_key(f2key(x) - 1)); }
-__device__ __forceinline__ float fup(float x) { return __uint_as_float(bits_of_key(f2key(x) + 1)); }
-
 // ---------------------------------------------------------------------------------------
 // 1. sample kernel: one warp per metric sorts 32 * EPL sampled keys in registers
 // ---------------------------------------------------------------------------------------
-template <int EPL>
-__device__ __forceinline__ void warp_bitonic_sort(uint32_t (&v)[EPL], const int lane) {
-    constexpr int N = 32 * EPL;
-#pragma unroll
-    for (int size = 2; size <= N; size <<= 1) {
-#pragma unroll
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            if (stride >= EPL) {   // partner element lives in lane ^ (stride / EPL), same register
-                const int lm = stride / EPL;
-                const bool upper = (lane & lm) != 0;
-#pragma unroll
-                for (int j = 0; j < EPL; ++j) {
-                    const bool asc = (((lane * EPL + j) & size) == 0);
-                    const uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, v[j], lm);
-                    v[j] = (asc != upper) ? min(v[j], o) : max(v[j], o);
-                }
-            } else {               // both elements in this lane
-#pragma unroll
-                for (int j = 0; j < EPL; ++j) {
-                    if ((j & stride) == 0) {
-                        const bool asc = (((lane * EPL + j) & size) == 0);
-                        const uint32_t x = v[j], y = v[j | stride];
-                        const uint32_t mn = min(x, y), mx = max(x, y);
-                        v[j] = asc ? mn : mx;
-                        v[j | stride] = asc ? mx : mn;
-                    }
-                }
-            }
-        }
-    }
-}
-
 template <int EPL>
 __global__ void __launch_bounds__(1024) xrank_sample_kernel(const XrankArgs a, const XrankScratch sc, const int delta) {
     constexpr int s = 32 * EPL;
@@ -137,28 +101,6 @@ __global__ void __launch_bounds__(1024) xrank_sample_kernel(const XrankArgs a, c
 // ---------------------------------------------------------------------------------------
 // 2./4. streaming kernels
 // ---------------------------------------------------------------------------------------
-// Exclusive scan of `n` over the lanes of a warp that share the same quad index
-// (lanes q, q + NQ, q + 2 NQ, ...); returns the exclusive prefix and the group total.
-template <int NQ>
-__device__ __forceinline__ void group_scan(int n, int &excl, int &total) {
-    const int lane = lane_id();
-    int incl = n;
-#pragma unroll
-    for (int d = NQ; d < 32; d <<= 1) {
-        const int u = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-        if (lane >= d) incl += u;
-    }
-    excl = incl - n;
-    total = __shfl_sync(0xFFFFFFFFu, incl, 32 - NQ + (lane & (NQ - 1)));
-}
-
-template <int NQ>
-__device__ __forceinline__ int group_sum(int v) {
-#pragma unroll
-    for (int d = NQ; d < 32; d <<= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
-    return v;
-}
-
 // MODE 0: median sweep.  MODE 1: MAD + exceedance sweep.
 template <int NQ, int MODE, typename MaskT>
 __global__ void __launch_bounds__(kBrThreads) xrank_stream_kernel(const XrankArgs a, const MetricParams p,
