@@ -125,6 +125,11 @@ struct guard_ctx {
     int mask_bytes() const { return M <= 8 ? 1 : 4; }
     // Cross-rank statistics of S rows: the bracketed path where it applies, else the direct one.
     cudaError_t xrank(XrankArgs a, int S, cudaStream_t st) {
+        // a few rows at a time: one CTA per column keeps the whole GPU busy
+        if (xrank_column_supported(R) && (long long)S * M <= 64 && !a.cut) {
+            launches += 1;
+            return launch_xrank_column(a, p, S, st);
+        }
         if (L.xr_fused) {
             a.fallbacks = status() + 1;
             launches += 1;
@@ -382,7 +387,7 @@ int guard_sweep_qualify(const float *d_S, int nodes, int gpus_per_node, int reps
     x.mad_user = d_fleet_mad;
     for (int m = 0; m < metrics; ++m) x.cut_rank[m] = p.dir[m] < 0 ? (int)(j - 1) : (int)(G - j);
     x.status = d_status;
-    e = launch_xrank_direct(x, p, 1, st);
+    e = xrank_column_supported(G) ? launch_xrank_column(x, p, 1, st) : launch_xrank_direct(x, p, 1, st);
     if (e != cudaSuccess) { set_error(g_error, "sweep fleet statistics launch: %s", cudaGetErrorString(e)); return GUARD_ERR_CUDA; }
     if (d_fleet_cut) {
         e = cudaMemcpyAsync(d_fleet_cut, fleet + 2 * kMaxMetrics, metrics * sizeof(float), cudaMemcpyDeviceToDevice, st);

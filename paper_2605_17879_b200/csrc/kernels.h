@@ -41,6 +41,9 @@ struct XrankScratch {
     int cap, amb_cap, S_max;
 };
 enum { kWhyCtaList = 0, kWhyStepList = 1, kWhyAmbList = 2, kWhyMedianMiss = 3, kWhySelect = 4, kWhyMadMiss = 5 };
+// One CTA per (row, metric) column with the column in registers: for a few rows at a time.
+bool xrank_column_supported(int R);
+cudaError_t launch_xrank_column(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st);
 bool xrank_fused_supported(int R, int M);
 cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, cudaStream_t st);
 bool xrank_bracket_supported(int R, int M);

@@ -1,10 +1,12 @@
-// Top-k slowest ranks, block then grid: every CTA keeps the best entries of its slice of
-// ranks with a shared-memory bitonic network, writes its K best to scratch, and the CTA
-// that takes the last ticket merges the per-CTA lists.  No CTA ever waits for another.
+// Top-k slowest ranks, block then grid: every CTA finds the K best entries of its slice of
+// ranks (K-th largest key by histogram refinement in registers, then a small shared-memory
+// bitonic sort of the entries at or above it), writes them to scratch, and the CTA that takes
+// the last ticket folds the per-CTA lists the same way.  No CTA ever waits for another.
 #include <cstdio>
 #include <mutex>
 
 #include "../../include/guard_b200.h"
+#include "colreg.cuh"
 #include "kernels.h"
 
 namespace guard {
@@ -12,15 +14,15 @@ namespace guard {
 namespace {
 
 constexpr int kTopThreads = 1024;
-constexpr int kTopChunk = 2048;  // entries merged into the running list at a time
+constexpr int kTopChunk = 1024;                 // ranks folded into the running list at a time
+constexpr int kTopList = kTopChunk + 1024;      // a chunk plus the running list
 
-// Sorts buf[0 .. 2 * kTopChunk) in descending order (all threads of the CTA).
-__device__ void bitonic_desc(unsigned long long *buf) {
-    constexpr int N = 2 * kTopChunk;
-    for (int size = 2; size <= N; size <<= 1) {
+// Sorts buf[0 .. n2) in descending order (n2 a power of two; all threads of the CTA).
+__device__ void bitonic_desc(unsigned long long *buf, int n2) {
+    for (int size = 2; size <= n2; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
             __syncthreads();
-            for (int t = threadIdx.x; t < N / 2; t += blockDim.x) {
+            for (int t = threadIdx.x; t < n2 / 2; t += blockDim.x) {
                 const int i = 2 * t - (t & (stride - 1));
                 const int j = i + stride;
                 const bool desc = ((i & size) == 0);
@@ -35,31 +37,76 @@ __device__ void bitonic_desc(unsigned long long *buf) {
     __syncthreads();
 }
 
+// Folds up to two entries per thread (64-bit composites: key of the value in the high
+// word, ~rank in the low word; 0 = no entry) into the K best, left sorted in run[0..K).
+// The K-th largest key is found by histogram refinement in registers; only the entries at
+// or above it (K of them, plus ties) are sorted.
+__device__ void fold_topk(const unsigned long long (&e)[2], int K, unsigned long long *list, unsigned long long *run,
+                          ColShared &sh, uint32_t *s_n) {
+    const int tid = threadIdx.x;
+    uint32_t key[2];
+    uint32_t valid = 0;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        key[i] = (uint32_t)(e[i] >> 32);
+        if (e[i] != 0ull) valid |= 1u << i;
+    }
+    if (tid == 0) *s_n = 0;
+    __syncthreads();
+    const uint32_t mine = __popc(valid);
+    const uint32_t wsum = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if (lane_id() == 0 && wsum) atomicAdd(s_n, wsum);
+    __syncthreads();
+    const uint32_t n = *s_n;
+    __syncthreads();
+    uint32_t thr = 0, dummy;
+    if (n > (uint32_t)K) {
+        if (!col_select_regs<2>(key, valid, n - (uint32_t)K, false, sh, thr, dummy)) thr = 0;
+    }
+    if (tid == 0) *s_n = 0;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+        if (((valid >> i) & 1u) && key[i] >= thr) list[atomicAdd(s_n, 1u)] = e[i];
+    __syncthreads();
+    const int cnt = (int)*s_n;
+    int n2 = 2;
+    while (n2 < cnt) n2 <<= 1;
+    for (int i = cnt + tid; i < n2; i += blockDim.x) list[i] = 0ull;
+    bitonic_desc(list, n2);
+    for (int i = tid; i < K; i += blockDim.x) run[i] = i < cnt ? list[i] : 0ull;
+    __syncthreads();
+}
+
 __global__ void __launch_bounds__(kTopThreads) topk_kernel(const TopkArgs a, const MetricParams p, const int nblocks) {
-    __shared__ unsigned long long buf[2 * kTopChunk];
+    __shared__ unsigned long long list[kTopList];
+    __shared__ unsigned long long run[GUARD_MAX_TOPK];
+    __shared__ ColShared sh;
+    __shared__ uint32_t s_n;
     __shared__ int is_last;
     const int tid = threadIdx.x, b = blockIdx.x;
     const int pm = p.primary, dirp = p.dir[pm];
     const int per = (a.R + nblocks - 1) / nblocks;
     const int lo = b * per, hi = min(a.R, lo + per);
+    const int K = a.K;
 
-    for (int i = tid; i < kTopChunk; i += blockDim.x) buf[i] = 0ull;
-    for (int c0 = lo; c0 < hi; c0 += kTopChunk) {
-        for (int i = tid; i < kTopChunk; i += blockDim.x) {
-            const int r = c0 + i;
-            unsigned long long e = 0ull;
-            if (r < hi) {
-                float v = a.wmed[(size_t)r * a.M + pm];
-                if (dirp < 0) v = -v;
-                e = ((unsigned long long)f2key(v) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)r);
-            }
-            buf[kTopChunk + i] = e;
-        }
-        bitonic_desc(buf);
-    }
+    for (int i = tid; i < K; i += blockDim.x) run[i] = 0ull;
     __syncthreads();
+    for (int c0 = lo; c0 < hi; c0 += kTopChunk) {
+        unsigned long long e[2];
+        const int r = c0 + tid;
+        e[0] = 0ull;
+        if (r < hi) {
+            float v = a.wmed[(size_t)r * a.M + pm];
+            if (dirp < 0) v = -v;
+            e[0] = ((unsigned long long)f2key(v) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)r);
+        }
+        e[1] = tid < K ? run[tid] : 0ull;
+        __syncthreads();
+        fold_topk(e, K, list, run, sh, &s_n);
+    }
     if (nblocks > 1) {
-        for (int i = tid; i < a.K; i += blockDim.x) a.cand[(size_t)b * a.K + i] = buf[i];
+        for (int i = tid; i < K; i += blockDim.x) a.cand[(size_t)b * K + i] = run[i];
         __threadfence();
         __syncthreads();
         if (tid == 0) {
@@ -70,19 +117,22 @@ __global__ void __launch_bounds__(kTopThreads) topk_kernel(const TopkArgs a, con
         __syncthreads();
         if (!is_last) return;
         __threadfence();
-        const int total = nblocks * a.K;
-        for (int i = tid; i < kTopChunk; i += blockDim.x) buf[i] = 0ull;
-        for (int c0 = 0; c0 < total; c0 += kTopChunk) {
-            for (int i = tid; i < kTopChunk; i += blockDim.x)
-                buf[kTopChunk + i] = (c0 + i < total) ? a.cand[c0 + i] : 0ull;
-            bitonic_desc(buf);
-        }
+        const int total = nblocks * K;
+        for (int i = tid; i < K; i += blockDim.x) run[i] = 0ull;
         __syncthreads();
+        for (int c0 = 0; c0 < total; c0 += kTopChunk) {
+            unsigned long long e[2];
+            const int j = c0 + tid;
+            e[0] = j < total ? __ldcg(a.cand + j) : 0ull;
+            e[1] = tid < K ? run[tid] : 0ull;
+            __syncthreads();
+            fold_topk(e, K, list, run, sh, &s_n);
+        }
     }
     const float B = a.fleet_med[pm];
     const float Ds = scale_of(a.fleet_mad[pm], B, p.floor_rel[pm], p.floor_abs[pm]);
-    for (int i = tid; i < a.K; i += blockDim.x) {
-        const int r = (int)(0xFFFFFFFFu - (uint32_t)(buf[i] & 0xFFFFFFFFull));
+    for (int i = tid; i < K; i += blockDim.x) {
+        const int r = (int)(0xFFFFFFFFu - (uint32_t)(run[i] & 0xFFFFFFFFull));
         if (a.idx) a.idx[i] = r;
         if (a.score) {
             float dev = __fsub_rn(a.wmed[(size_t)r * a.M + pm], B);

@@ -1,0 +1,132 @@
+// Cross-rank selection, column path: one CTA of 1024 threads per (row, metric) column, the
+// whole column held in registers (up to 32 values per thread, i.e. up to 32 768 ranks).
+// Used when only a few rows are processed at a time -- the fleet baseline of an evaluation,
+// single-step streaming ingest, the node sweep's fleet statistics -- where one CTA per row
+// would leave the GPU idle and a sampled interval is not worth its set-up.
+//
+// The wanted order statistic is found exactly by histogram refinement on order-preserving
+// keys: a 2048-bin shared-memory histogram over [min key, max key] locates the bin of the
+// wanted rank, the bin becomes the new range, until a bin is a single key (three rounds for
+// typical telemetry).  The MAD repeats this on |x - med|, and the exceedance bits are OR-ed
+// into the (pre-zeroed) mask row, four ranks per 32-bit atomic.
+#include "colreg.cuh"
+#include "kernels.h"
+
+namespace guard {
+
+namespace {
+
+template <int VPT, typename MaskT>
+__global__ void __launch_bounds__(kColThreads) xrank_column_kernel(const XrankArgs a, const MetricParams p) {
+    __shared__ ColShared sh;
+    const int m = blockIdx.x, t = blockIdx.y, tid = threadIdx.x, lane = lane_id();
+    const int R = a.R, M = a.M;
+    const int slot = (int)(((long long)a.first_slot + t) % a.capacity);
+    const float *row = a.base + (size_t)slot * a.row_stride;
+    const size_t col = (size_t)t * M + m;
+    const bool even = (R & 1) == 0;
+    const uint32_t k1 = (uint32_t)((R - 1) / 2);
+
+    float x[VPT];
+    uint32_t key[VPT];
+    uint32_t valid = 0;
+    bool bad = false;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int r = i * kColThreads + tid;
+        x[i] = 0.0f;
+        if (r < R) {
+            x[i] = __ldg(row + (size_t)r * M + m);
+            valid |= 1u << i;
+            bad |= nonfinite_bits(__float_as_uint(x[i]));
+        }
+        key[i] = f2key(x[i]);
+    }
+    if (a.check_finite && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(a.status, kStatNonFinite);
+
+    uint32_t v1, v2;
+    bool ok = col_select_regs<VPT>(key, valid, k1, even, sh, v1, v2);
+    const float med = median_from_keys(v1, v2, even);
+    if (a.cut) {
+        uint32_t c1, c2;
+        ok = col_select_regs<VPT>(key, valid, (uint32_t)a.cut_rank[m], false, sh, c1, c2) && ok;
+        if (tid == 0) a.cut[col] = key2f(c1);
+    }
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) key[i] = f2key(fabsf(__fsub_rn(x[i], med)));
+    ok = col_select_regs<VPT>(key, valid, k1, even, sh, v1, v2) && ok;
+    const float mad = median_from_keys(v1, v2, even);
+    if (tid == 0) {
+        if (!ok) atomicOr(a.status, kStatInternal);
+        a.med[col] = med;
+        a.mad[col] = mad;
+        if (a.med_user) a.med_user[col] = med;
+        if (a.mad_user) a.mad_user[col] = mad;
+    }
+    if (a.mask_base) {
+        // the mask row was zeroed before the launch; the M column CTAs of a row OR their bits in
+        const float rhs = __fmul_rn(p.thrp[m], scale_of(mad, med, p.floor_rel[m], p.floor_abs[m]));
+        const int dir = p.dir[m];
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int r = i * kColThreads + tid;
+            const uint32_t e = (((valid >> i) & 1u) && exceeds(x[i], med, dir, rhs)) ? 1u : 0u;
+            if (sizeof(MaskT) == 1) {
+                // four adjacent ranks share a 32-bit word: combine their bits, one atomic per word
+                uint32_t b = (e << m) << (8 * (tid & 3));
+                b |= __shfl_xor_sync(0xFFFFFFFFu, b, 1);
+                b |= __shfl_xor_sync(0xFFFFFFFFu, b, 2);
+                if ((tid & 3) == 0 && b) {
+                    const size_t idx = (size_t)slot * R + (size_t)r;   // r is a multiple of 4 here
+                    if ((R & 3) == 0) {
+                        atomicOr(reinterpret_cast<unsigned int *>(reinterpret_cast<uintptr_t>(a.mask_base) + idx), b);
+                    } else {   // rows are not word aligned: fall back to one atomic per byte position
+                        for (int qd = 0; qd < 4; ++qd) {
+                            const uint32_t byte = (b >> (8 * qd)) & 255u;
+                            if (byte) {
+                                const size_t bi = idx + qd;
+                                unsigned int *w = reinterpret_cast<unsigned int *>(reinterpret_cast<uintptr_t>(a.mask_base) + (bi & ~(size_t)3));
+                                atomicOr(w, byte << (8 * (bi & 3)));
+                            }
+                        }
+                    }
+                }
+            } else if (e) {
+                atomicOr(reinterpret_cast<unsigned int *>(a.mask_base) + (size_t)slot * R + r, 1u << m);
+            }
+        }
+    }
+}
+
+template <int VPT>
+cudaError_t launch_vpt(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st) {
+    const dim3 grid(a.M, S);
+    if (a.mask_bytes == 4) xrank_column_kernel<VPT, uint32_t><<<grid, kColThreads, 0, st>>>(a, p);
+    else xrank_column_kernel<VPT, uint8_t><<<grid, kColThreads, 0, st>>>(a, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool xrank_column_supported(int R) { return R >= 1024 && R <= 32 * kColThreads; }
+
+// Zeroes the exceedance rows of the S steps (at most two memsets when the span wraps), then
+// runs one CTA per column.
+cudaError_t launch_xrank_column(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st) {
+    if (S <= 0) return cudaSuccess;
+    if (a.mask_base) {
+        const size_t rowb = (size_t)a.R * a.mask_bytes;
+        const int first = a.first_slot % a.capacity;
+        const int n1 = (first + S <= a.capacity) ? S : (a.capacity - first);
+        cudaError_t e = cudaMemsetAsync((char *)a.mask_base + (size_t)first * rowb, 0, (size_t)n1 * rowb, st);
+        if (e == cudaSuccess && n1 < S) e = cudaMemsetAsync(a.mask_base, 0, (size_t)(S - n1) * rowb, st);
+        if (e != cudaSuccess) return e;
+    }
+    const int vpt = (a.R + kColThreads - 1) / kColThreads;
+    if (vpt <= 4) return launch_vpt<4>(a, p, S, st);
+    if (vpt <= 8) return launch_vpt<8>(a, p, S, st);
+    if (vpt <= 16) return launch_vpt<16>(a, p, S, st);
+    return launch_vpt<32>(a, p, S, st);
+}
+
+}  // namespace guard
