@@ -35,7 +35,8 @@ Layout make_layout(int R, int M, int C, int K) {
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
-    L.xr_big = off;    off = align_up(off + (L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps) : 0));
+    L.xr_big = off;    off = align_up(off + (L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps)
+                                                      : (L.xr_fused ? (size_t)kFusedMaxSteps * M * 8 * sizeof(uint32_t) : 0)));
     L.mask = off;      off = align_up(off + (size_t)C * R * (M <= 8 ? 1 : 4));
     L.ring = off;      off = align_up(off + (size_t)C * R * M * sizeof(float));
     L.total = off;
@@ -132,8 +133,20 @@ struct guard_ctx {
         }
         if (L.xr_fused) {
             a.fallbacks = status() + 1;
-            launches += 1;
-            return launch_xrank_fused(a, p, S, status() + 2, st);
+            const int first = a.first_slot;
+            for (int s0 = 0; s0 < S; s0 += kFusedMaxSteps) {
+                const int n = (S - s0 < kFusedMaxSteps) ? (S - s0) : kFusedMaxSteps;
+                XrankArgs g = a;
+                g.first_slot = (int)(((long long)first + s0) % a.capacity);
+                g.med = a.med + (size_t)s0 * M;
+                g.mad = a.mad + (size_t)s0 * M;
+                if (a.med_user) g.med_user = a.med_user + (size_t)s0 * M;
+                if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
+                cudaError_t e = launch_xrank_fused(g, p, n, status() + 2, (uint32_t *)(ws + L.xr_big), st);
+                if (e != cudaSuccess) return e;
+                launches += 2;
+            }
+            return cudaSuccess;
         }
         if (L.xr_steps == 0) { launches += 1; return launch_xrank_direct(a, p, S, st); }
         XrankScratch sc = carve_xrank_scratch(ws + L.xr_small, ws + L.xr_big, R, M, L.xr_steps);

@@ -45,7 +45,10 @@ enum { kWhyCtaList = 0, kWhyStepList = 1, kWhyAmbList = 2, kWhyMedianMiss = 3, k
 bool xrank_column_supported(int R);
 cudaError_t launch_xrank_column(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st);
 bool xrank_fused_supported(int R, int M);
-cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, cudaStream_t st);
+// qscratch: S * M * 8 words.
+cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, uint32_t *qscratch,
+                               cudaStream_t st);
+constexpr int kFusedMaxSteps = 1024;   // steps per launch of the fused path (sizes its scratch)
 bool xrank_bracket_supported(int R, int M);
 int xrank_scratch_steps(int R, int M, int want);
 size_t xrank_scratch_small_bytes(int M, int S_max);   // must be zero before first use

@@ -12,12 +12,29 @@ __device__ __forceinline__ float fup(float x) { return __uint_as_float(bits_of_k
 
 // Ascending bitonic sort of 32 * EPL keys held EPL per lane (element e lives in lane e / EPL,
 // register e % EPL): small strides are register-to-register, large ones go over shuffles.
+// The stage loops are kept rolled (only the per-register loop is unrolled): the network runs
+// once per CTA, and fully unrolled it is tens of kilobytes of straight-line code whose
+// instruction-cache misses cost more than the sort itself.
+template <int EPL, int STRIDE>
+__device__ __forceinline__ void bitonic_in_lane(uint32_t (&v)[EPL], const int lane, const int size) {
+#pragma unroll
+    for (int j = 0; j < EPL; ++j) {
+        if ((j & STRIDE) == 0) {
+            const bool asc = (((lane * EPL + j) & size) == 0);
+            const uint32_t x = v[j], y = v[j | STRIDE];
+            const uint32_t mn = min(x, y), mx = max(x, y);
+            v[j] = asc ? mn : mx;
+            v[j | STRIDE] = asc ? mx : mn;
+        }
+    }
+}
+
 template <int EPL>
 __device__ __forceinline__ void warp_bitonic_sort(uint32_t (&v)[EPL], const int lane) {
     constexpr int N = 32 * EPL;
-#pragma unroll
+#pragma unroll 1
     for (int size = 2; size <= N; size <<= 1) {
-#pragma unroll
+#pragma unroll 1
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
             if (stride >= EPL) {   // partner element lives in lane ^ (stride / EPL), same register
                 const int lm = stride / EPL;
@@ -29,15 +46,13 @@ __device__ __forceinline__ void warp_bitonic_sort(uint32_t (&v)[EPL], const int 
                     v[j] = (asc != upper) ? min(v[j], o) : max(v[j], o);
                 }
             } else {               // both elements in this lane
-#pragma unroll
-                for (int j = 0; j < EPL; ++j) {
-                    if ((j & stride) == 0) {
-                        const bool asc = (((lane * EPL + j) & size) == 0);
-                        const uint32_t x = v[j], y = v[j | stride];
-                        const uint32_t mn = min(x, y), mx = max(x, y);
-                        v[j] = asc ? mn : mx;
-                        v[j | stride] = asc ? mx : mn;
-                    }
+                switch (stride) {
+                    case 1: bitonic_in_lane<EPL, 1>(v, lane, size); break;
+                    case 2: if (EPL > 2) bitonic_in_lane<EPL, (EPL > 2 ? 2 : 1)>(v, lane, size); break;
+                    case 4: if (EPL > 4) bitonic_in_lane<EPL, (EPL > 4 ? 4 : 1)>(v, lane, size); break;
+                    case 8: if (EPL > 8) bitonic_in_lane<EPL, (EPL > 8 ? 8 : 1)>(v, lane, size); break;
+                    case 16: if (EPL > 16) bitonic_in_lane<EPL, (EPL > 16 ? 16 : 1)>(v, lane, size); break;
+                    default: break;
                 }
             }
         }

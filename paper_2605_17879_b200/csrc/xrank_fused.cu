@@ -1,10 +1,12 @@
-// Cross-rank selection, fused path: ONE launch, one CTA of 1024 threads per step, for
+// Cross-rank selection, fused path: a sample kernel plus ONE main launch, one CTA of 1024
+// threads per step, for
 // fleets whose candidate lists fit in shared memory (4 or 8 metrics, up to ~20 000 ranks
 // with 8 metrics).  The step's row is streamed twice (the second time it comes out of L2):
 //
-//   0. sample      two warps per metric sort 512 strided samples each in registers; seven
-//                  order statistics of the merged sample (middle +- delta, quartiles +- delta)
-//                  give the interval [lo, hi] of the median and [dlo, dhi] of the MAD;
+//   0. sample      (a small kernel of its own) two warps per metric sort 512 strided samples
+//                  each in registers; seven order statistics of the merged sample (middle +-
+//                  delta, quartiles +- delta) give the interval [lo, hi] of the median and
+//                  [dlo, dhi] of the MAD;
 //   1. sweep       every element is counted if below lo and kept (shared-memory list) if
 //                  inside [lo, hi];
 //   2. select      per metric, a group of threads checks the counts and finds the exact
@@ -125,9 +127,47 @@ __device__ bool group_select(const uint32_t *list, uint32_t n, uint32_t k, bool 
     return ok;
 }
 
+// Sample kernel of the fused path: one CTA per step, two warps per metric.  Each warp sorts
+// 512 strided samples of its column in registers; seven order statistics of the two merged
+// halves (middle, middle +- delta, quartiles +- delta_q) go to scratch as keys.  It is a
+// kernel of its own because the register sort wants more than the 64 registers a thread
+// gets inside the 1024-thread fused kernel.
+__global__ void __launch_bounds__(512) xrank_sample_q_kernel(const XrankArgs a, const int delta, const int delta_q,
+                                                             uint32_t *__restrict__ qout) {
+    __shared__ uint32_t samp[kMaxMetrics > 8 ? 8 * 1024 : 8 * 1024];
+    const int t = blockIdx.x, tid = threadIdx.x, lane = lane_id(), warp = warp_id();
+    const int R = a.R, M = a.M;
+    const int slot = (int)(((long long)a.first_slot + t) % a.capacity);
+    const float *row = a.base + (size_t)slot * a.row_stride;
+    if (warp < 2 * M) {
+        const int m = warp >> 1, h = warp & 1;
+        const int stride = R / kFuSample;
+        uint32_t v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int e = h * 512 + lane * 16 + j;
+            v[j] = f2key(__ldg(row + (size_t)(e * stride + (stride >> 1)) * M + m));
+        }
+        warp_bitonic_sort<16>(v, lane);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) samp[(m * 2 + h) * 512 + lane * 16 + j] = v[j];
+    }
+    __syncthreads();
+    if (tid < M * 8) {
+        const int m = tid >> 3, qq = tid & 7;
+        const int mid = kFuSample / 2, q1 = kFuSample / 4, q3 = 3 * kFuSample / 4;
+        int k = mid;
+        if (qq == 0) k = mid - delta; else if (qq == 2) k = mid + delta;
+        else if (qq == 3) k = q1 - delta_q; else if (qq == 4) k = q1 + delta_q;
+        else if (qq == 5) k = q3 - delta_q; else if (qq == 6) k = q3 + delta_q;
+        k = min(max(k, 0), kFuSample - 1);
+        qout[((size_t)t * M + m) * 8 + qq] = kth_of_two(samp + (m * 2) * 512, samp + (m * 2 + 1) * 512, 512, k);
+    }
+}
+
 template <int NQ, typename MaskT>
-__global__ void __launch_bounds__(kFuThreads, 1) xrank_fused_kernel(const XrankArgs a, const MetricParams p, const int delta,
-                                                                    const int delta_q, uint32_t *reasons) {
+__global__ void __launch_bounds__(kFuThreads, 1) xrank_fused_kernel(const XrankArgs a, const MetricParams p,
+                                                                    const uint32_t *__restrict__ qin, uint32_t *reasons) {
     constexpr int M = 4 * NQ, G = kFuThreads / M, CAP = kFuCandWords / M, LPI = kFuThreads / NQ;
     extern __shared__ __align__(16) uint32_t smem[];
     uint32_t *cand = smem;                   // [M][CAP]; holds the sorted samples [M][2][512] during phase 0
@@ -154,31 +194,8 @@ __global__ void __launch_bounds__(kFuThreads, 1) xrank_fused_kernel(const XrankA
     if (tid == 0) { s_namb = 0; s_fail = 0; }
     if (tid < M) s_shift[tid] = 0;
 
-    // ---- 0. sample -----------------------------------------------------------------------
-    if (warp < 2 * M) {
-        const int m = warp >> 1, h = warp & 1;
-        const int stride = R / kFuSample;
-        uint32_t v[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int e = h * 512 + lane * 16 + j;
-            v[j] = f2key(__ldg(row + (size_t)(e * stride + (stride >> 1)) * M + m));
-        }
-        warp_bitonic_sort<16>(v, lane);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) cand[(m * 2 + h) * 512 + lane * 16 + j] = v[j];
-    }
-    __syncthreads();
-    if (tid < M * 8) {
-        const int m = tid >> 3, qq = tid & 7;
-        const int mid = kFuSample / 2, q1 = kFuSample / 4, q3 = 3 * kFuSample / 4;
-        int k = mid;
-        if (qq == 0) k = mid - delta; else if (qq == 2) k = mid + delta;
-        else if (qq == 3) k = q1 - delta_q; else if (qq == 4) k = q1 + delta_q;
-        else if (qq == 5) k = q3 - delta_q; else if (qq == 6) k = q3 + delta_q;
-        k = min(max(k, 0), kFuSample - 1);
-        s_q[m][qq] = kth_of_two(cand + (m * 2) * 512, cand + (m * 2 + 1) * 512, 512, k);
-    }
+    // ---- 0. the sample kernel's order statistics -> intervals ---------------------------------
+    if (tid < M * 8) s_q[tid >> 3][tid & 7] = qin[so * 8 + tid];
     __syncthreads();
     if (tid < M) {
         const int m = tid;
@@ -461,7 +478,8 @@ bool xrank_fused_supported(int R, int M) {
     return frac * R * 1.15 <= (double)(kFuCandWords / M);
 }
 
-cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, cudaStream_t st) {
+cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, uint32_t *qscratch,
+                               cudaStream_t st) {
     if (S <= 0) return cudaSuccess;
     // half-widths in sample ranks: 5.5 standard deviations of the sampled median's rank; the
     // quartile intervals bracket a count, the sum of two quartile ranks (sd ~ 0.61 sqrt(s)), at
@@ -470,26 +488,28 @@ cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S,
     const int delta_q = (int)ceil(0.5 * 4.0 * 0.612 * sqrt((double)kFuSample));
     const size_t smem = (size_t)(kFuCandWords + a.M * kFuBins + kFuAmb) * sizeof(uint32_t);
     const bool wide = a.mask_bytes == 4;
-    cudaError_t e;
+    xrank_sample_q_kernel<<<S, 64 * a.M, 0, st>>>(a, delta, delta_q, qscratch);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
     if (a.M == 8) {
         if (wide) {
             e = cudaFuncSetAttribute(xrank_fused_kernel<2, uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            xrank_fused_kernel<2, uint32_t><<<S, kFuThreads, smem, st>>>(a, p, delta, delta_q, reasons);
+            xrank_fused_kernel<2, uint32_t><<<S, kFuThreads, smem, st>>>(a, p, qscratch, reasons);
         } else {
             e = cudaFuncSetAttribute(xrank_fused_kernel<2, uint8_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            xrank_fused_kernel<2, uint8_t><<<S, kFuThreads, smem, st>>>(a, p, delta, delta_q, reasons);
+            xrank_fused_kernel<2, uint8_t><<<S, kFuThreads, smem, st>>>(a, p, qscratch, reasons);
         }
     } else {
         if (wide) {
             e = cudaFuncSetAttribute(xrank_fused_kernel<1, uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            xrank_fused_kernel<1, uint32_t><<<S, kFuThreads, smem, st>>>(a, p, delta, delta_q, reasons);
+            xrank_fused_kernel<1, uint32_t><<<S, kFuThreads, smem, st>>>(a, p, qscratch, reasons);
         } else {
             e = cudaFuncSetAttribute(xrank_fused_kernel<1, uint8_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            xrank_fused_kernel<1, uint8_t><<<S, kFuThreads, smem, st>>>(a, p, delta, delta_q, reasons);
+            xrank_fused_kernel<1, uint8_t><<<S, kFuThreads, smem, st>>>(a, p, qscratch, reasons);
         }
     }
     return cudaGetLastError();
