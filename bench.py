@@ -35,6 +35,9 @@ if ROOT not in sys.path:
 METRIC = "rank-step-metric cells scored/s"
 UNIT = "cells/s"
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum of one xrank_fused_kernel launch on this workload, from the
+# ncu capture summarised under profiles/ (None once the kernel has changed since the capture)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
 FALLBACK_HBM_GBS = 6650.0   # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
 
 
@@ -119,6 +122,62 @@ def oracle_sample_rate(cfg, block_host, sample_steps):
     return x.size / dt, dt
 
 
+def run_streaming(dev, steps, warm):
+    """Streaming configuration: 32 768 ranks x 8 metrics, one step per ingest into a 512-step
+    ring, an evaluation after every step, flags and top-k read back to pinned host memory.
+    Returns per-step ingest-to-flag latency percentiles (host clock) and sustained cells/s."""
+    import torch
+    from paper_2605_17879_b200 import guard, synth
+    cfg = synth.paper_configs()["streaming"]
+    R, M = cfg.ranks, cfg.metrics
+    g = guard.Guard(R, M, cfg.W, cfg.k, dir=synth.fleet_dir(M), capacity=cfg.ring_capacity, topk=cfg.topk, device=dev)
+    pool = 256                                   # generated steps, produced outside the timed region
+    gen = synth.fleet_block(cfg, 0, pool, device=dev)
+    out = g.alloc_outputs()
+    h_flags = torch.empty(R, dtype=torch.uint8, pin_memory=True)
+    h_idx = torch.empty(cfg.topk, dtype=torch.int32, pin_memory=True)
+    lat = []
+
+    def one(t, timed):
+        slot = g.ring_reserve(1)
+        slot.copy_(gen[t % pool:t % pool + 1])    # the producer lands the step in its ring slot
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        g.ingest(slot)
+        g.score(out)
+        h_flags.copy_(out["flags"], non_blocking=True)
+        h_idx.copy_(out["topk_idx"], non_blocking=True)
+        torch.cuda.synchronize()
+        if timed:
+            lat.append(time.perf_counter() - t0)
+
+    for t in range(warm):
+        one(t, False)
+    for t in range(warm, warm + steps):
+        one(t, True)
+    # sustained: no host synchronisation between steps
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(steps):
+        slot = g.ring_reserve(1)
+        slot.copy_(gen[t % pool:t % pool + 1])
+        g.ingest(slot)
+        g.score(out)
+    e1.record()
+    torch.cuda.synchronize()
+    g.sync_status()
+    sustained = steps * R * M / (e0.elapsed_time(e1) / 1e3)
+    lat.sort()
+    pick = lambda q: lat[min(len(lat) - 1, int(q * len(lat)))] * 1e6
+    res = {"workload": "streaming: 32768 ranks x 8 metrics, ring 512, W=200 k=120 top-64, evaluation every step",
+           "steps": steps, "latency_us": {"p50": pick(0.50), "p99": pick(0.99), "max": lat[-1] * 1e6},
+           "sustained_cells_per_s": sustained, "us_per_step_sustained": e0.elapsed_time(e1) * 1e3 / steps,
+           "cells_per_step": R * M, "fallback_rows": g.fallback_steps()}
+    g.close()
+    return res
+
+
 def run_reference(args):
     """The reference arm: the oracle as it stands, on the host cores."""
     from paper_2605_17879_b200 import dist as gd, synth
@@ -162,6 +221,7 @@ def main():
     ap.add_argument("--impl", default="guard", choices=["guard", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--streaming-steps", type=int, default=500)
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -210,6 +270,7 @@ def main():
         one_pass()
     g.sync_status()
     sampler = ClockSampler(local_rank)
+    g.profile_enable(True)
     launches0 = g.kernel_launches
     gd.barrier()
     torch.cuda.synchronize()
@@ -222,6 +283,8 @@ def main():
     torch.cuda.synchronize()
     gd.barrier()
     clocks = sampler.stop()
+    kern_ms, kern_n = g.profile_read()
+    g.profile_enable(False)
     g.sync_status()
     launches = g.kernel_launches - launches0
     fallback_rows = g.fallback_steps()
@@ -229,18 +292,21 @@ def main():
     value, tmax = gd.aggregate_throughput(cells_per_step * args.steps, secs, device=dev)
     flagged = int(out["flags"].sum().item())
 
-    # roofline of the dominant kernel: the cross-rank selection behind guard_ingest.  One
-    # launch reads a block of 200 steps once (4 B per cell) and writes one exceedance byte
-    # per (step, rank) (1/8 B per cell).
+    # roofline of the dominant kernel: the fused cross-rank sweep behind guard_ingest, timed by
+    # the library with CUDA events recorded on the launching stream right around that kernel.
+    # One launch reads a block of 200 steps once from HBM (4 B per cell; its second sweep is
+    # served by L2) and writes one exceedance byte per (step, rank) (1/8 B per cell).
     ingest_ms = [a.elapsed_time(b) for a, b in ev_pairs]
-    launch_s = statistics.fmean(ingest_ms) / 1e3
+    launch_s = (kern_ms / kern_n / 1e3) if kern_n else statistics.fmean(ingest_ms) / 1e3
     algo_bytes = B * R * M * 4 + B * R * 1
     peak, peak_kind = measured_hbm_peak()
     achieved = algo_bytes / launch_s / 1e9
-    roofline = {"bound": "hbm", "kernel": "xrank (cross-rank median/MAD/exceedance, one launch per ingested block)",
+    roofline = {"bound": "hbm", "kernel": "xrank_fused_kernel (cross-rank median / MAD / exceedance of one ingested block)",
                 "achieved": achieved, "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_ms": launch_s * 1e3,
-                "share_of_step": sum(ingest_ms) / 1e3 / secs,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes_per_launch": algo_bytes,
+                "avg_launch_ms": launch_s * 1e3, "launches_timed": kern_n,
+                "ingest_call_ms": statistics.fmean(ingest_ms),
+                "share_of_step": (kern_ms / 1e3 / secs) if kern_n else None,
                 "path_algorithmic_GBps": (8.125 * cells_per_step * args.steps) / secs / 1e9,
                 "path_frac_of_peak": (8.125 * cells_per_step * args.steps) / secs / 1e9 / peak}
 
@@ -292,6 +358,13 @@ def main():
                         "sample": "ingest + one evaluation of the first %d steps at full width (%d ranks x %d metrics)"
                                   % (sample_steps, R, M)}
 
+    streaming = None
+    if rank == 0 and world == 1 and args.streaming_steps > 0:
+        del ring, out
+        g.close()
+        torch.cuda.empty_cache()
+        streaming = run_streaming(dev, args.streaming_steps, 50)
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
@@ -303,6 +376,7 @@ def main():
                        "l2": "inputs (10.49 GB) larger than L2", "parallelism": "replicas only",
                        "flagged_last_evaluation": flagged, "direct_path_fallback_rows_last_pass": fallback_rows},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+            "streaming": streaming,
         }
         print(json.dumps(line), flush=True)
     g.close()

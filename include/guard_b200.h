@@ -194,6 +194,15 @@ int guard_sync_status(guard_ctx *ctx, void *stream);
 /* Clears the ring position, exceedance ring, consecutive counters and status. */
 int guard_reset(guard_ctx *ctx, void *stream);
 
+/* Kernel timing for benchmarks: while enabled, guard_ingest records a pair of CUDA events on
+ * the stream right around its main kernel (the fused cross-rank sweep; contexts whose sizes
+ * take another path record nothing).  guard_profile_read waits for the recorded events, returns
+ * the sum of the kernel durations in milliseconds and their number, and forgets them.
+ * Disabling destroys any events not yet read.  Off by default; do not leave it on in a
+ * long-running service without reading (events accumulate in host memory). */
+int guard_profile_enable(guard_ctx *ctx, int on);
+int guard_profile_read(guard_ctx *ctx, double *total_ms, int64_t *launches);
+
 /* Steps ingested since creation or the last reset. */
 int64_t guard_steps_seen(const guard_ctx *ctx);
 

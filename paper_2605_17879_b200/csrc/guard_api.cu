@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "../../include/guard_b200.h"
 #include "kernels.h"
@@ -110,6 +111,8 @@ struct guard_ctx {
     char *ws;
     long long seen;
     long long launches;  // kernels enqueued by this context so far
+    bool profiling = false;                                   // record events around the main ingest kernel
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof;    // recorded, not yet read
     char error[256];
 
     uint32_t *status() const { return (uint32_t *)(ws + L.status); }
@@ -142,7 +145,8 @@ struct guard_ctx {
                 g.mad = a.mad + (size_t)s0 * M;
                 if (a.med_user) g.med_user = a.med_user + (size_t)s0 * M;
                 if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
-                cudaError_t e = launch_xrank_fused(g, p, n, status() + 2, (uint32_t *)(ws + L.xr_big), st);
+                cudaError_t e = launch_xrank_fused(g, p, n, status() + 2, (uint32_t *)(ws + L.xr_big), st,
+                                                   (profiling && a.mask_base) ? &prof : nullptr);
                 if (e != cudaSuccess) return e;
                 launches += 2;
             }
@@ -441,6 +445,34 @@ int guard_reset(guard_ctx *c, void *stream) {
     return GUARD_OK;
 }
 
+int guard_profile_enable(guard_ctx *c, int on) {
+    if (!c) return GUARD_ERR_ARG;
+    c->profiling = on != 0;
+    if (!on) {
+        for (auto &pr : c->prof) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
+        c->prof.clear();
+    }
+    return GUARD_OK;
+}
+
+int guard_profile_read(guard_ctx *c, double *total_ms, int64_t *launches) {
+    if (!c || !total_ms || !launches) return GUARD_ERR_ARG;
+    double sum = 0.0;
+    for (auto &pr : c->prof) {
+        cudaError_t e = cudaEventSynchronize(pr.second);
+        float ms = 0.0f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, pr.first, pr.second);
+        if (e != cudaSuccess) return c->cuda_fail(e, "guard_profile_read");
+        sum += ms;
+        cudaEventDestroy(pr.first);
+        cudaEventDestroy(pr.second);
+    }
+    *total_ms = sum;
+    *launches = (int64_t)c->prof.size();
+    c->prof.clear();
+    return GUARD_OK;
+}
+
 int64_t guard_steps_seen(const guard_ctx *c) { return c ? c->seen : 0; }
 
 int64_t guard_kernel_launches(const guard_ctx *c) { return c ? c->launches : 0; }
@@ -462,7 +494,10 @@ int64_t guard_fallback_steps(guard_ctx *c, void *stream) {
     return (int64_t)n;
 }
 
-void guard_destroy(guard_ctx *c) { delete c; }
+void guard_destroy(guard_ctx *c) {
+    if (c) guard_profile_enable(c, 0);
+    delete c;
+}
 
 const char *guard_last_error(const guard_ctx *c) { return c ? c->error : g_error; }
 

@@ -1,5 +1,8 @@
 // Host-side launchers of the scoring kernels (internal to the library).
 #pragma once
+#include <utility>
+#include <vector>
+
 #include "common.cuh"
 
 namespace guard {
@@ -46,8 +49,9 @@ bool xrank_column_supported(int R);
 cudaError_t launch_xrank_column(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st);
 bool xrank_fused_supported(int R, int M);
 // qscratch: S * M * 8 words.
+// prof: if not NULL, a pair of events recorded on st right around the main kernel is appended.
 cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, uint32_t *qscratch,
-                               cudaStream_t st);
+                               cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof = nullptr);
 constexpr int kFusedMaxSteps = 1024;   // steps per launch of the fused path (sizes its scratch)
 bool xrank_bracket_supported(int R, int M);
 int xrank_scratch_steps(int R, int M, int want);

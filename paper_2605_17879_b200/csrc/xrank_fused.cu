@@ -479,7 +479,7 @@ bool xrank_fused_supported(int R, int M) {
 }
 
 cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, uint32_t *qscratch,
-                               cudaStream_t st) {
+                               cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof) {
     if (S <= 0) return cudaSuccess;
     // half-widths in sample ranks: 5.5 standard deviations of the sampled median's rank; the
     // quartile intervals bracket a count, the sum of two quartile ranks (sd ~ 0.61 sqrt(s)), at
@@ -491,6 +491,11 @@ cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S,
     xrank_sample_q_kernel<<<S, 64 * a.M, 0, st>>>(a, delta, delta_q, qscratch);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if (prof) {
+        if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return cudaGetLastError();
+        cudaEventRecord(ev0, st);
+    }
     if (a.M == 8) {
         if (wide) {
             e = cudaFuncSetAttribute(xrank_fused_kernel<2, uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -512,7 +517,12 @@ cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S,
             xrank_fused_kernel<1, uint8_t><<<S, kFuThreads, smem, st>>>(a, p, qscratch, reasons);
         }
     }
-    return cudaGetLastError();
+    e = cudaGetLastError();
+    if (prof) {
+        cudaEventRecord(ev1, st);
+        prof->emplace_back(ev0, ev1);
+    }
+    return e;
 }
 
 }  // namespace guard

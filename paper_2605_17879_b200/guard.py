@@ -77,6 +77,10 @@ def lib():
         L.guard_fallback_steps.argtypes = [vp, vp]
         L.guard_fallback_reasons.restype = C.c_int
         L.guard_fallback_reasons.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        L.guard_profile_enable.restype = C.c_int
+        L.guard_profile_enable.argtypes = [vp, C.c_int]
+        L.guard_profile_read.restype = C.c_int
+        L.guard_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.guard_destroy.restype = None
         L.guard_destroy.argtypes = [vp]
         L.guard_last_error.restype = C.c_char_p
@@ -190,6 +194,15 @@ class Guard:
             self._check(lib().guard_fallback_reasons(self._h, out, _stream()))
         names = ("cta_list", "step_list", "deferred_list", "median_miss", "select", "mad_miss")
         return dict(zip(names, [int(v) for v in out]))
+
+    def profile_enable(self, on: bool = True) -> None:
+        self._check(lib().guard_profile_enable(self._h, 1 if on else 0))
+
+    def profile_read(self):
+        """(total milliseconds, launches) of the main ingest kernel since the last read."""
+        ms, n = C.c_double(), C.c_int64()
+        self._check(lib().guard_profile_read(self._h, C.byref(ms), C.byref(n)))
+        return ms.value, n.value
 
     def ring_reserve(self, steps: int) -> torch.Tensor:
         """View [steps, ranks, metrics] of the ring slots the next `steps` steps occupy."""
