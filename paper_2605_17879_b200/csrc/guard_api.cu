@@ -111,6 +111,7 @@ struct guard_ctx {
     char *ws;
     long long seen;
     long long launches;  // kernels enqueued by this context so far
+    long long evals;     // evaluations since creation / reset
     bool profiling = false;                                   // record events around the main ingest kernel
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof;    // recorded, not yet read
     char error[256];
@@ -208,7 +209,7 @@ int guard_create(guard_ctx **out, int ranks, int metrics, int W, int k, const gu
     guard_ctx *c = new (std::nothrow) guard_ctx();
     if (!c) { set_error(g_error, "out of host memory"); return GUARD_ERR_ARG; }
     c->R = ranks; c->M = metrics; c->W = W; c->k = k; c->C = capacity_steps; c->K = topk;
-    c->p = p; c->L = L; c->ws = (char *)d_workspace; c->seen = 0; c->launches = 0; c->error[0] = 0;
+    c->p = p; c->L = L; c->ws = (char *)d_workspace; c->seen = 0; c->launches = 0; c->evals = 0; c->error[0] = 0;
     // state: status word, ticket, fleet statistics, consecutive counters
     cudaError_t e = cudaMemsetAsync(c->ws, 0, L.wmed, (cudaStream_t)stream);
     if (e != cudaSuccess) {
@@ -287,6 +288,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     w.series = (int)row;
     w.wmed = c->wmed();
     w.wmed_user = d_wmed;
+    w.use_hint = c->evals > 0 ? 1 : 0;
     w.status = c->status();
     cudaError_t e = launch_window_select(w, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "window_select launch");
@@ -325,6 +327,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     s.tier = d_tier;
     e = launch_score_flag(s, c->p, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
+    c->evals += 1;
     c->launches += 2;
 
     if (c->K > 0 && (d_topk_idx || d_topk_score)) {
@@ -442,6 +445,7 @@ int guard_reset(guard_ctx *c, void *stream) {
     cudaError_t e = cudaMemsetAsync(c->ws, 0, c->L.wmed, (cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "cudaMemsetAsync");
     c->seen = 0;
+    c->evals = 0;
     return GUARD_OK;
 }
 

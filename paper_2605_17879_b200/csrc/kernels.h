@@ -72,6 +72,7 @@ struct WindowArgs {
     int n;                  // window length in steps
     int series;             // R * M
     float *wmed;            // [series] (never NULL)
+    int use_hint;           // wmed holds the previous evaluation's medians: use them as first pivots
     float *wmed_user;       // or NULL
     uint32_t *status;
 };

@@ -129,17 +129,22 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // Median of the n keys held by the warp (kv sorted ascending per lane, padded with
-// 0xFFFFFFFF; nreal real keys in this lane).  Returns false if the loop bound was hit.
+// 0xFFFFFFFF; nreal real keys in this lane).  `hint` (a key, or 0 for none) is a first pivot
+// guess -- the series' median at the previous evaluation -- and need not be one of the keys.
+// Returns false if a loop bound was hit.
 template <int VPL>
-__device__ __forceinline__ bool warp_median(const uint32_t (&kv)[VPL], const int nreal, const int n, float &med) {
+__device__ __forceinline__ bool warp_median(const uint32_t (&kv)[VPL], const int nreal, const int n, const uint32_t hint,
+                                            float &med) {
+    constexpr uint32_t kNone = 0xFFFFFFFFu, kStale = 0xFFFFFFFEu;   // neither is the key of a finite value
     const int lane = lane_id();
     const bool even = !(n & 1);
     const int kq = n >> 1;             // upper middle rank (the middle for odd n)
     int lo_i = 0, hi_i = nreal;        // this lane's active run [lo_i, hi_i)
-    uint32_t v1 = 0, v2 = 0;
-    // first pivot: median of the lanes' middle keys
-    const unsigned have = __ballot_sync(0xFFFFFFFFu, nreal > 0);
-    uint32_t p = warp_sorted_at(nreal > 0 ? lane_pick<VPL>(kv, nreal >> 1) : 0xFFFFFFFFu, __popc(have) >> 1);
+    uint32_t p = hint;
+    if (p == 0u) {                     // no guess: median of the lanes' middle keys
+        const unsigned have = __ballot_sync(0xFFFFFFFFu, nreal > 0);
+        p = warp_sorted_at(nreal > 0 ? lane_pick<VPL>(kv, nreal >> 1) : kNone, __popc(have) >> 1);
+    }
     for (int round = 0; round < 300; ++round) {
         int clt = 0, cle = 0;
 #pragma unroll
@@ -150,59 +155,77 @@ __device__ __forceinline__ bool warp_median(const uint32_t (&kv)[VPL], const int
         const uint32_t tot = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)clt | ((uint32_t)cle << 16));
         const int tlt = (int)(tot & 0xFFFFu), tle = (int)(tot >> 16);   // ranks [tlt, tle) hold p
         if (kq >= tlt && kq < tle) {
-            v2 = p;
-            v1 = p;
-            if (even && kq == tlt) {   // lower middle: the largest key below the pivot
+            uint32_t v1 = p;
+            if (even && kq == tlt)     // lower middle: the largest key below the pivot
                 v1 = __reduce_max_sync(0xFFFFFFFFu, clt > 0 ? lane_pick<VPL>(kv, clt - 1) : 0u);
-            }
-            med = median_from_keys(v1, v2, even);
+            med = median_from_keys(v1, p, even);
             return true;
         }
         if (kq >= tle) {
-            lo_i = cle;
+            lo_i = max(lo_i, cle);
             if (kq - tle < kWalkMax) {   // walk upwards: ranks tle, tle + 1, ...
-                int cur = tle, nxt = cle;
-                v1 = p;                  // rank kq - 1 if it is still inside the pivot's run
+                // rank kq - 1 when it is not reached by the walk: inside the pivot's run, or
+                // (pivot not a key) the largest key below the pivot
+                uint32_t v1 = p;
+                if (even && kq == tle && tle == tlt)
+                    v1 = __reduce_max_sync(0xFFFFFFFFu, clt > 0 ? lane_pick<VPL>(kv, clt - 1) : 0u);
+                int nxt = cle, cur = tle;
+                uint32_t offer = nxt < nreal ? lane_pick<VPL>(kv, nxt) : kNone;          // this lane's next key
+                uint32_t after = nxt + 1 < nreal ? lane_pick<VPL>(kv, nxt + 1) : kNone;  // and the one after
                 for (int step = 0; step <= kWalkMax; ++step) {
-                    const uint32_t prop = nxt < nreal ? lane_pick<VPL>(kv, nxt) : 0xFFFFFFFFu;
-                    const uint32_t m = __reduce_min_sync(0xFFFFFFFFu, prop);
-                    const bool is = (prop == m) && (nxt < nreal);
+                    const uint32_t m = __reduce_min_sync(0xFFFFFFFFu, offer);
+                    const bool is = (offer == m) && (m != kNone);
                     const int c = __popc(__ballot_sync(0xFFFFFFFFu, is));
+                    if (c == 0) return false;
                     if (kq - 1 >= cur && kq - 1 < cur + c) v1 = m;
                     if (kq < cur + c) {
                         med = even ? median_from_keys(v1, m, true) : key2f(m);
                         return true;
                     }
-                    nxt += is;
                     cur += c;
+                    if (is) { ++nxt; offer = after; after = kStale; }
+                    if (__any_sync(0xFFFFFFFFu, offer == kStale)) {   // a lane used both prefetched keys
+                        if (offer == kStale) {
+                            offer = nxt < nreal ? lane_pick<VPL>(kv, nxt) : kNone;
+                            after = nxt + 1 < nreal ? lane_pick<VPL>(kv, nxt + 1) : kNone;
+                        }
+                    }
                 }
                 return false;
             }
         } else {
-            hi_i = clt;
+            hi_i = min(hi_i, clt);
             if (tlt - kq <= kWalkMax) {  // walk downwards: ranks tlt - 1, tlt - 2, ...
-                int cur = tlt, nxt = clt;   // ranks [.., cur) are still below; this lane's next is kv[nxt - 1]
+                int nxt = clt, cur = tlt;   // this lane's next key is kv[nxt - 1]; ranks below cur are left
+                uint32_t v2 = 0;
+                uint32_t offer = nxt > 0 ? lane_pick<VPL>(kv, nxt - 1) : 0u;
+                uint32_t after = nxt > 1 ? lane_pick<VPL>(kv, nxt - 2) : 0u;
+                constexpr uint32_t kStaleLow = 1u;   // 0 and 1 are not keys of finite values either
                 for (int step = 0; step <= kWalkMax + 1; ++step) {
-                    const uint32_t prop = nxt > 0 ? lane_pick<VPL>(kv, nxt - 1) : 0u;
-                    const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, prop);
-                    const bool is = (prop == m) && (nxt > 0);
+                    const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, offer);
+                    const bool is = (offer == m) && (m != 0u);
                     const int c = __popc(__ballot_sync(0xFFFFFFFFu, is));
                     if (c == 0) return false;
                     // ranks [cur - c, cur) hold m
                     if (kq >= cur - c && kq < cur) v2 = m;
-                    if (kq - 1 >= cur - c) {     // rank kq - 1 (or, for odd n, rank kq) reached
-                        if (!even) { med = key2f(v2); return true; }
-                        med = median_from_keys(m, v2, true);
+                    if (kq - 1 >= cur - c || (!even && kq >= cur - c)) {
+                        med = even ? median_from_keys(m, v2, true) : key2f(v2);
                         return true;
                     }
-                    nxt -= is;
                     cur -= c;
+                    if (is) { --nxt; offer = after; after = kStaleLow; }
+                    if (__any_sync(0xFFFFFFFFu, offer == kStaleLow)) {
+                        if (offer == kStaleLow) {
+                            offer = nxt > 0 ? lane_pick<VPL>(kv, nxt - 1) : 0u;
+                            after = nxt > 1 ? lane_pick<VPL>(kv, nxt - 2) : 0u;
+                        }
+                    }
                 }
                 return false;
             }
         }
         // far off: next pivot is the middle key of the longest still-active run
-        const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, ((uint32_t)(hi_i - lo_i) << 5) | (uint32_t)lane);
+        const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, ((uint32_t)max(hi_i - lo_i, 0) << 5) | (uint32_t)lane);
         if ((best >> 5) == 0) return false;
         p = __shfl_sync(0xFFFFFFFFu, lane_pick<VPL>(kv, (lo_i + hi_i) >> 1), best & 31u);
     }
@@ -225,7 +248,9 @@ __global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a
         if (use_bulk) {
             if (tid == 0) mbar_arrive_expect_tx(&bar[b], (uint32_t)n * (uint32_t)ncols * 4u);
             __syncthreads();   // the expectation is registered before any copy can complete
-            for (int row = tid; row < n; row += 1024) {
+            // lane l of warp w issues rows w + 32 l, w + 32 l + 1024, ...: a warp's bulk copies are
+            // issued one lane after the other, so they are spread over all warps
+            for (int row = w + 32 * lane; row < n; row += 1024) {
                 int slot = first + row;
                 if (slot >= a.capacity) slot -= a.capacity;
                 bulk_g2s(buf + row * kWarpPitch, a.ring + (size_t)slot * a.row_stride + col0, (uint32_t)ncols * 4u, &bar[b]);
@@ -276,7 +301,8 @@ __global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a
             }
             lane_sort<VPL>(kv);
             float med = 0.0f;
-            const bool ok = warp_median<VPL>(kv, nreal, n, med);
+            const uint32_t hint = a.use_hint ? f2key(a.wmed[series]) : 0u;   // last evaluation's median
+            const bool ok = warp_median<VPL>(kv, nreal, n, hint, med);
             if (lane == 0) {
                 if (!ok) atomicOr(a.status, kStatInternal);
                 a.wmed[series] = med;
