@@ -18,9 +18,12 @@
  *     memory of its own: the caller hands it one workspace (guard_workspace_bytes) that
  *     holds the telemetry ring and all state, and must keep it alive and untouched until
  *     guard_destroy.
- *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it and no
- *     call synchronises, except guard_sync_status.  Calls on one context must be issued
- *     in order on streams that are ordered with respect to each other.
+ *   - `stream` is a cudaStream_t passed as void*.  All work is ordered on it and no call
+ *     synchronises, except guard_sync_status.  (guard_score may run the window medians on an
+ *     internal stream forked from and joined back into `stream` with events, so that they
+ *     overlap the preceding guard_ingest; to the caller everything behaves as if enqueued on
+ *     `stream`.  guard_set_overlap(ctx, 0) turns that off.)  Calls on one context must be
+ *     issued in order on streams that are ordered with respect to each other.
  *   - Every function returns a status (GUARD_OK = 0, errors negative) and never throws,
  *     aborts or traps.  Argument errors are detected on the host before anything is
  *     enqueued.  Data-dependent errors (non-finite telemetry, a bounded wait that ran out)
@@ -193,6 +196,9 @@ int guard_sync_status(guard_ctx *ctx, void *stream);
 
 /* Clears the ring position, exceedance ring, consecutive counters and status. */
 int guard_reset(guard_ctx *ctx, void *stream);
+
+/* Enables (default) or disables the internal fork/join stream described under Conventions. */
+int guard_set_overlap(guard_ctx *ctx, int on);
 
 /* Kernel timing for benchmarks: while enabled, guard_ingest records a pair of CUDA events on
  * the stream right around its main kernel (the fused cross-rank sweep; contexts whose sizes

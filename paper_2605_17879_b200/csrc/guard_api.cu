@@ -112,6 +112,23 @@ struct guard_ctx {
     long long seen;
     long long launches;  // kernels enqueued by this context so far
     long long evals;     // evaluations since creation / reset
+    // overlap of the window medians (which need only the ring) with the cross-rank kernels of the
+    // ingest that precedes them: an internal stream forked from and joined into the caller's
+    bool overlap = true;
+    bool fork_fresh = false;          // ev_fork was recorded by an ingest not yet followed by an evaluation
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    bool ensure_side() {
+        if (side) return true;
+        if (cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking) != cudaSuccess) { side = nullptr; return false; }
+        if (cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming) != cudaSuccess) {
+            cudaStreamDestroy(side);
+            side = nullptr;
+            return false;
+        }
+        return true;
+    }
     bool profiling = false;                                   // record events around the main ingest kernel
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof;    // recorded, not yet read
     char error[256];
@@ -247,6 +264,9 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
                                 cudaMemcpyDeviceToDevice, st);
         if (e != cudaSuccess) return c->cuda_fail(e, "cudaMemcpyAsync(ring)");
     }
+    // the ring now holds the block (in stream order): evaluations may start reading it from here
+    c->fork_fresh = false;
+    if (c->overlap && c->ensure_side() && cudaEventRecord(c->ev_fork, st) == cudaSuccess) c->fork_fresh = true;
     XrankArgs a{};
     a.base = c->ring();
     a.row_stride = (long long)row;
@@ -290,7 +310,20 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     w.wmed_user = d_wmed;
     w.use_hint = c->evals > 0 ? 1 : 0;
     w.status = c->status();
-    cudaError_t e = launch_window_select(w, st);
+    // The window medians read only the ring: run them on the internal stream, forked where the
+    // ring became complete, so that they overlap the cross-rank kernels of the preceding ingest;
+    // the caller's stream waits for them before anything that uses them.
+    cudaError_t e;
+    const bool forked = c->overlap && c->fork_fresh && c->side;
+    c->fork_fresh = false;
+    if (forked) {
+        e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
+        if (e == cudaSuccess) e = launch_window_select(w, c->side);
+        if (e == cudaSuccess) e = cudaEventRecord(c->ev_join, c->side);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_join, 0);
+    } else {
+        e = launch_window_select(w, st);
+    }
     if (e != cudaSuccess) return c->cuda_fail(e, "window_select launch");
 
     XrankArgs x{};
@@ -498,8 +531,22 @@ int64_t guard_fallback_steps(guard_ctx *c, void *stream) {
     return (int64_t)n;
 }
 
+int guard_set_overlap(guard_ctx *c, int on) {
+    if (!c) return GUARD_ERR_ARG;
+    c->overlap = on != 0;
+    c->fork_fresh = false;
+    return GUARD_OK;
+}
+
 void guard_destroy(guard_ctx *c) {
-    if (c) guard_profile_enable(c, 0);
+    if (c) {
+        guard_profile_enable(c, 0);
+        if (c->side) {
+            cudaStreamDestroy(c->side);
+            cudaEventDestroy(c->ev_fork);
+            cudaEventDestroy(c->ev_join);
+        }
+    }
     delete c;
 }
 

@@ -77,6 +77,8 @@ def lib():
         L.guard_fallback_steps.argtypes = [vp, vp]
         L.guard_fallback_reasons.restype = C.c_int
         L.guard_fallback_reasons.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        L.guard_set_overlap.restype = C.c_int
+        L.guard_set_overlap.argtypes = [vp, C.c_int]
         L.guard_profile_enable.restype = C.c_int
         L.guard_profile_enable.argtypes = [vp, C.c_int]
         L.guard_profile_read.restype = C.c_int
@@ -194,6 +196,10 @@ class Guard:
             self._check(lib().guard_fallback_reasons(self._h, out, _stream()))
         names = ("cta_list", "step_list", "deferred_list", "median_miss", "select", "mad_miss")
         return dict(zip(names, [int(v) for v in out]))
+
+    def set_overlap(self, on: bool) -> None:
+        """Window medians of an evaluation on an internal stream overlapping the preceding ingest."""
+        self._check(lib().guard_set_overlap(self._h, 1 if on else 0))
 
     def profile_enable(self, on: bool = True) -> None:
         self._check(lib().guard_profile_enable(self._h, 1 if on else 0))

@@ -110,6 +110,33 @@ def test_in_place_ingest_equals_copy_ingest():
         assert np.array_equal(a[key], b[key])
 
 
+def test_overlap_stream_on_and_off_agree():
+    """The window medians may run on an internal stream overlapping the preceding ingest; with
+    that switched off the same results must come out (and both match the oracle)."""
+    from paper_2605_17879_b200 import guard
+    X, dirs = _rand_fleet(60, 4500, 8, seed=21)
+    Xd = torch.from_numpy(X).cuda()
+    res = []
+    for overlap in (True, False):
+        g = guard.Guard(4500, 8, 20, 10, dir=dirs, capacity=40, topk=8)
+        g.set_overlap(overlap)
+        outs = []
+        for t in range(0, 60, 20):
+            g.ingest(Xd[t:t + 20])
+            o = g.score()
+            g.sync_status()
+            outs.append({k: to_np(v).copy() for k, v in o.items()})
+        res.append(outs)
+        g.close()
+    o = go.Oracle(4500, 8, 20, 10, 8, dir=dirs)
+    for i, t in enumerate(range(0, 60, 20)):
+        o.ingest(X[t:t + 20])
+        ref = o.score()
+        for key in ("wmed", "fleet_med", "fleet_mad", "counts", "mask", "flags", "tier", "topk_idx"):
+            assert_bit_equal(res[0][i][key], ref[key], key)
+            assert_bit_equal(res[1][i][key], ref[key], key)
+
+
 def test_long_window_paths():
     # windows too long for the warp-per-series path: 128-, 64- and 32-column staged tiles, and the
     # global-memory fallback
