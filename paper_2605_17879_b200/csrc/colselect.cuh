@@ -63,29 +63,32 @@ __device__ __forceinline__ uint32_t col_select(uint32_t *col, int stride, int n,
     return col[(size_t)l * stride];
 }
 
-// Median of a column of keys (midpoint rule for even n).  For even n the upper middle
-// element (rank n/2) is selected; the lower middle one is then the largest key among the
+// Keys of ranks k - 1 (if want_prev) and k of a column.  Rank k is selected; rank k - 1 is then
+// the same key if a further copy of it sits before position k, else the largest key among the
 // positions the partitioning left before it.
-__device__ __forceinline__ float col_median(uint32_t *col, int stride, int n) {
+__device__ __forceinline__ void col_rank_pair(uint32_t *col, int stride, int n, int k, bool want_prev, uint32_t &v_prev,
+                                              uint32_t &v_k) {
     int below_end;
-    const int k = n >> 1;   // n odd: the middle; n even: the upper middle
-    const uint32_t v2 = col_select(col, stride, n, k, &below_end);
-    if (n & 1) return key2f(v2);
-    // rank k - 1: equal to v2 if a further copy of it sits at or before position k - 1,
-    // i.e. if fewer than k keys are strictly below v2; otherwise the maximum of the keys
-    // strictly below v2, all of which lie in positions [0, below_end).
-    uint32_t v1 = v2;
-    if (below_end >= k) {
-        v1 = 0;
+    v_k = col_select(col, stride, n, k, &below_end);
+    v_prev = v_k;
+    if (want_prev && below_end >= k) {
+        uint32_t m = 0;
         for (int i = 0; i < below_end; i += kSelBatch) {
             uint32_t v[kSelBatch];
 #pragma unroll
             for (int u = 0; u < kSelBatch; ++u) v[u] = (i + u < below_end) ? col[(size_t)(i + u) * stride] : 0u;
 #pragma unroll
-            for (int u = 0; u < kSelBatch; ++u) v1 = max(v1, v[u]);
+            for (int u = 0; u < kSelBatch; ++u) m = max(m, v[u]);
         }
+        v_prev = m;
     }
-    return median_from_keys(v1, v2, true);
+}
+
+// Median of a column of keys (midpoint rule for even n): ranks n/2 - 1 and n/2, or the middle.
+__device__ __forceinline__ float col_median(uint32_t *col, int stride, int n) {
+    uint32_t v1, v2;
+    col_rank_pair(col, stride, n, n >> 1, !(n & 1), v1, v2);
+    return median_from_keys(v1, v2, !(n & 1));
 }
 
 // ---- bulk async copy (TMA) + mbarrier ---------------------------------------------------
@@ -98,6 +101,9 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;

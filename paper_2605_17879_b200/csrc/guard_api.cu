@@ -17,7 +17,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, xr_big, mask, ring, total;
+    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wlist, xr_big, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_fused;   // the single-launch fused cross-rank path applies
 };
@@ -36,6 +36,8 @@ Layout make_layout(int R, int M, int C, int K) {
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
+    L.wspread = off;   off = align_up(off + (size_t)R * M * sizeof(float));
+    L.wlist = off;     off = align_up(off + (size_t)R * M * sizeof(uint32_t));
     L.xr_big = off;    off = align_up(off + (L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps)
                                                       : (L.xr_fused ? (size_t)kFusedMaxSteps * M * 8 * sizeof(uint32_t) : 0)));
     L.mask = off;      off = align_up(off + (size_t)C * R * (M <= 8 ? 1 : 4));
@@ -309,6 +311,9 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     w.wmed = c->wmed();
     w.wmed_user = d_wmed;
     w.use_hint = c->evals > 0 ? 1 : 0;
+    w.spread = (float *)(c->ws + c->L.wspread);
+    w.fb_list = (uint32_t *)(c->ws + c->L.wlist);
+    w.fb_count = c->status() + 8;
     w.status = c->status();
     // The window medians read only the ring: run them on the internal stream, forked where the
     // ring became complete, so that they overlap the cross-rank kernels of the preceding ingest;
@@ -361,7 +366,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     e = launch_score_flag(s, c->p, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
     c->evals += 1;
-    c->launches += 2;
+    c->launches += 1 + window_launch_count(w);
 
     if (c->K > 0 && (d_topk_idx || d_topk_score)) {
         TopkArgs t{};

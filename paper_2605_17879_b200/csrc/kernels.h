@@ -74,9 +74,14 @@ struct WindowArgs {
     float *wmed;            // [series] (never NULL)
     int use_hint;           // wmed holds the previous evaluation's medians: use them as first pivots
     float *wmed_user;       // or NULL
+    float *spread;          // [series] tuned half-width of the bracket path's interval (state), or NULL
+    uint32_t *fb_list;      // [series] series the bracket path hands to the list kernel, or NULL
+    uint32_t *fb_count;     // their number
     uint32_t *status;
 };
+// Launches 1 kernel (warp or staged path) or 2 (bracket path + list kernel).
 cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st);
+int window_launch_count(const WindowArgs &a);
 
 // Fused k-of-W count, robust score, thresholds, multi-signal flag, tier, consecutive counter.
 struct ScoreArgs {

@@ -232,6 +232,21 @@ __device__ __forceinline__ bool warp_median(const uint32_t (&kv)[VPL], const int
     return false;
 }
 
+// A first guess of the half-width the bracket path should search around a series' previous
+// median: 0.45 x the mean absolute deviation of the window about its median (for Gaussian
+// noise that spans about +-0.36 sigma, some 3 standard errors of a 200-step median and ~28 %
+// of the window).  Only a starting point: the bracket path re-tunes it from its own counts.
+template <int VPL>
+__device__ __forceinline__ float warp_spread_guess(const uint32_t (&kv)[VPL], const int n, const float med) {
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+        if (kv[i] != 0xFFFFFFFFu) s += fabsf(key2f(kv[i]) - med);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    return 0.45f * s / (float)n;
+}
+
 template <int VPL>
 __global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a, const int ntiles, const int use_bulk) {
     extern __shared__ __align__(128) uint32_t wbuf[];   // 2 x [n][kWarpPitch]
@@ -303,10 +318,12 @@ __global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a
             float med = 0.0f;
             const uint32_t hint = a.use_hint ? f2key(a.wmed[series]) : 0u;   // last evaluation's median
             const bool ok = warp_median<VPL>(kv, nreal, n, hint, med);
+            const float h0 = warp_spread_guess<VPL>(kv, n, med);
             if (lane == 0) {
                 if (!ok) atomicOr(a.status, kStatInternal);
                 a.wmed[series] = med;
                 if (a.wmed_user) a.wmed_user[series] = med;
+                if (a.spread) a.spread[series] = h0;
             }
         }
         __syncthreads();   // every warp is done with this buffer before it is refilled
@@ -324,6 +341,160 @@ cudaError_t launch_warp_path(const WindowArgs &a, int use_bulk, cudaStream_t st)
     const int ntiles = (a.series + kWarpTileCols - 1) / kWarpTileCols;
     const int grid = ntiles < 2 * sms ? ntiles : 2 * sms;
     window_warp_kernel<VPL><<<grid, 1024, smem, st>>>(a, ntiles, use_bulk);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Bracket path: from the second evaluation on, a series' previous median and a tuned
+// half-width h give an interval [hint - h, hint + h] that almost always holds the new middle
+// elements.  One THREAD per series then suffices: the window's rows stream through a small
+// TMA-fed ring of shared-memory stages (8 rows x 256 series each), every thread counts its
+// keys below the interval and keeps those inside it (a few dozen) in its own shared-memory
+// column, checks from the counts that the middle ranks are among them and selects them there.
+// That is ~10 instructions per element and thread instead of a warp's cooperative walk.
+// Series whose interval missed (or overflowed) go to a list that a warp-per-series kernel
+// finishes exactly; h is re-tuned every time from the number of keys the interval caught.
+// ---------------------------------------------------------------------------------------
+constexpr int kBrCols = 256;     // series per CTA = threads per CTA
+constexpr int kBrRows = 8;       // rows per stage (one per warp)
+constexpr int kBrStages = 4;
+constexpr int kBrSlots = 72;     // kept keys per series
+constexpr int kBrTarget = 44;    // number of keys the interval is tuned to catch
+
+__global__ void __launch_bounds__(kBrCols, 2) window_bracket_kernel(const WindowArgs a) {
+    extern __shared__ __align__(128) uint32_t bsm[];
+    uint32_t *tile = bsm;                                        // [kBrStages][kBrRows][kBrCols]
+    uint32_t *kept = bsm + kBrStages * kBrRows * kBrCols;        // [kBrSlots][kBrCols]
+    __shared__ __align__(8) uint64_t bar[kBrStages];
+    const int tid = threadIdx.x, lane = lane_id(), w = warp_id();
+    const int n = a.n;
+    const int col0 = blockIdx.x * kBrCols;
+    const int ncols = min(kBrCols, a.series - col0);
+    const int c = col0 + tid;
+    const bool active = tid < ncols;
+    const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;
+    const int nchunks = (n + kBrRows - 1) / kBrRows;
+
+    if (tid == 0)
+        for (int s = 0; s < kBrStages; ++s) mbar_init(&bar[s], kBrRows);
+    __syncthreads();
+    // lane 0 of warp w feeds row w of every chunk (or just arrives when the chunk has no such row)
+    auto feed = [&](int chunk) {
+        if (lane != 0) return;
+        const int stage = chunk % kBrStages;
+        const int row = chunk * kBrRows + w;
+        if (row < n) {
+            int slot = first + row;
+            if (slot >= a.capacity) slot -= a.capacity;
+            mbar_arrive_expect_tx(&bar[stage], (uint32_t)ncols * 4u);
+            bulk_g2s(tile + (stage * kBrRows + w) * kBrCols, a.ring + (size_t)slot * a.row_stride + col0, (uint32_t)ncols * 4u,
+                     &bar[stage]);
+        } else {
+            mbar_arrive(&bar[stage]);
+        }
+    };
+    for (int ch = 0; ch < kBrStages && ch < nchunks; ++ch) feed(ch);
+
+    float hint = 0.0f, h = 0.0f;
+    if (active) { hint = a.wmed[c]; h = a.spread[c]; }
+    const bool usable = active && (h > 0.0f) && (h < 3.0e38f) && (fabsf(hint) < 3.0e38f);
+    // an unusable interval keeps nothing and counts nothing below it: it fails the check below
+    const uint32_t klo = usable ? f2key(hint - h) : 0xFFFFFFFFu, khi = usable ? f2key(hint + h) : 0u;
+    int clt = 0, nk = 0;
+    for (int ch = 0; ch < nchunks; ++ch) {
+        const int stage = ch % kBrStages;
+        if (!mbar_wait_bounded(&bar[stage], (uint32_t)((ch / kBrStages) & 1), kWaitLimitCycles)) {
+            atomicOr(a.status, kStatTimeout);
+            for (int s2 = 0; s2 < kBrStages; ++s2) {   // let copies in flight land before leaving
+                const int fed = ch + ((s2 - stage + kBrStages) % kBrStages);   // the chunk stage s2 is waiting for
+                if (fed < nchunks) mbar_wait_bounded(&bar[s2], (uint32_t)((fed / kBrStages) & 1), kWaitLimitCycles);
+            }
+            return;
+        }
+        const int rows = min(kBrRows, n - ch * kBrRows);
+        const uint32_t *t = tile + stage * kBrRows * kBrCols + tid;
+#pragma unroll
+        for (int r = 0; r < kBrRows; ++r) {
+            if (r < rows) {
+                const uint32_t key = key_of_bits(t[r * kBrCols]);
+                clt += (key < klo);
+                if (key >= klo && key <= khi) {
+                    if (nk < kBrSlots) kept[nk * kBrCols + tid] = key;
+                    ++nk;
+                }
+            }
+        }
+        __syncthreads();   // the stage is free again
+        if (ch + kBrStages < nchunks) feed(ch + kBrStages);
+    }
+    if (!active) return;
+    const bool even = !(n & 1);
+    const int k1 = (n - 1) >> 1, k2 = n >> 1;
+    const bool ok = usable && clt <= k1 && k2 < clt + nk && nk <= kBrSlots;
+    if (ok) {
+        uint32_t v1, v2;
+        col_rank_pair(kept + tid, kBrCols, nk, k2 - clt, even, v1, v2);
+        const float med = median_from_keys(v1, v2, even);
+        a.wmed[c] = med;
+        if (a.wmed_user) a.wmed_user[c] = med;
+        // re-tune the half-width so that the interval catches about kBrTarget keys next time
+        const float f = fminf(2.0f, fmaxf(0.5f, (float)kBrTarget / (float)max(nk, 1)));
+        a.spread[c] = h * f;
+    } else {
+        a.fb_list[atomicAdd(a.fb_count, 1u)] = (uint32_t)c;   // the list kernel finishes this series
+    }
+}
+
+// Finishes the series the bracket path could not: one warp per listed series, window read
+// straight from the ring (few series, so the scattered loads do not matter).
+template <int VPL>
+__global__ void __launch_bounds__(256) window_list_kernel(const WindowArgs a) {
+    const int lane = lane_id();
+    const int wglobal = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, wtotal = (gridDim.x * blockDim.x) >> 5;
+    const int n = a.n;
+    const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;
+    const uint32_t count = *a.fb_count;
+    for (uint32_t i = wglobal; i < count; i += wtotal) {
+        const int series = (int)a.fb_list[i];
+        uint32_t kv[VPL];
+        int nreal = 0;
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int row = lane + 32 * j;
+            kv[j] = 0xFFFFFFFFu;
+            if (row < n) {
+                int slot = first + row;
+                if (slot >= a.capacity) slot -= a.capacity;
+                kv[j] = f2key(a.ring[(size_t)slot * a.row_stride + series]);
+                ++nreal;
+            }
+        }
+        lane_sort<VPL>(kv);
+        float med = 0.0f;
+        const bool ok = warp_median<VPL>(kv, nreal, n, 0u, med);
+        const float h0 = warp_spread_guess<VPL>(kv, n, med);
+        if (lane == 0) {
+            if (!ok) atomicOr(a.status, kStatInternal);
+            a.wmed[series] = med;
+            if (a.wmed_user) a.wmed_user[series] = med;
+            a.spread[series] = h0;
+        }
+    }
+}
+
+template <int VPL>
+cudaError_t launch_bracket_path(const WindowArgs &a, cudaStream_t st) {
+    const size_t smem = (size_t)(kBrStages * kBrRows + kBrSlots) * kBrCols * 4;
+    cudaError_t e = cudaFuncSetAttribute(window_bracket_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(a.fb_count, 0, sizeof(uint32_t), st);
+    if (e != cudaSuccess) return e;
+    window_bracket_kernel<<<(a.series + kBrCols - 1) / kBrCols, kBrCols, smem, st>>>(a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    window_list_kernel<VPL><<<sms, 256, 0, st>>>(a);
     return cudaGetLastError();
 }
 
@@ -381,11 +552,21 @@ cudaError_t launch_staged(const WindowArgs &a, int use_bulk, cudaStream_t st) {
 
 }  // namespace
 
+int window_launch_count(const WindowArgs &a) {
+    const bool bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
+    return (a.use_hint && bulk && a.spread && a.fb_list && a.n <= 256) ? 2 : 1;
+}
+
 cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st) {
     constexpr size_t kMaxTile = 200 * 1024;
     // bulk copies need 16-byte aligned sources and sizes
     const int use_bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
     const size_t n = (size_t)a.n;
+    if (a.use_hint && use_bulk && a.spread && a.fb_list && n <= 256) {
+        if (n <= 64) return launch_bracket_path<2>(a, st);
+        if (n <= 128) return launch_bracket_path<4>(a, st);
+        return launch_bracket_path<8>(a, st);
+    }
     if (n <= 64) return launch_warp_path<2>(a, use_bulk, st);
     if (n <= 128) return launch_warp_path<4>(a, use_bulk, st);
     if (n <= 256) return launch_warp_path<8>(a, use_bulk, st);
