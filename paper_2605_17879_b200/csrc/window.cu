@@ -2,6 +2,8 @@
 // last n ring steps.  A CTA stages a [n steps] x [TC series] tile of the ring in shared
 // memory with bulk asynchronous copies (one per ring row, completion on an mbarrier),
 // then every thread selects inside its own column.
+#include <math_constants.h>
+
 #include "colselect.cuh"
 #include "kernels.h"
 
@@ -359,7 +361,50 @@ constexpr int kBrCols = 256;     // series per CTA = threads per CTA
 constexpr int kBrRows = 8;       // rows per stage (one per warp)
 constexpr int kBrStages = 4;
 constexpr int kBrSlots = 72;     // kept keys per series
-constexpr int kBrTarget = 44;    // number of keys the interval is tuned to catch
+constexpr int kBrTarget = 52;    // number of keys the interval is tuned to catch
+
+// Ranks t - 1 and t among the nk keys a thread kept (column `col`, pitch kBrCols), all inside
+// [klo, khi].  Kept keys of a narrow interval are close to evenly spread, so the pivot is
+// interpolated in key space (regula falsi on the count below the pivot): a pass counts the
+// keys below the pivot and tracks the two largest keys below it and the two smallest keys not
+// below it; when t - 1, t or t + 1 keys are below, two of those four ARE ranks t - 1 and t.
+// Every thread runs the same fixed-length scans, so a warp does not diverge the way per-thread
+// partitioning does.  Returns false after a few passes (e.g. when the ranks sit inside a long
+// run of equal keys) to let the caller fall back to partitioning.
+__device__ __forceinline__ bool kept_rank_pair(const uint32_t *col, int nk, int t, uint32_t klo, uint32_t khi,
+                                               uint32_t &v_prev, uint32_t &v_t) {
+    unsigned long long pl = klo, ph = (unsigned long long)khi + 1ull;   // counts below: al at pl, ah at ph
+    int al = 0, ah = nk;
+    for (int pass = 0; pass < 8; ++pass) {
+        if (ph - pl < 2ull) return false;
+        // aim between the bracket's ends in proportion to the missing count
+        unsigned long long p = pl + (unsigned long long)((float)(ph - pl) * (((float)(t - al) + 0.5f) / (float)(ah - al)));
+        p = p <= pl ? pl + 1ull : (p >= ph ? ph - 1ull : p);
+        const uint32_t pv = (uint32_t)p;
+        int below = 0;
+        uint32_t b1 = 0u, b2 = 0u, u1 = 0xFFFFFFFFu, u2 = 0xFFFFFFFFu;
+        for (int i = 0; i < nk; i += kSelBatch) {
+            uint32_t v[kSelBatch];
+#pragma unroll
+            for (int q = 0; q < kSelBatch; ++q) v[q] = (i + q < nk) ? col[(size_t)(i + q) * kBrCols] : 0xFFFFFFFFu;
+#pragma unroll
+            for (int q = 0; q < kSelBatch; ++q) {
+                const bool lt = v[q] < pv;
+                below += lt;
+                const uint32_t lo_v = lt ? v[q] : 0u, hi_v = lt ? 0xFFFFFFFFu : v[q];   // neutral on the other side
+                b2 = max(b2, min(b1, lo_v));
+                b1 = max(b1, lo_v);
+                u2 = min(u2, max(u1, hi_v));
+                u1 = min(u1, hi_v);
+            }
+        }
+        if (below == t) { v_prev = b1; v_t = u1; return true; }
+        if (below == t + 1) { v_prev = b2; v_t = b1; return true; }
+        if (below == t - 1) { v_prev = u1; v_t = u2; return true; }
+        if (below < t) { pl = p; al = below; } else { ph = p; ah = below; }
+    }
+    return false;
+}
 
 __global__ void __launch_bounds__(kBrCols, 2) window_bracket_kernel(const WindowArgs a) {
     extern __shared__ __align__(128) uint32_t bsm[];
@@ -398,8 +443,15 @@ __global__ void __launch_bounds__(kBrCols, 2) window_bracket_kernel(const Window
     float hint = 0.0f, h = 0.0f;
     if (active) { hint = a.wmed[c]; h = a.spread[c]; }
     const bool usable = active && (h > 0.0f) && (h < 3.0e38f) && (fabsf(hint) < 3.0e38f);
-    // an unusable interval keeps nothing and counts nothing below it: it fails the check below
-    const uint32_t klo = usable ? f2key(hint - h) : 0xFFFFFFFFu, khi = usable ? f2key(hint + h) : 0u;
+    // The interval is tested with float compares (keys are made only of what is kept).  That
+    // agrees with the key order as long as an end that is zero admits both zeros: -0 as lower
+    // end, +0 as upper end.  An unusable interval keeps nothing and counts nothing below it, so
+    // it fails the check after the loop.
+    float flo = hint - h, fhi = hint + h;
+    if (flo == 0.0f) flo = -0.0f;
+    if (fhi == 0.0f) fhi = 0.0f;
+    if (!usable) { flo = CUDART_INF_F; fhi = -CUDART_INF_F; }
+    const uint32_t klo = usable ? f2key(flo) : 0xFFFFFFFFu, khi = usable ? f2key(fhi) : 0u;
     int clt = 0, nk = 0;
     for (int ch = 0; ch < nchunks; ++ch) {
         const int stage = ch % kBrStages;
@@ -413,13 +465,15 @@ __global__ void __launch_bounds__(kBrCols, 2) window_bracket_kernel(const Window
         }
         const int rows = min(kBrRows, n - ch * kBrRows);
         const uint32_t *t = tile + stage * kBrRows * kBrCols + tid;
+        float x[kBrRows];
+#pragma unroll
+        for (int r = 0; r < kBrRows; ++r) x[r] = __uint_as_float(t[r * kBrCols]);
 #pragma unroll
         for (int r = 0; r < kBrRows; ++r) {
-            if (r < rows) {
-                const uint32_t key = key_of_bits(t[r * kBrCols]);
-                clt += (key < klo);
-                if (key >= klo && key <= khi) {
-                    if (nk < kBrSlots) kept[nk * kBrCols + tid] = key;
+            if (r < rows) {   // rows beyond the window's end hold stale data
+                clt += (x[r] < flo);
+                if (x[r] >= flo && x[r] <= fhi) {
+                    if (nk < kBrSlots) kept[nk * kBrCols + tid] = f2key(x[r]);
                     ++nk;
                 }
             }
@@ -433,13 +487,15 @@ __global__ void __launch_bounds__(kBrCols, 2) window_bracket_kernel(const Window
     const bool ok = usable && clt <= k1 && k2 < clt + nk && nk <= kBrSlots;
     if (ok) {
         uint32_t v1, v2;
-        col_rank_pair(kept + tid, kBrCols, nk, k2 - clt, even, v1, v2);
-        const float med = median_from_keys(v1, v2, even);
+        const int t = k2 - clt;   // rank of the upper middle among the kept keys (t >= 1 when even)
+        if (!kept_rank_pair(kept + tid, nk, t, klo, khi, v1, v2)) col_rank_pair(kept + tid, kBrCols, nk, t, even, v1, v2);
+        const float med = median_from_keys(even ? v1 : v2, v2, even);
         a.wmed[c] = med;
         if (a.wmed_user) a.wmed_user[c] = med;
         // re-tune the half-width so that the interval catches about kBrTarget keys next time
+        // (half of the way: one window's count is a noisy estimate of the density)
         const float f = fminf(2.0f, fmaxf(0.5f, (float)kBrTarget / (float)max(nk, 1)));
-        a.spread[c] = h * f;
+        a.spread[c] = h * (0.5f + 0.5f * f);
     } else {
         a.fb_list[atomicAdd(a.fb_count, 1u)] = (uint32_t)c;   // the list kernel finishes this series
     }
