@@ -363,13 +363,11 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     s.metric_mask = d_metric_mask;
     s.flags = d_flags;
     s.tier = d_tier;
-    e = launch_score_flag(s, c->p, st);
-    if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
-    c->evals += 1;
-    c->launches += 1 + window_launch_count(w);
-
-    if (c->K > 0 && (d_topk_idx || d_topk_score)) {
-        TopkArgs t{};
+    // top-k and the score pass are independent of each other: top-k goes to the internal stream
+    const bool want_topk = c->K > 0 && (d_topk_idx || d_topk_score);
+    bool topk_forked = false;
+    TopkArgs t{};
+    if (want_topk) {
         t.R = c->R;
         t.M = c->M;
         t.K = c->K;
@@ -380,6 +378,24 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         t.ticket = c->ticket();
         t.idx = d_topk_idx;
         t.score = d_topk_score;
+        if (c->overlap && c->ensure_side()) {
+            e = cudaEventRecord(c->ev_fork, st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
+            if (e == cudaSuccess) e = launch_topk(t, c->p, c->side);
+            if (e == cudaSuccess) e = cudaEventRecord(c->ev_join, c->side);
+            if (e != cudaSuccess) return c->cuda_fail(e, "topk launch");
+            topk_forked = true;
+            c->launches += 1;
+        }
+    }
+    e = launch_score_flag(s, c->p, st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
+    c->evals += 1;
+    c->launches += 1 + window_launch_count(w);
+    if (topk_forked) {
+        e = cudaStreamWaitEvent(st, c->ev_join, 0);
+        if (e != cudaSuccess) return c->cuda_fail(e, "topk join");
+    } else if (want_topk) {
         e = launch_topk(t, c->p, st);
         if (e != cudaSuccess) return c->cuda_fail(e, "topk launch");
         c->launches += 1;
