@@ -3,8 +3,8 @@
 // fleets whose candidate lists fit in shared memory (4 or 8 metrics, up to ~20 000 ranks
 // with 8 metrics).  The step's row is streamed twice (the second time it comes out of L2):
 //
-//   0. sample      (a small kernel of its own) two warps per metric sort 512 strided samples
-//                  each in registers; seven order statistics of the merged sample (middle +-
+//   0. sample      (a small kernel of its own, one 64-thread CTA per column) two warps sort 512
+//                  strided samples each in registers; seven order statistics of the merged sample (middle +-
 //                  delta, quartiles +- delta) give the interval [lo, hi] of the median and
 //                  [dlo, dhi] of the MAD;
 //   1. sweep       every element is counted if below lo and kept (shared-memory list) if
@@ -127,41 +127,38 @@ __device__ bool group_select(const uint32_t *list, uint32_t n, uint32_t k, bool 
     return ok;
 }
 
-// Sample kernel of the fused path: one CTA per step, two warps per metric.  Each warp sorts
-// 512 strided samples of its column in registers; seven order statistics of the two merged
-// halves (middle, middle +- delta, quartiles +- delta_q) go to scratch as keys.  It is a
-// kernel of its own because the register sort wants more than the 64 registers a thread
-// gets inside the 1024-thread fused kernel.
-__global__ void __launch_bounds__(512) xrank_sample_q_kernel(const XrankArgs a, const int delta, const int delta_q,
-                                                             uint32_t *__restrict__ qout) {
-    __shared__ uint32_t samp[kMaxMetrics > 8 ? 8 * 1024 : 8 * 1024];
-    const int t = blockIdx.x, tid = threadIdx.x, lane = lane_id(), warp = warp_id();
+// Sample kernel of the fused path: one CTA of two warps per (step, metric) column.  Each warp
+// sorts 512 strided samples of the column in registers; seven order statistics of the two
+// merged halves (middle, middle +- delta, quartiles +- delta_q) go to scratch as keys.  It is a
+// kernel of its own because the register sort wants more than the 64 registers a thread gets
+// inside the 1024-thread fused kernel, and small CTAs spread evenly over the SMs.
+__global__ void __launch_bounds__(64) xrank_sample_q_kernel(const XrankArgs a, const int delta, const int delta_q,
+                                                            uint32_t *__restrict__ qout) {
+    __shared__ uint32_t samp[2 * 512];
+    const int m = blockIdx.x, t = blockIdx.y, tid = threadIdx.x, lane = lane_id(), h = warp_id();
     const int R = a.R, M = a.M;
     const int slot = (int)(((long long)a.first_slot + t) % a.capacity);
     const float *row = a.base + (size_t)slot * a.row_stride;
-    if (warp < 2 * M) {
-        const int m = warp >> 1, h = warp & 1;
-        const int stride = R / kFuSample;
-        uint32_t v[16];
+    const int stride = R / kFuSample;
+    uint32_t v[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int e = h * 512 + lane * 16 + j;
-            v[j] = f2key(__ldg(row + (size_t)(e * stride + (stride >> 1)) * M + m));
-        }
-        warp_bitonic_sort<16>(v, lane);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) samp[(m * 2 + h) * 512 + lane * 16 + j] = v[j];
+    for (int j = 0; j < 16; ++j) {
+        const int e = h * 512 + lane * 16 + j;
+        v[j] = f2key(__ldg(row + (size_t)(e * stride + (stride >> 1)) * M + m));
     }
+    warp_bitonic_sort<16>(v, lane);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) samp[h * 512 + lane * 16 + j] = v[j];
     __syncthreads();
-    if (tid < M * 8) {
-        const int m = tid >> 3, qq = tid & 7;
+    if (tid < 8) {
+        const int qq = tid;
         const int mid = kFuSample / 2, q1 = kFuSample / 4, q3 = 3 * kFuSample / 4;
         int k = mid;
         if (qq == 0) k = mid - delta; else if (qq == 2) k = mid + delta;
         else if (qq == 3) k = q1 - delta_q; else if (qq == 4) k = q1 + delta_q;
         else if (qq == 5) k = q3 - delta_q; else if (qq == 6) k = q3 + delta_q;
         k = min(max(k, 0), kFuSample - 1);
-        qout[((size_t)t * M + m) * 8 + qq] = kth_of_two(samp + (m * 2) * 512, samp + (m * 2 + 1) * 512, 512, k);
+        qout[((size_t)t * M + m) * 8 + qq] = kth_of_two(samp, samp + 512, 512, k);
     }
 }
 
@@ -488,7 +485,7 @@ cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S,
     const int delta_q = (int)ceil(0.5 * 4.0 * 0.612 * sqrt((double)kFuSample));
     const size_t smem = (size_t)(kFuCandWords + a.M * kFuBins + kFuAmb) * sizeof(uint32_t);
     const bool wide = a.mask_bytes == 4;
-    xrank_sample_q_kernel<<<S, 64 * a.M, 0, st>>>(a, delta, delta_q, qscratch);
+    xrank_sample_q_kernel<<<dim3(a.M, S), 64, 0, st>>>(a, delta, delta_q, qscratch);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
