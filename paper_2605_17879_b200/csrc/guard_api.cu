@@ -20,6 +20,7 @@ struct Layout {
     size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wlist, xr_big, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_fused;   // the single-launch fused cross-rank path applies
+    int xr_cluster; // the cluster-per-step cross-rank path applies
 };
 
 // State and scratch first, the two rings last (the telemetry ring is by far the largest).
@@ -30,8 +31,9 @@ Layout make_layout(int R, int M, int C, int K) {
     L.ticket = off;    off = align_up(off + 64);
     L.fleet = off;     off = align_up(off + 3 * kMaxMetrics * sizeof(float));
     L.consec = off;    off = align_up(off + (size_t)R);
-    L.xr_fused = xrank_fused_supported(R, M) ? 1 : 0;
-    L.xr_steps = (!L.xr_fused && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
+    L.xr_cluster = xrank_cluster_supported(R, M) ? 1 : 0;
+    L.xr_fused = (!L.xr_cluster && xrank_fused_supported(R, M)) ? 1 : 0;
+    L.xr_steps = (!L.xr_cluster && !L.xr_fused && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
     L.xr_small = off;  off = align_up(off + (L.xr_steps ? xrank_scratch_small_bytes(M, L.xr_steps) : 0));
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
@@ -153,6 +155,11 @@ struct guard_ctx {
         if (xrank_column_supported(R) && (long long)S * M <= 64 && !a.cut) {
             launches += 1;
             return launch_xrank_column(a, p, S, st);
+        }
+        if (L.xr_cluster && a.mask_bytes == 1) {
+            a.fallbacks = status() + 1;
+            launches += 1;
+            return launch_xrank_cluster(a, p, S, status() + 2, st, (profiling && a.mask_base) ? &prof : nullptr);
         }
         if (L.xr_fused) {
             a.fallbacks = status() + 1;

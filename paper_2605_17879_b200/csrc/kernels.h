@@ -52,6 +52,10 @@ bool xrank_fused_supported(int R, int M);
 // prof: if not NULL, a pair of events recorded on st right around the main kernel is appended.
 cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, uint32_t *qscratch,
                                cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof = nullptr);
+// One cluster of four CTAs per step (4 or 8 metrics, a few thousand ranks and more).
+bool xrank_cluster_supported(int R, int M);
+cudaError_t launch_xrank_cluster(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, cudaStream_t st,
+                                 std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof = nullptr);
 constexpr int kFusedMaxSteps = 1024;   // steps per launch of the fused path (sizes its scratch)
 bool xrank_bracket_supported(int R, int M);
 int xrank_scratch_steps(int R, int M, int want);
