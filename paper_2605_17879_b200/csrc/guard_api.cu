@@ -21,6 +21,7 @@ struct Layout {
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_fused;   // the single-launch fused cross-rank path applies
     int xr_cluster; // the cluster-per-step cross-rank path applies
+    int xr_split;   // the six-kernel split cross-rank path applies
 };
 
 // State and scratch first, the two rings last (the telemetry ring is by far the largest).
@@ -31,17 +32,19 @@ Layout make_layout(int R, int M, int C, int K) {
     L.ticket = off;    off = align_up(off + 64);
     L.fleet = off;     off = align_up(off + 3 * kMaxMetrics * sizeof(float));
     L.consec = off;    off = align_up(off + (size_t)R);
-    L.xr_cluster = xrank_cluster_supported(R, M) ? 1 : 0;
-    L.xr_fused = (!L.xr_cluster && xrank_fused_supported(R, M)) ? 1 : 0;
-    L.xr_steps = (!L.xr_cluster && !L.xr_fused && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
+    L.xr_split = xrank_split_supported(R, M) ? 1 : 0;
+    L.xr_cluster = (!L.xr_split && xrank_cluster_supported(R, M)) ? 1 : 0;
+    L.xr_fused = (!L.xr_split && !L.xr_cluster && xrank_fused_supported(R, M)) ? 1 : 0;
+    L.xr_steps = (!L.xr_split && !L.xr_cluster && !L.xr_fused && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
     L.xr_small = off;  off = align_up(off + (L.xr_steps ? xrank_scratch_small_bytes(M, L.xr_steps) : 0));
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
     L.wspread = off;   off = align_up(off + (size_t)R * M * sizeof(float));
     L.wlist = off;     off = align_up(off + (size_t)R * M * sizeof(uint32_t));
-    L.xr_big = off;    off = align_up(off + (L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps)
-                                                      : (L.xr_fused ? (size_t)kFusedMaxSteps * M * 8 * sizeof(uint32_t) : 0)));
+    L.xr_big = off;    off = align_up(off + (L.xr_split ? xrank_split_scratch_bytes(R, M, C < kSplitMaxSteps ? C : kSplitMaxSteps)
+                                             : L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps)
+                                                          : (L.xr_fused ? (size_t)kFusedMaxSteps * M * 8 * sizeof(uint32_t) : 0)));
     L.mask = off;      off = align_up(off + (size_t)C * R * (M <= 8 ? 1 : 4));
     L.ring = off;      off = align_up(off + (size_t)C * R * M * sizeof(float));
     L.total = off;
@@ -155,6 +158,25 @@ struct guard_ctx {
         if (xrank_column_supported(R) && (long long)S * M <= 64 && !a.cut) {
             launches += 1;
             return launch_xrank_column(a, p, S, st);
+        }
+        if (L.xr_split && a.mask_bytes == 1) {
+            a.fallbacks = status() + 1;
+            const int first = a.first_slot;
+            const int smax = C < kSplitMaxSteps ? C : kSplitMaxSteps;
+            for (int s0 = 0; s0 < S; s0 += smax) {
+                const int n = (S - s0 < smax) ? (S - s0) : smax;
+                XrankArgs g = a;
+                g.first_slot = (int)(((long long)first + s0) % a.capacity);
+                g.med = a.med + (size_t)s0 * M;
+                g.mad = a.mad + (size_t)s0 * M;
+                if (a.med_user) g.med_user = a.med_user + (size_t)s0 * M;
+                if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
+                cudaError_t e = launch_xrank_split(g, p, n, ws + L.xr_big, status() + 2, st,
+                                                   (profiling && a.mask_base) ? &prof : nullptr);
+                if (e != cudaSuccess) return e;
+                launches += 6;
+            }
+            return cudaSuccess;
         }
         if (L.xr_cluster && a.mask_bytes == 1) {
             a.fallbacks = status() + 1;

@@ -56,6 +56,13 @@ cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S,
 bool xrank_cluster_supported(int R, int M);
 cudaError_t launch_xrank_cluster(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, cudaStream_t st,
                                  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof = nullptr);
+// Six uniform kernels per block (sample, sweep, select, sweep, select, finish) with the kept
+// elements in global scratch (4 or 8 metrics, a few thousand to ~20 000 ranks).
+bool xrank_split_supported(int R, int M);
+constexpr int kSplitMaxSteps = 256;   // steps per launch group of the split path (sizes its scratch)
+size_t xrank_split_scratch_bytes(int R, int M, int S_max);
+cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S, void *scratch, uint32_t *reasons,
+                               cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof = nullptr);
 constexpr int kFusedMaxSteps = 1024;   // steps per launch of the fused path (sizes its scratch)
 bool xrank_bracket_supported(int R, int M);
 int xrank_scratch_steps(int R, int M, int want);

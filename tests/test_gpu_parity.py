@@ -70,22 +70,22 @@ def test_bracketed_cross_rank_path(R, M, W, T, quant):
 
 
 @pytest.mark.parametrize("R,M,B,T,quant", [
-    (4096, 8, 12, 24, None),       # smallest fleet on the cluster path (blocks large enough to leave the column path)
-    (5000, 4, 20, 40, None),       # four metrics: one selection group per CTA; ragged last CTA
+    (4096, 8, 12, 24, None),       # smallest fleet on the split path (blocks large enough to leave the column path)
+    (5000, 4, 20, 40, None),       # four metrics; ragged last chunk
     (4100, 8, 9, 27, None),        # rank count not a multiple of 16: partial batches
     (16384, 8, 10, 20, None),      # width of the large configuration
-    (20000, 8, 9, 9, None),
+    (20000, 8, 9, 9, None),        # beyond the split path's kept-list size: cluster path
     (4096, 8, 12, 24, 50),         # quantised: intervals collapse onto tied values
     (8192, 4, 20, 20, 4),          # very coarse: kept lists overflow, every step takes the direct path
 ])
-def test_cluster_cross_rank_path(R, M, B, T, quant):
+def test_wide_block_cross_rank_paths(R, M, B, T, quant):
     X, dirs = _rand_fleet(T, R, M, seed=3 * R + M, quant=quant)
     run_both(X, B, max(1, B // 2), 16, dirs, [B], capacity=2 * B, min_signals=2)
 
 
-def test_cluster_path_degenerate_columns():
-    # constant, two-valued and single-valued steps inside a block of the cluster path: the
-    # sample cannot bracket anything, the direct path must take over for those steps only
+def test_wide_block_degenerate_columns():
+    # constant, two-valued and single-valued steps inside a wide block: the sample cannot
+    # bracket anything, the direct path must take over for those steps only
     X, dirs = _rand_fleet(24, 4096, 8, seed=78)
     X[2] = 1.0
     X[3, ::2] = 1.0
