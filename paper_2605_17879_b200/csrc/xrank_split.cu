@@ -3,9 +3,9 @@
 // of work on many small CTAs, so that the streaming sweeps run with all their warps streaming
 // and the short, latency-bound selections of hundreds of columns overlap one another:
 //
-//   0. sample   one CTA per (step, metric) column: 32 spread values are sorted in a warp;
-//               their median and quartile span fix a linear map onto 2048 bins; every
-//               stride-th rank of the column (about 4096 values) is counted into those bins;
+//   0. sample   one CTA per (step, four metrics): per metric 32 spread values are sorted in a
+//               warp; their median and quartile span fix a linear map onto 2048 bins; about
+//               4096 ranks of the step (runs of four, evenly spread) are counted into those bins;
 //               the bins that hold the sample ranks middle +- delta and quartiles +- delta_q
 //               give the interval [lo, hi] of the column's median and [dlo, dhi] of its MAD;
 //   1. sweep    one CTA per (step, chunk of ranks): counts the elements below lo and keeps
@@ -50,7 +50,7 @@ struct SpGeom {
     int slice;      // ranks per sweep CTA (a multiple of 16)
     int cap;        // kept elements per metric and sweep CTA (shared memory)
     int gcap;       // kept elements per column (global scratch)
-    int stride;     // sampled ranks are stride / 2, stride / 2 + stride, ...
+    int stride;     // one run of four consecutive ranks is sampled out of every 4 * stride
     int s;          // number of sampled ranks
     int delta;      // half-width of the median interval in sample ranks
     int delta_q;    // half-width of the quartile intervals in sample ranks
@@ -120,43 +120,59 @@ struct SpSelShared {
     uint32_t warp_tot[kSpSelThreads / 32];
     uint32_t bin, before, cnt, vmin, scount, r1, r2;
     int found;
-    float inv_bw, off;
-    int sample_ok;
-    uint32_t tk[6], tb[6];
     uint32_t small[32];
 };
 
-__global__ void __launch_bounds__(kSpSelThreads) xsplit_sample_kernel(const XrankArgs a, const SpGeom g, const SpScratch sc,
+constexpr int kSpSmpThreads = 256;                      // sample CTA: one per (step, quad of metrics)
+constexpr int kSpSmpG = kSpSmpThreads / 4;              // threads per metric in the scan
+constexpr int kSpSmpLoads = kSpSample / kSpSmpThreads;  // sampled ranks per thread
+
+struct SpSampleShared {
+    uint32_t hist[4][kSpBins];   // 2048 16-bit bins per metric
+    uint32_t warp_tot[4][2];
+    float inv_bw[4], off[4];
+    int ok[4];
+    uint32_t tk[6], tb[4][6];
+};
+
+// The sample of a step: runs of four consecutive ranks, one run every 4 * stride ranks, so
+// that a warp's 128-bit loads use whole cache lines (a column-wise strided sample costs one
+// line per value).  One CTA handles four metrics: every thread bins the four components of
+// its float4 into the four histograms; then 64 threads per metric scan their histogram.
+__global__ void __launch_bounds__(kSpSmpThreads) xsplit_sample_kernel(const XrankArgs a, const SpGeom g, const SpScratch sc,
                                                                       uint32_t *reasons) {
-    constexpr int G = kSpSelThreads, SPT = kSpSample / G;
-    __shared__ SpSelShared sh;
-    const int m = blockIdx.x, t = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
+    __shared__ SpSampleShared sh;
+    const int q = blockIdx.x, t = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int R = a.R, M = a.M;
     const int slot = (int)(((long long)a.first_slot + t) % a.capacity);
     const float *row = a.base + (size_t)slot * a.row_stride;
-    SpCol &col = sc.col[(size_t)t * M + m];
+    const int period = 4 * g.stride, first = (period - 4) >> 1;
 
-    // all loads first: the sample of the column and the 32 spread values that fix the bin map
-    float xs[SPT];
-    {
-        const float *p0 = row + (size_t)(tid * g.stride + (g.stride >> 1)) * M + m;
-        const size_t step = (size_t)G * g.stride * M;
-        const int nmine = (g.s - tid + G - 1) / G;   // samples of this thread
+    // all loads first: the sampled ranks, and (warps 0..3) the 32 spread values that fix a metric's bin map
+    float4 xs[kSpSmpLoads];
 #pragma unroll
-        for (int j = 0; j < SPT; ++j) {
-            xs[j] = CUDART_NAN_F;
-            if (j < nmine) xs[j] = __ldg(p0 + j * step);
-        }
+    for (int j = 0; j < kSpSmpLoads; ++j) {
+        const int i = tid + j * kSpSmpThreads;   // index into the sample
+        xs[j] = make_float4(CUDART_NAN_F, CUDART_NAN_F, CUDART_NAN_F, CUDART_NAN_F);
+        if (i < g.s) xs[j] = __ldg(reinterpret_cast<const float4 *>(row + (size_t)((i >> 2) * period + first + (i & 3)) * M) + q);
     }
     float xpre = 0.0f;
-    if (tid < 32) xpre = __ldg(row + (size_t)min(R - 1, (int)(((long long)(2 * lane + 1) * R) >> 6)) * M + m);
-    for (int i = tid; i < kSpBins; i += G) sh.hist[i] = 0;
-    if (tid == 0) {
+    if (warp < 4) xpre = __ldg(row + (size_t)min(R - 1, (int)(((long long)(2 * lane + 1) * R) >> 6)) * M + 4 * q + warp);
+    for (int i = tid; i < 4 * kSpBins; i += kSpSmpThreads) (&sh.hist[0][0])[i] = 0;
+    if (tid < 4) {
+        SpCol &col = sc.col[(size_t)t * M + 4 * q + tid];
         col.cnt = 0;
         col.n = 0;
-        if (m == 0) { sc.fail[t] = 0; sc.namb[t] = 0; }
     }
-    if (tid < 32) {
+    if (tid == 0 && q == 0) { sc.fail[t] = 0; sc.namb[t] = 0; }
+    if (tid == 0) {
+        const int mid = g.s / 2, q1 = g.s / 4, q3 = (3 * g.s) / 4;
+        const int tk[6] = {mid - g.delta, mid + g.delta, q1 - g.delta_q, q1 + g.delta_q, q3 - g.delta_q, q3 + g.delta_q};
+#pragma unroll
+        for (int i = 0; i < 6; ++i) sh.tk[i] = (uint32_t)min(max(tk[i], 0), g.s - 1);
+    }
+    if (tid < 24) sh.tb[tid / 6][tid % 6] = 0xFFFFFFFFu;
+    if (warp < 4) {
         const uint32_t key = sp_warp_sort(f2key(xpre), lane);
         const float c50 = key2f(__shfl_sync(0xFFFFFFFFu, key, 16));
         const float c25 = key2f(__shfl_sync(0xFFFFFFFFu, key, 8)), c75 = key2f(__shfl_sync(0xFFFFFFFFu, key, 23));
@@ -164,83 +180,83 @@ __global__ void __launch_bounds__(kSpSelThreads) xsplit_sample_kernel(const Xran
             const float sig = (c75 - c25) / 1.35f;
             const float inv_bw = 64.0f / sig;     // 2048 bins over +-16 sigma
             const float off = (float)(1024.0 - (double)c50 * (double)inv_bw);
-            sh.inv_bw = inv_bw;
-            sh.off = off;
-            sh.sample_ok = (sig > 0.0f) && (inv_bw < kFltMax) && (fabsf(off) < kFltMax);
-            const int mid = g.s / 2, q1 = g.s / 4, q3 = (3 * g.s) / 4;
-            const int tk[6] = {mid - g.delta, mid + g.delta, q1 - g.delta_q, q1 + g.delta_q, q3 - g.delta_q, q3 + g.delta_q};
-#pragma unroll
-            for (int i = 0; i < 6; ++i) { sh.tk[i] = (uint32_t)min(max(tk[i], 0), g.s - 1); sh.tb[i] = 0xFFFFFFFFu; }
+            sh.inv_bw[warp] = inv_bw;
+            sh.off[warp] = off;
+            sh.ok[warp] = (sig > 0.0f) && (inv_bw < kFltMax) && (fabsf(off) < kFltMax);
         }
     }
     __syncthreads();
-    const bool sample_ok = sh.sample_ok != 0;
-    if (sample_ok) {
-        const float inv_bw = sh.inv_bw, off = sh.off;
-        // slots without a sample hold NaN and are skipped
+    {
+        float ib[4], of[4];
 #pragma unroll
-        for (int j = 0; j < SPT; ++j) {
-            int b = __float2int_rd(__fmaf_rn(xs[j], inv_bw, off));
-            b = min(max(b, 0), kSpSBins - 1);
-            if (xs[j] == xs[j]) atomicAdd(&sh.hist[b >> 1], (b & 1) ? 0x10000u : 1u);
-        }
-    }
-    __syncthreads();
-    if (sample_ok) {
-        // bins of the six sample ranks: scan of the 2048 bin counts, WPT words (2 bins each) per thread
-        constexpr int WPT = kSpBins / G;
-        uint32_t w[WPT], sum = 0;
+        for (int c = 0; c < 4; ++c) { ib[c] = sh.ok[c] ? sh.inv_bw[c] : 0.0f; of[c] = sh.ok[c] ? sh.off[c] : 0.0f; }
 #pragma unroll
-        for (int i = 0; i < WPT; ++i) { w[i] = sh.hist[tid * WPT + i]; sum += (w[i] & 0xFFFFu) + (w[i] >> 16); }
-        uint32_t incl = sum;
-        const int gw = tid >> 5;
+        for (int j = 0; j < kSpSmpLoads; ++j) {
+            if (tid + j * kSpSmpThreads < g.s) {
+                const float v[4] = {xs[j].x, xs[j].y, xs[j].z, xs[j].w};
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) { const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, incl, d); if (lane >= d) incl += u; }
-        if (lane == 31) sh.warp_tot[gw] = incl;
-        __syncthreads();
-        uint32_t offw = 0;
-        for (int ww = 0; ww < gw; ++ww) offw += sh.warp_tot[ww];
-        const uint32_t excl = offw + incl - sum;
-#pragma unroll
-        for (int i6 = 0; i6 < 6; ++i6) {
-            const uint32_t k = sh.tk[i6];
-            if (k >= excl && k < excl + sum) {
-                uint32_t run = excl;
-#pragma unroll
-                for (int i = 0; i < WPT; ++i) {
-                    const uint32_t c0 = w[i] & 0xFFFFu, c1 = w[i] >> 16;
-                    if (k >= run && k < run + c0) sh.tb[i6] = (uint32_t)(2 * (tid * WPT + i));
-                    run += c0;
-                    if (k >= run && k < run + c1) sh.tb[i6] = (uint32_t)(2 * (tid * WPT + i) + 1);
-                    run += c1;
+                for (int c = 0; c < 4; ++c) {
+                    int b = __float2int_rd(__fmaf_rn(v[c], ib[c], of[c]));
+                    b = min(max(b, 0), kSpSBins - 1);
+                    atomicAdd(&sh.hist[c][b >> 1], (b & 1) ? 0x10000u : 1u);
                 }
             }
         }
     }
     __syncthreads();
-    if (tid == 0) {
-        bool ok = sample_ok;
+    // bins of the six sample ranks: 64 threads per metric scan its 2048 bin counts, WPT words (2 bins each) per thread
+    const int c = tid / kSpSmpG, gt = tid % kSpSmpG, gw = gt >> 5;
+    constexpr int WPT = kSpBins / kSpSmpG;
+    uint32_t w[WPT], sum = 0;
 #pragma unroll
-        for (int i = 0; i < 6; ++i) ok = ok && sh.tb[i] != 0xFFFFFFFFu;
+    for (int i = 0; i < WPT; ++i) { w[i] = sh.hist[c][gt * WPT + i]; sum += (w[i] & 0xFFFFu) + (w[i] >> 16); }
+    uint32_t incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, incl, d); if (lane >= d) incl += u; }
+    if (lane == 31) sh.warp_tot[c][gw] = incl;
+    __syncthreads();
+    const uint32_t excl = (gw ? sh.warp_tot[c][0] : 0u) + incl - sum;
+#pragma unroll 1
+    for (int i6 = 0; i6 < 6; ++i6) {
+        const uint32_t k = sh.tk[i6];
+        if (k >= excl && k < excl + sum) {
+            uint32_t run = excl;
+#pragma unroll
+            for (int i = 0; i < WPT; ++i) {
+                const uint32_t c0 = w[i] & 0xFFFFu, c1 = w[i] >> 16;
+                if (k >= run && k < run + c0) sh.tb[c][i6] = (uint32_t)(2 * (gt * WPT + i));
+                run += c0;
+                if (k >= run && k < run + c1) sh.tb[c][i6] = (uint32_t)(2 * (gt * WPT + i) + 1);
+                run += c1;
+            }
+        }
+    }
+    __syncthreads();
+    if (tid < 4) {
+        const int cc = tid;
+        SpCol &col = sc.col[(size_t)t * M + 4 * q + cc];
+        bool ok = sh.ok[cc] != 0;
+#pragma unroll
+        for (int i = 0; i < 6; ++i) ok = ok && sh.tb[cc][i] != 0xFFFFFFFFu;
         float lo = 0.0f, hi = 0.0f, dlo = 0.0f, dhi = 0.0f;
         if (ok) {
             // value at the lower edge of bin b under the map x -> x * inv_bw + off
-            const double inv = 1.0 / (double)sh.inv_bw, offd = (double)sh.off;
+            const double inv = 1.0 / (double)sh.inv_bw[cc], offd = (double)sh.off[cc];
             auto edge = [&](uint32_t b) -> float {
                 if (b == 0) return -kFltMax;
                 if (b >= (uint32_t)kSpSBins) return kFltMax;
                 const double e = ((double)b - offd) * inv;
                 return (float)fmin(fmax(e, -(double)kFltMax), (double)kFltMax);
             };
-            lo = fdown(edge(sh.tb[0]));
-            hi = fup(edge(sh.tb[1] + 1));
+            lo = fdown(edge(sh.tb[cc][0]));
+            hi = fup(edge(sh.tb[cc][1] + 1));
             if (lo < -kFltMax) lo = -kFltMax;
             if (hi > kFltMax) hi = kFltMax;
             // The MAD is the half-width d at which [med - d, med + d] holds half of the column: the
             // span between the quartiles' outer (inner) neighbours holds more (less) than half with
             // high probability, and for a column roughly symmetric about its median the half-lengths
             // of those spans bracket d.  (A miss is caught by the counts.)
-            const float a_lo = edge(sh.tb[2]), a_hi = edge(sh.tb[3] + 1), b_lo = edge(sh.tb[4]), b_hi = edge(sh.tb[5] + 1);
+            const float a_lo = edge(sh.tb[cc][2]), a_hi = edge(sh.tb[cc][3] + 1), b_lo = edge(sh.tb[cc][4]), b_hi = edge(sh.tb[cc][5] + 1);
             const float d0 = 0.5f * (b_lo - a_hi), d1 = 0.5f * (b_hi - a_lo);
             dlo = d0 > 0.0f ? fdown(d0) : 0.0f;
             dhi = (d1 >= 0.0f && d1 < kFltMax) ? fup(d1) : kFltMax;
@@ -373,7 +389,7 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
                     for (int c = 0; c < 4; ++c) v[j][c] = MODE == 0 ? CUDART_NAN_F : __fmul_rn(sg[c], -nsm[c]);   // MODE 1: x = med
                 }
         }
-        uint32_t packed = 0;
+        uint32_t packed = 0, slowmask = 0;
 #pragma unroll
         for (int j = 0; j < kSpU; ++j) {
             if (MODE == 1) {
@@ -388,12 +404,7 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
                     v[j][c] = d;
                     slow |= !(d <= rlo[c]);
                 }
-                if (slow) {
-                    const int r = base + j * LPI + rl;
-                    if (!guard || r < r1)
-                        sp_slow_row<NQ>(row, r, q, sh, sc.namb + t, sc.amb + (size_t)t * kSpAmb, maskrow,
-                                        a.check_finite ? a.status : nullptr);
-                }
+                if (slow) slowmask |= 1u << j;   // handled at the end of the batch, where little else is live
                 if (guard && base + j * LPI + rl >= r1) {
 #pragma unroll
                     for (int c = 0; c < 4; ++c) v[j][c] = CUDART_NAN_F;
@@ -429,6 +440,15 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
         for (int j = 0; j < kSpU; ++j)
 #pragma unroll
             for (int c = 0; c < 4; ++c) sp_cell_keep(v[j][c], lo[c], hi[c], addr[c]);
+        if (MODE == 1 && slowmask) {
+#pragma unroll 1
+            for (int j = 0; j < kSpU; ++j) {
+                const int r = base + j * LPI + rl;
+                if (((slowmask >> j) & 1u) && r < r1)
+                    sp_slow_row<NQ>(row, r, q, sh, sc.namb + t, sc.amb + (size_t)t * kSpAmb, maskrow,
+                                    a.check_finite ? a.status : nullptr);
+            }
+        }
     };
     const int span = LPI * kSpU;
     int base = r0;
@@ -674,7 +694,7 @@ SpGeom split_geometry(int R) {
     g.slice = ((R + g.chunks - 1) / g.chunks + 15) / 16 * 16;
     g.stride = (R + kSpSample - 1) / kSpSample;
     if (g.stride < 1) g.stride = 1;
-    g.s = (R - (g.stride >> 1) + g.stride - 1) / g.stride;
+    g.s = 4 * (R / (4 * g.stride));
     const double sq = sqrt((double)g.s);
     // half-widths in sample ranks: 5.5 standard deviations of the sampled median's rank; the quartile
     // intervals bracket a count, the sum of two quartile ranks (sd ~ 0.61 sqrt(s)), at 5 standard deviations
@@ -748,7 +768,7 @@ cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S,
         cudaEventRecord(ev0, st);
     }
     const dim3 gcol(M, S), gsw(g.chunks, S);
-    xsplit_sample_kernel<<<gcol, kSpSelThreads, 0, st>>>(a, g, sc, reasons);
+    xsplit_sample_kernel<<<dim3(M / 4, S), kSpSmpThreads, 0, st>>>(a, g, sc, reasons);
     if (M == 8) xsplit_sweep_kernel<2, 0><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
     else xsplit_sweep_kernel<1, 0><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
     xsplit_select_kernel<0><<<gcol, kSpSelThreads, 0, st>>>(a, p, g, sc, reasons);
