@@ -42,6 +42,7 @@ constexpr int kSpSBins = 2048;      // sample histogram bins (16-bit counters, t
 constexpr int kSpBins = 1024;       // selection histogram bins
 constexpr int kSpSelThreads = 128;  // sample / select CTA
 constexpr int kSpJmax = 20;         // kept elements per thread the register selection can hold
+constexpr int kSpSegs = 4;          // sweep CTAs per step the selection can gather from
 constexpr int kSpMaxM = 8;
 constexpr float kFltMax = 3.402823466e+38f;
 
@@ -49,7 +50,6 @@ struct SpGeom {
     int chunks;     // sweep CTAs per step
     int slice;      // ranks per sweep CTA (a multiple of 16)
     int cap;        // kept elements per metric and sweep CTA (shared memory)
-    int gcap;       // kept elements per column (global scratch)
     int stride;     // one run of four consecutive ranks is sampled out of every 4 * stride
     int s;          // number of sampled ranks
     int delta;      // half-width of the median interval in sample ranks
@@ -61,8 +61,7 @@ struct SpCol {
     float lo, hi, dlo, dhi;   // intervals of the median and of the MAD
     float med, rlo, rhi, rhs; // median; range of the exceedance threshold over [dlo, dhi]; exact threshold
     uint32_t cnt;             // elements below the current interval
-    uint32_t n;               // elements kept
-    uint32_t pad[2];
+    uint32_t pad[3];
 };
 
 struct SpScratch {
@@ -70,17 +69,22 @@ struct SpScratch {
     uint32_t *fail;   // [S] the step goes to the direct path
     uint32_t *namb;   // [S] deferred exceedance decisions
     uint32_t *amb;    // [S][kSpAmb] (rank << 5 | metric)
-    uint32_t *list;   // [S][M][gcap] kept elements (raw bits)
+    uint32_t *nseg;   // [S][M][chunks] kept elements of each sweep CTA
+    uint32_t *list;   // [S][M][chunks][cap] kept elements (raw bits), one segment per sweep CTA
 };
 
 // ---- per-element operations of the sweeps, written out so that each is a fixed handful of
 // instructions (compare, predicated add / predicated store) ---------------------------------
-// cnt += (x < lo); packed += INC if lo <= x <= hi (NaN is neither).
+// cnt += !(x >= lo); packed += INC if lo <= x <= hi.
+// Written without predicates (comparison results as 0 / -1 words): sixteen of these in a row
+// would otherwise have the compiler shuffle predicates through registers.
 template <uint32_t INC>
 __device__ __forceinline__ void sp_cell_count(const float x, const float lo, const float hi, uint32_t &cnt, uint32_t &packed) {
-    asm("{\n\t.reg .pred p, q;\n\tsetp.lt.f32 p, %2, %3;\n\tsetp.le.and.f32 q, %2, %4, !p;\n\t@p add.u32 %0, %0, 1;\n\t@q add.u32 %1, %1, %5;\n\t}"
-        : "+r"(cnt), "+r"(packed)
-        : "f"(x), "f"(lo), "f"(hi), "n"(INC));
+    uint32_t ge, le;
+    asm("set.ge.u32.f32 %0, %1, %2;" : "=r"(ge) : "f"(x), "f"(lo));
+    asm("set.le.u32.f32 %0, %1, %2;" : "=r"(le) : "f"(x), "f"(hi));
+    cnt += 1u + ge;               // + 1 unless x >= lo
+    packed += (ge & le) & INC;
 }
 // if (lo <= x <= hi) { shared[addr] = x; addr += 4; }
 __device__ __forceinline__ void sp_cell_keep(const float x, const float lo, const float hi, uint32_t &addr) {
@@ -162,7 +166,6 @@ __global__ void __launch_bounds__(kSpSmpThreads) xsplit_sample_kernel(const Xran
     if (tid < 4) {
         SpCol &col = sc.col[(size_t)t * M + 4 * q + tid];
         col.cnt = 0;
-        col.n = 0;
     }
     if (tid == 0 && q == 0) { sc.fail[t] = 0; sc.namb[t] = 0; }
     if (tid == 0) {
@@ -275,7 +278,6 @@ struct SpSweepShared {
     float lo[kSpMaxM], hi[kSpMaxM], med[kSpMaxM], rlo[kSpMaxM], rhi[kSpMaxM], sgn[kSpMaxM];
     uint32_t cnt[kSpMaxM];   // elements below the interval, this CTA
     uint32_t n32[4];         // kept counts, two 16-bit fields per word (metric m: word m / 2)
-    uint32_t gbase[kSpMaxM]; // where this CTA's kept elements go in the step's global lists
     uint32_t fail;
 };
 
@@ -326,10 +328,6 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
     extern __shared__ __align__(16) uint32_t slist[];   // [M][cap + kSpSlack]
     __shared__ SpSweepShared sh;
     const int chunk = blockIdx.x, t = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
-    // other CTAs of the step may raise the flag while this one runs: one read, the same answer for all threads
-    if (tid == 0) sh.fail = sc.fail[t];
-    __syncthreads();
-    if (sh.fail) return;
     const int R = a.R;
     const int slot = (int)(((long long)a.first_slot + t) % a.capacity);
     const float *row = a.base + (size_t)slot * a.row_stride;
@@ -338,6 +336,8 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
     SpCol *cols = sc.col + (size_t)t * M;
     const int cap = g.cap;
 
+    // other CTAs of the step may raise the flag while this one runs: one read, the same answer for all threads
+    if (tid == M) sh.fail = sc.fail[t];
     if (tid < M) {
         const SpCol cc = cols[tid];
         sh.lo[tid] = MODE == 0 ? cc.lo : cc.dlo;
@@ -348,9 +348,12 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
     }
     if (tid < 4) sh.n32[tid] = 0u;
     // this CTA's part of the exceedance row starts at zero; bits are OR-ed in
-    if (MODE == 1 && maskrow)
-        for (int i = r0 + 4 * tid; i < r1; i += 4 * kSpThreads) *reinterpret_cast<uint32_t *>(maskrow + i) = 0u;
     __syncthreads();
+    if (sh.fail) return;
+    if (MODE == 1 && maskrow) {
+        for (int i = r0 + 4 * tid; i < r1; i += 4 * kSpThreads) *reinterpret_cast<uint32_t *>(maskrow + i) = 0u;
+        __syncthreads();   // zeroed before any thread ORs a bit in
+    }
 
     const int q = tid & (NQ - 1), rl = tid / NQ;
     float lo[4], hi[4], sg[4], nsm[4], rlo[4];
@@ -462,21 +465,19 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
     }
     __syncthreads();
     // this CTA's counts and kept elements join the step's
+    // (every CTA has its own segment of the step's lists: plain stores, nothing to wait for)
     if (tid < M) {
         const uint32_t nl = (sh.n32[tid >> 1] >> (16 * (tid & 1))) & 0xFFFFu;
         if (sh.cnt[tid]) atomicAdd(&cols[tid].cnt, sh.cnt[tid]);
-        sh.gbase[tid] = atomicAdd(&cols[tid].n, nl);
+        sc.nseg[((size_t)t * M + tid) * g.chunks + chunk] = nl;
         if (nl > (uint32_t)cap) atomicOr(&sc.fail[t], 1u);
     }
-    __syncthreads();
 #pragma unroll 1
     for (int m = 0; m < M; ++m) {
         const uint32_t nl = min((sh.n32[m >> 1] >> (16 * (m & 1))) & 0xFFFFu, (uint32_t)cap);
-        const uint32_t gb = sh.gbase[m];
-        uint32_t *dst = sc.list + ((size_t)t * M + m) * g.gcap;
+        uint32_t *dst = sc.list + (((size_t)t * M + m) * g.chunks + chunk) * cap;
         const uint32_t *srcl = slist + (size_t)m * (cap + kSpSlack);
-        for (uint32_t i = tid; i < nl; i += kSpThreads)
-            if (gb + i < (uint32_t)g.gcap) dst[gb + i] = srcl[i];
+        for (uint32_t i = tid; i < nl; i += kSpThreads) dst[i] = srcl[i];
     }
 }
 
@@ -509,23 +510,25 @@ __device__ __forceinline__ void sp_find_bin(SpSelShared &sh, uint32_t k) {
 }
 
 // Keys of ranks k and (if want_next) k + 1 among the n kept elements of a column (raw float
-// bits in global scratch), all of whose keys lie in [base, base + width].  The elements are
-// fetched once into registers (JMAX per thread).  A 1024-bin histogram over the interval
+// bits in global scratch, one segment per sweep CTA), all of whose keys lie in [base, base +
+// width].  The elements are fetched once into registers (JMAX per thread).  A 1024-bin histogram over the interval
 // locates the bin of rank k; while that bin holds more than 32 keys it becomes the next,
 // narrower range; then the bin's keys are gathered and one warp ranks them.  The next order
 // statistic is the following gathered key or, if the bin ends there, the smallest key above it.
 template <int JMAX>
-__device__ bool sp_select_regs(const uint32_t *__restrict__ list, const uint32_t n, uint32_t k, bool want_next, uint32_t base,
-                               uint32_t width, SpSelShared &sh, uint32_t &v1, uint32_t &v2) {
-    constexpr int G = kSpSelThreads;
+__device__ bool sp_select_regs(const uint32_t *__restrict__ list, const int cap, const uint32_t (&nseg)[kSpSegs], uint32_t k,
+                               bool want_next, uint32_t base, uint32_t width, SpSelShared &sh, uint32_t &v1, uint32_t &v2) {
+    constexpr int G = kSpSelThreads, JS = JMAX / kSpSegs;   // registers per segment
     const int tid = threadIdx.x;
     uint32_t off[JMAX];   // key - base; 0xFFFFFFFF (beyond any width) where there is no element
 #pragma unroll
-    for (int j = 0; j < JMAX; ++j) {
-        const uint32_t i = (uint32_t)(tid + j * G);
-        off[j] = 0x7F800000u;   // bits of +inf: its key lies above every finite key
-        if (i < n) off[j] = list[i];
-    }
+    for (int sg = 0; sg < kSpSegs; ++sg)
+#pragma unroll
+        for (int j = 0; j < JS; ++j) {
+            const uint32_t i = (uint32_t)(tid + j * G);
+            off[sg * JS + j] = 0x7F800000u;   // bits of +inf: its key lies above every finite key
+            if (i < nseg[sg]) off[sg * JS + j] = list[(size_t)sg * cap + i];
+        }
 #pragma unroll
     for (int j = 0; j < JMAX; ++j) {
         const uint32_t key = key_of_bits(off[j]);
@@ -622,17 +625,26 @@ __global__ void __launch_bounds__(kSpSelThreads) xsplit_select_kernel(const Xran
     SpCol &col = sc.col[so + m];
     const bool even = (R & 1) == 0;
     const uint32_t k1 = (uint32_t)((R - 1) / 2), k2 = (uint32_t)(R / 2);
-    const uint32_t clt = col.cnt, n = col.n;
+    const uint32_t clt = col.cnt;
+    uint32_t nseg[kSpSegs], n = 0;
+    bool over = false;
+#pragma unroll
+    for (int sg = 0; sg < kSpSegs; ++sg) {
+        nseg[sg] = sg < g.chunks ? sc.nseg[(so + m) * g.chunks + sg] : 0u;
+        over |= nseg[sg] > (uint32_t)g.cap;
+        n += nseg[sg];
+    }
     const float flo = MODE == 0 ? col.lo : col.dlo, fhi = MODE == 0 ? col.hi : col.dhi;
     int why = -1;
-    if (n > (uint32_t)g.gcap || n > (uint32_t)(kSpJmax * kSpSelThreads)) why = kWhyCtaList;
+    if (over) why = kWhyCtaList;
     else if (clt > k1 || k2 >= clt + n) why = MODE == 0 ? kWhyMedianMiss : kWhyMadMiss;
     if (MODE == 1 && sc.namb[t] > (uint32_t)kSpAmb) why = kWhyAmbList;
     uint32_t v1 = 0, v2 = 0;
     if (why < 0) {
         const uint32_t base = f2key((MODE == 0 && flo == 0.0f) ? -0.0f : flo);
         const uint32_t width = f2key((MODE == 0 && fhi == 0.0f) ? 0.0f : fhi) - base;
-        if (!sp_select_regs<kSpJmax>(sc.list + (so + m) * g.gcap, n, k1 - clt, even, base, width, sh, v1, v2)) why = kWhySelect;
+        if (!sp_select_regs<kSpJmax>(sc.list + (so + m) * g.chunks * g.cap, g.cap, nseg, k1 - clt, even, base, width, sh, v1, v2))
+            why = kWhySelect;
     }
     if (tid == 0) {
         if (why < 0) {
@@ -645,7 +657,6 @@ __global__ void __launch_bounds__(kSpSelThreads) xsplit_select_kernel(const Xran
                 col.rlo = __fmul_rn(p.thrp[m], fmaxf(fmaxf(col.dlo, rel), p.floor_abs[m]));
                 col.rhi = __fmul_rn(p.thrp[m], fmaxf(fmaxf(col.dhi, rel), p.floor_abs[m]));
                 col.cnt = 0;   // the MAD sweep counts anew
-                col.n = 0;
             } else {
                 a.mad[so + m] = val;
                 if (a.mad_user) a.mad_user[so + m] = val;
@@ -705,9 +716,6 @@ SpGeom split_geometry(int R) {
     g.cap = (int)ceil(g.slice * f * 1.2) + 64;
     g.cap = (g.cap + 31) / 32 * 32;
     if (g.cap < 256) g.cap = 256;
-    g.gcap = (int)ceil((double)R * f * 1.1) + 64;
-    if (g.gcap > g.chunks * g.cap) g.gcap = g.chunks * g.cap;
-    g.gcap = (g.gcap + 31) / 32 * 32;
     return g;
 }
 
@@ -722,7 +730,8 @@ bool xrank_split_supported(int R, int M) {
     if (R < 4096 || (R & 3) != 0) return false;
     const SpGeom g = split_geometry(R);
     if (g.slice > 32768) return false;
-    if (g.gcap > kSpJmax * kSpSelThreads) return false;   // the register selection holds a whole column's kept elements
+    // the register selection holds a whole column's kept elements: kSpJmax / kSpSegs per thread and segment
+    if (g.chunks > kSpSegs || g.cap > (kSpJmax / kSpSegs) * kSpSelThreads) return false;
     return split_sweep_smem(g, M) <= 64 * 1024;
 }
 
@@ -732,7 +741,8 @@ size_t xrank_split_scratch_bytes(int R, int M, int S_max) {
     b += align256((size_t)S_max * M * sizeof(SpCol));
     b += align256((size_t)S_max * sizeof(uint32_t)) * 2;
     b += align256((size_t)S_max * kSpAmb * sizeof(uint32_t));
-    b += align256((size_t)S_max * M * g.gcap * sizeof(uint32_t));
+    b += align256((size_t)S_max * M * g.chunks * sizeof(uint32_t));
+    b += align256((size_t)S_max * M * g.chunks * g.cap * sizeof(uint32_t));
     return b;
 }
 
@@ -747,6 +757,7 @@ cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S,
     sc.fail = (uint32_t *)b;  b += align256((size_t)S * sizeof(uint32_t));
     sc.namb = (uint32_t *)b;  b += align256((size_t)S * sizeof(uint32_t));
     sc.amb = (uint32_t *)b;   b += align256((size_t)S * kSpAmb * sizeof(uint32_t));
+    sc.nseg = (uint32_t *)b;  b += align256((size_t)S * M * g.chunks * sizeof(uint32_t));
     sc.list = (uint32_t *)b;
     const size_t smem = split_sweep_smem(g, M);
     static bool attr_set_dev[64] = {};
