@@ -200,6 +200,24 @@ int guard_reset(guard_ctx *ctx, void *stream);
 /* Enables (default) or disables the internal fork/join stream described under Conventions. */
 int guard_set_overlap(guard_ctx *ctx, int on);
 
+/* Deferred evaluations (off by default).  While on, guard_score enqueues the evaluation on
+ * streams of the library's own, ordered after everything enqueued on `stream` so far, and
+ * `stream` does NOT wait for it: the evaluation (Section 4.2's peer comparison over the last
+ * window) then runs beside the next guard_ingest instead of in front of it.  The output
+ * buffers of that guard_score call are complete, in the order of a stream, only after that
+ * stream has passed the next guard_score, guard_join, guard_sync_status or guard_reset on
+ * this context; until then the caller must neither read nor reuse them.  At most one
+ * evaluation is pending.  The ring slots of the pending evaluation's window must not be
+ * overwritten: guard_ingest waits for the evaluation by itself when its block reuses them,
+ * and guard_ring_reserve refuses (GUARD_ERR_NOT_READY) to hand them out, since it cannot
+ * order the caller's writes; with capacity_steps >= W + block size neither ever happens.
+ * Results are identical to the default mode. */
+int guard_set_deferred(guard_ctx *ctx, int on);
+
+/* Makes `stream` wait for the pending deferred evaluation, if there is one (no host
+ * synchronisation). */
+int guard_join(guard_ctx *ctx, void *stream);
+
 /* Kernel timing for benchmarks: while enabled, guard_ingest records a pair of CUDA events on
  * the stream right around its main kernel (the fused cross-rank sweep; contexts whose sizes
  * take another path record nothing).  guard_profile_read waits for the recorded events, returns

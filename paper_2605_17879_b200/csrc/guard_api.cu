@@ -136,6 +136,35 @@ struct guard_ctx {
         }
         return true;
     }
+    // Deferred evaluations: guard_score enqueues the evaluation on internal streams and does not
+    // make the caller's stream wait for it, so that the evaluation's short, latency-bound tail runs
+    // beside the next guard_ingest.  At most one evaluation is pending; the next guard_score,
+    // guard_join, guard_sync_status, guard_reset and guard_destroy wait for it.
+    bool deferred = false;
+    bool pending = false;             // an evaluation has been enqueued whose end the caller's stream has not waited for
+    int pending_n = 0;                // its window length
+    cudaStream_t tail = nullptr;
+    cudaEvent_t ev_x = nullptr, ev_w = nullptr, ev_e = nullptr;
+    bool ensure_tail() {
+        if (tail) return true;
+        if (!ensure_side()) return false;
+        if (cudaStreamCreateWithFlags(&tail, cudaStreamNonBlocking) != cudaSuccess) { tail = nullptr; return false; }
+        if (cudaEventCreateWithFlags(&ev_x, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ev_w, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ev_e, cudaEventDisableTiming) != cudaSuccess) {
+            cudaStreamDestroy(tail);
+            tail = nullptr;
+            return false;
+        }
+        return true;
+    }
+    // Makes `st` wait for the pending evaluation, if any.
+    cudaError_t join(cudaStream_t st) {
+        if (!pending) return cudaSuccess;
+        cudaError_t e = cudaStreamWaitEvent(st, ev_e, 0);
+        if (e == cudaSuccess) pending = false;
+        return e;
+    }
     bool profiling = false;                                   // record events around the main ingest kernel
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof;    // recorded, not yet read
     char error[256];
@@ -274,6 +303,8 @@ int guard_ring_reserve(guard_ctx *c, int steps, float **d_slot) {
     if (!d_slot || steps < 1 || steps > c->C) return c->fail(GUARD_ERR_ARG, "steps must be in 1..capacity and d_slot non-NULL");
     const int slot = (int)(c->seen % c->C);
     if (slot + steps > c->C) return c->fail(GUARD_ERR_ARG, "reserved span would wrap around the ring (slot %d + %d > %d)", slot, steps, c->C);
+    if (c->pending && steps + c->pending_n > c->C)
+        return c->fail(GUARD_ERR_NOT_READY, "the reserved slots belong to the window of the deferred evaluation still pending: call guard_join first");
     *d_slot = c->ring() + (size_t)slot * c->R * c->M;
     return GUARD_OK;
 }
@@ -286,6 +317,10 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
     const size_t row = (size_t)c->R * c->M;
     const int slot = (int)(c->seen % c->C);
     const bool in_place = (d_block == c->ring() + (size_t)slot * row) && (slot + B <= c->C);
+    if (c->pending && B + c->pending_n > c->C) {   // this block's slots are read by the pending evaluation
+        cudaError_t e = c->join(st);
+        if (e != cudaSuccess) return c->cuda_fail(e, "join of the deferred evaluation");
+    }
     if (!in_place) {
         const int first = (slot + B <= c->C) ? B : (c->C - slot);
         cudaError_t e = cudaMemcpyAsync(c->ring() + (size_t)slot * row, d_block, (size_t)first * row * sizeof(float),
@@ -348,9 +383,32 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     // ring became complete, so that they overlap the cross-rank kernels of the preceding ingest;
     // the caller's stream waits for them before anything that uses them.
     cudaError_t e;
+    // a deferred evaluation still pending is complete, in the caller's stream order, from here on
+    const bool had_pending = c->pending;
+    e = c->join(st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "join of the deferred evaluation");
     const bool forked = c->overlap && c->fork_fresh && c->side;
     c->fork_fresh = false;
-    if (forked) {
+    const bool defer = c->deferred && c->ensure_tail();
+    cudaStream_t ts = st;   // stream of the evaluation's tail: fleet baseline, scores / flags, top-k
+    if (defer) {
+        // window medians on the internal stream (after the ring is complete and after the previous
+        // evaluation's tail, which still reads the medians they overwrite); the tail on a stream of
+        // its own after them and after this block's cross-rank kernels; the caller's stream waits
+        // for none of it
+        if (!forked) {
+            e = cudaEventRecord(c->ev_fork, st);
+            if (e != cudaSuccess) return c->cuda_fail(e, "event record");
+        }
+        e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
+        if (e == cudaSuccess && had_pending) e = cudaStreamWaitEvent(c->side, c->ev_e, 0);
+        if (e == cudaSuccess) e = launch_window_select(w, c->side);
+        if (e == cudaSuccess) e = cudaEventRecord(c->ev_w, c->side);
+        if (e == cudaSuccess) e = cudaEventRecord(c->ev_x, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_w, 0);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_x, 0);
+        ts = c->tail;
+    } else if (forked) {
         e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
         if (e == cudaSuccess) e = launch_window_select(w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_join, c->side);
@@ -372,7 +430,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     x.med_user = d_fleet_med;
     x.mad_user = d_fleet_mad;
     x.status = c->status();
-    e = c->xrank(x, 1, st);
+    e = c->xrank(x, 1, ts);
     if (e != cudaSuccess) return c->cuda_fail(e, "fleet baseline launch");
 
     ScoreArgs s{};
@@ -407,7 +465,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         t.ticket = c->ticket();
         t.idx = d_topk_idx;
         t.score = d_topk_score;
-        if (c->overlap && c->ensure_side()) {
+        if (!defer && c->overlap && c->ensure_side()) {
             e = cudaEventRecord(c->ev_fork, st);
             if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
             if (e == cudaSuccess) e = launch_topk(t, c->p, c->side);
@@ -417,7 +475,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
             c->launches += 1;
         }
     }
-    e = launch_score_flag(s, c->p, st);
+    e = launch_score_flag(s, c->p, ts);
     if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
     c->evals += 1;
     c->launches += 1 + window_launch_count(w);
@@ -425,9 +483,15 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         e = cudaStreamWaitEvent(st, c->ev_join, 0);
         if (e != cudaSuccess) return c->cuda_fail(e, "topk join");
     } else if (want_topk) {
-        e = launch_topk(t, c->p, st);
+        e = launch_topk(t, c->p, ts);
         if (e != cudaSuccess) return c->cuda_fail(e, "topk launch");
         c->launches += 1;
+    }
+    if (defer) {
+        e = cudaEventRecord(c->ev_e, c->tail);
+        if (e != cudaSuccess) return c->cuda_fail(e, "event record");
+        c->pending = true;
+        c->pending_n = n;
     }
     return GUARD_OK;
 }
@@ -515,7 +579,8 @@ int guard_sweep_qualify(const float *d_S, int nodes, int gpus_per_node, int reps
 int guard_sync_status(guard_ctx *c, void *stream) {
     if (!c) return GUARD_ERR_ARG;
     uint32_t s = 0;
-    cudaError_t e = cudaMemcpyAsync(&s, c->status(), sizeof(s), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    cudaError_t e = c->join((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&s, c->status(), sizeof(s), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "guard_sync_status");
     const int code = status_to_code(s);
@@ -525,7 +590,8 @@ int guard_sync_status(guard_ctx *c, void *stream) {
 
 int guard_reset(guard_ctx *c, void *stream) {
     if (!c) return GUARD_ERR_ARG;
-    cudaError_t e = cudaMemsetAsync(c->ws, 0, c->L.wmed, (cudaStream_t)stream);
+    cudaError_t e = c->join((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws, 0, c->L.wmed, (cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "cudaMemsetAsync");
     c->seen = 0;
     c->evals = 0;
@@ -581,6 +647,19 @@ int64_t guard_fallback_steps(guard_ctx *c, void *stream) {
     return (int64_t)n;
 }
 
+int guard_set_deferred(guard_ctx *c, int on) {
+    if (!c) return GUARD_ERR_ARG;
+    c->deferred = on != 0;
+    return GUARD_OK;
+}
+
+int guard_join(guard_ctx *c, void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    cudaError_t e = c->join((cudaStream_t)stream);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_join");
+    return GUARD_OK;
+}
+
 int guard_set_overlap(guard_ctx *c, int on) {
     if (!c) return GUARD_ERR_ARG;
     c->overlap = on != 0;
@@ -591,6 +670,13 @@ int guard_set_overlap(guard_ctx *c, int on) {
 void guard_destroy(guard_ctx *c) {
     if (c) {
         guard_profile_enable(c, 0);
+        if (c->tail) {
+            cudaStreamSynchronize(c->tail);
+            cudaStreamDestroy(c->tail);
+            cudaEventDestroy(c->ev_x);
+            cudaEventDestroy(c->ev_w);
+            cudaEventDestroy(c->ev_e);
+        }
         if (c->side) {
             cudaStreamDestroy(c->side);
             cudaEventDestroy(c->ev_fork);

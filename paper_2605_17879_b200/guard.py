@@ -79,6 +79,10 @@ def lib():
         L.guard_fallback_reasons.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.guard_set_overlap.restype = C.c_int
         L.guard_set_overlap.argtypes = [vp, C.c_int]
+        L.guard_set_deferred.restype = C.c_int
+        L.guard_set_deferred.argtypes = [vp, C.c_int]
+        L.guard_join.restype = C.c_int
+        L.guard_join.argtypes = [vp, vp]
         L.guard_profile_enable.restype = C.c_int
         L.guard_profile_enable.argtypes = [vp, C.c_int]
         L.guard_profile_read.restype = C.c_int
@@ -200,6 +204,16 @@ class Guard:
     def set_overlap(self, on: bool) -> None:
         """Window medians of an evaluation on an internal stream overlapping the preceding ingest."""
         self._check(lib().guard_set_overlap(self._h, 1 if on else 0))
+
+    def set_deferred(self, on: bool) -> None:
+        """Deferred evaluations: score() does not make the current stream wait for its results; they
+        are complete after the next score(), join(), sync_status() or reset()."""
+        self._check(lib().guard_set_deferred(self._h, 1 if on else 0))
+
+    def join(self) -> None:
+        """Makes the current stream wait for the pending deferred evaluation, if any."""
+        with torch.cuda.device(self.device):
+            self._check(lib().guard_join(self._h, _stream()))
 
     def profile_enable(self, on: bool = True) -> None:
         self._check(lib().guard_profile_enable(self._h, 1 if on else 0))

@@ -166,6 +166,53 @@ def test_overlap_stream_on_and_off_agree():
             assert_bit_equal(res[1][i][key], ref[key], key)
 
 
+def test_deferred_evaluations_match_oracle():
+    """Deferred mode: score() leaves the evaluation running beside the next ingest; every
+    evaluation's outputs, read after the next score() / join(), match the oracle, in place and
+    copied, including a ring that forces the library to join by itself (capacity < W + block)."""
+    from paper_2605_17879_b200 import guard
+    R, M, W, B, T = 4500, 8, 20, 20, 120
+    X, dirs = _rand_fleet(T, R, M, seed=33)
+    Xd = torch.from_numpy(X).cuda()
+    o = go.Oracle(R, M, W, 10, 8, dir=dirs)
+    refs = []
+    for t in range(0, T, B):
+        o.ingest(X[t:t + B])
+        refs.append(o.score())
+    for cap, in_place in ((60, True), (40, False), (30, False)):
+        g = guard.Guard(R, M, W, 10, dir=dirs, capacity=cap, topk=8)
+        g.set_deferred(True)
+        bufs = [g.alloc_outputs() for _ in range(2)]
+        got = []
+        for i, t in enumerate(range(0, T, B)):
+            if in_place:
+                slot = g.ring_reserve(B)
+                slot.copy_(Xd[t:t + B])
+                g.ingest(slot)
+            else:
+                g.ingest(Xd[t:t + B])
+            g.score(bufs[i % 2])                      # also completes the evaluation before it
+            if i > 0:
+                torch.cuda.current_stream().synchronize()
+                got.append({k: to_np(v).copy() for k, v in bufs[(i - 1) % 2].items()})
+        g.join()
+        g.sync_status()
+        got.append({k: to_np(v).copy() for k, v in bufs[(len(refs) - 1) % 2].items()})
+        g.close()
+        for i, ref in enumerate(refs):
+            compare_score({k: torch.from_numpy(v) for k, v in got[i].items()}, ref, "cap=%d eval %d" % (cap, i))
+    # a ring too small for the caller to write the next block in place while an evaluation is pending
+    g = guard.Guard(R, M, W, 10, dir=dirs, capacity=30, topk=8)
+    g.set_deferred(True)
+    g.ingest(Xd[:B])
+    g.score()
+    with pytest.raises(guard.GuardError):
+        g.ring_reserve(B)
+    g.join()
+    g.ring_reserve(10)
+    g.close()
+
+
 def test_long_window_paths():
     # windows too long for the warp-per-series path: 128-, 64- and 32-column staged tiles, and the
     # global-memory fallback
