@@ -17,7 +17,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wlist, xr_big, mask, ring, total;
+    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, wlist, xr_big, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_fused;   // the single-launch fused cross-rank path applies
     int xr_cluster; // the cluster-per-step cross-rank path applies
@@ -41,6 +41,7 @@ Layout make_layout(int R, int M, int C, int K) {
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
     L.wspread = off;   off = align_up(off + (size_t)R * M * sizeof(float));
+    L.wcentre = off;   off = align_up(off + (size_t)R * M * sizeof(float));
     L.wlist = off;     off = align_up(off + (size_t)R * M * sizeof(uint32_t));
     L.xr_big = off;    off = align_up(off + (L.xr_split ? xrank_split_scratch_bytes(R, M, C < kSplitMaxSteps ? C : kSplitMaxSteps)
                                              : L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps)
@@ -376,6 +377,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     w.wmed_user = d_wmed;
     w.use_hint = c->evals > 0 ? 1 : 0;
     w.spread = (float *)(c->ws + c->L.wspread);
+    w.centre = (float *)(c->ws + c->L.wcentre);
     w.fb_list = (uint32_t *)(c->ws + c->L.wlist);
     w.fb_count = c->status() + 8;
     w.status = c->status();
@@ -465,8 +467,8 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         t.ticket = c->ticket();
         t.idx = d_topk_idx;
         t.score = d_topk_score;
-        if (!defer && c->overlap && c->ensure_side()) {
-            e = cudaEventRecord(c->ev_fork, st);
+        if (c->overlap && c->ensure_side()) {
+            e = cudaEventRecord(c->ev_fork, ts);
             if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
             if (e == cudaSuccess) e = launch_topk(t, c->p, c->side);
             if (e == cudaSuccess) e = cudaEventRecord(c->ev_join, c->side);
@@ -480,7 +482,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     c->evals += 1;
     c->launches += 1 + window_launch_count(w);
     if (topk_forked) {
-        e = cudaStreamWaitEvent(st, c->ev_join, 0);
+        e = cudaStreamWaitEvent(ts, c->ev_join, 0);
         if (e != cudaSuccess) return c->cuda_fail(e, "topk join");
     } else if (want_topk) {
         e = launch_topk(t, c->p, ts);

@@ -86,6 +86,7 @@ struct WindowArgs {
     int use_hint;           // wmed holds the previous evaluation's medians: use them as first pivots
     float *wmed_user;       // or NULL
     float *spread;          // [series] tuned half-width of the bracket path's interval (state), or NULL
+    float *centre;          // [series] smoothed median: the centre of the thread path's interval (state), or NULL
     uint32_t *fb_list;      // [series] series the bracket path hands to the list kernel, or NULL
     uint32_t *fb_count;     // their number
     uint32_t *status;

@@ -7,6 +7,10 @@
 #include "colselect.cuh"
 #include "kernels.h"
 
+#ifndef GUARD_WIN_THREAD
+#define GUARD_WIN_THREAD 1
+#endif
+
 namespace guard {
 
 namespace {
@@ -246,7 +250,7 @@ __device__ __forceinline__ float warp_spread_guess(const uint32_t (&kv)[VPL], co
         if (kv[i] != 0xFFFFFFFFu) s += fabsf(key2f(kv[i]) - med);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-    return 0.45f * s / (float)n;
+    return (GUARD_WIN_THREAD ? 0.36f : 0.45f) * s / (float)n;
 }
 
 template <int VPL>
@@ -326,6 +330,7 @@ __global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a
                 a.wmed[series] = med;
                 if (a.wmed_user) a.wmed_user[series] = med;
                 if (a.spread) a.spread[series] = h0;
+                if (a.centre) a.centre[series] = med;
             }
         }
         __syncthreads();   // every warp is done with this buffer before it is refilled
@@ -554,6 +559,224 @@ cudaError_t launch_bracket_path(const WindowArgs &a, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------
+// Thread path: the interval idea without staging.  One thread per series reads its window
+// straight from the ring (a warp reads 32 adjacent series of a row: one fully used 128-byte
+// line per load, eight rows in flight per thread), counts the values below the interval and
+// keeps those inside it, as raw bits, in its own shared-memory column.  No thread ever waits
+// for another one: there is no barrier in the kernel, CTAs are four warps, and with 60 kept
+// slots per thread seven CTAs share an SM.  The interval is centred on a smoothed median (a
+// single window's median carries its own sampling noise, which would add to the next one's).
+//
+// Selection among the kept keys runs the same instruction stream in every lane: the column
+// is turned into order-preserving keys once (128-bit shared-memory accesses; a column is 60
+// words, 4 x an odd number, so the lanes' quads fall on different banks), then counting
+// passes (keys below a pivot interpolated between the ends of a shrinking key bracket, every
+// third pass a bisection) run until t - 1, t or t + 1 keys lie below the pivot: the two
+// largest keys below it and the two smallest not below it then include ranks t - 1 and t.
+// If the bracket shrinks to one key, that key holds both ranks (ties).
+// A series whose interval missed, overflowed or did not converge is finished by its whole
+// warp: the lanes fetch the window (L2 hits), sort in registers and run the warp selection.
+// ---------------------------------------------------------------------------------------
+constexpr int kThCols = 128;     // series per CTA = threads per CTA
+constexpr int kThSlots = 60;     // kept keys per series
+constexpr int kThTarget = 42;    // number of keys the interval is tuned to catch
+constexpr int kThRows = 8;       // rows in flight per thread
+constexpr int kThMaxPasses = 12;
+constexpr float kThSmooth = 0.3f;   // weight of the newest median in the interval's centre
+
+// cnt += (x < lo); if (lo <= x <= hi) { if (addr < lim) shared[addr] = x; addr += 4; }
+__device__ __forceinline__ void th_cell(const float x, const float lo, const float hi, const uint32_t lim, uint32_t &cnt,
+                                        uint32_t &addr) {
+    asm volatile(
+        "{\n\t.reg .pred p, q, r;\n\t"
+        "setp.lt.f32 p, %2, %3;\n\t"
+        "setp.le.and.f32 q, %2, %4, !p;\n\t"
+        "setp.lt.and.u32 r, %1, %5, q;\n\t"
+        "@p add.u32 %0, %0, 1;\n\t"
+        "@r st.shared.f32 [%1], %2;\n\t"
+        "@q add.u32 %1, %1, 4;\n\t}"
+        : "+r"(cnt), "+r"(addr)
+        : "f"(x), "f"(lo), "f"(hi), "r"(lim)
+        : "memory");
+}
+__device__ __forceinline__ uint4 th_lds4(const uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void th_sts4(const uint32_t addr, const uint4 v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+template <int VPL>
+__global__ void __launch_bounds__(kThCols, 7) window_thread_kernel(const WindowArgs a) {
+    extern __shared__ __align__(16) uint32_t tkept[];   // [kThCols][kThSlots]
+    const int tid = threadIdx.x, lane = lane_id();
+    const int n = a.n;
+    const int c = blockIdx.x * kThCols + tid;
+    const bool active = c < a.series;
+    const int cc = active ? c : a.series - 1;           // idle lanes of the last CTA read a valid column
+    const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;
+    const int n1 = min(n, a.capacity - first);          // rows before the ring wraps
+
+    const float hint = a.centre[cc], h = a.spread[cc];
+    const bool usable = active && (h > 0.0f) && (h < 3.0e38f) && (fabsf(hint) < 3.0e38f);
+    // Float compares agree with the key order as long as an end that is zero admits both zeros
+    // (-0 as lower end, +0 as upper end).  An unusable interval keeps and counts nothing.
+    float flo = hint - h, fhi = hint + h;
+    if (flo == 0.0f) flo = -0.0f;
+    if (fhi == 0.0f) fhi = 0.0f;
+    if (!usable) { flo = CUDART_INF_F; fhi = -CUDART_INF_F; }
+    const uint32_t klo = usable ? f2key(flo) : 0xFFFFFFFFu, khi = usable ? f2key(fhi) : 0u;
+
+    const uint32_t kbase = smem_u32(tkept + tid * kThSlots), klim = kbase + (uint32_t)(kThSlots * 4);
+    uint32_t kaddr = kbase, clt = 0;
+    auto stream = [&](const float *__restrict__ p, const int rows) {
+        int r = 0;
+        for (; r + kThRows <= rows; r += kThRows) {
+            float x[kThRows];
+#pragma unroll
+            for (int u = 0; u < kThRows; ++u) x[u] = __ldg(p + (size_t)(r + u) * a.row_stride);
+#pragma unroll
+            for (int u = 0; u < kThRows; ++u) th_cell(x[u], flo, fhi, klim, clt, kaddr);
+        }
+        for (; r < rows; ++r) th_cell(__ldg(p + (size_t)r * a.row_stride), flo, fhi, klim, clt, kaddr);
+    };
+    stream(a.ring + (size_t)first * a.row_stride + cc, n1);
+    stream(a.ring + cc, n - n1);
+
+    const bool even = !(n & 1);
+    const int k1 = (n - 1) >> 1, k2 = n >> 1;
+    const int nk = (int)((kaddr - kbase) >> 2);
+    bool ok = usable && (int)clt <= k1 && k2 < (int)clt + nk && nk <= kThSlots;
+    const int t = k2 - (int)clt;     // rank of the upper middle among the kept keys (t >= 1 when n is even)
+    float med = 0.0f;
+    // ---- selection among the kept keys: the same instruction stream in every lane ---------------
+    const int nkmax = (int)__reduce_max_sync(0xFFFFFFFFu, ok ? (uint32_t)nk : 0u);
+    if (nkmax > 0) {
+        const int nkr = (nkmax + 3) & ~3;   // <= kThSlots (a multiple of 4)
+        for (int j = 0; j < nkr; j += 4) {  // raw bits -> keys; slots without a key compare above everything
+            uint4 v = th_lds4(kbase + 4u * j);
+            v.x = (ok && j + 0 < nk) ? key_of_bits(v.x) : 0xFFFFFFFFu;
+            v.y = (ok && j + 1 < nk) ? key_of_bits(v.y) : 0xFFFFFFFFu;
+            v.z = (ok && j + 2 < nk) ? key_of_bits(v.z) : 0xFFFFFFFFu;
+            v.w = (ok && j + 3 < nk) ? key_of_bits(v.w) : 0xFFFFFFFFu;
+            th_sts4(kbase + 4u * j, v);
+        }
+        // The pivot moves inside a key bracket (pl, ph) with below(pl) = al <= t - 2 and
+        // below(ph) = ah >= t + 2.
+        uint32_t pl = klo, ph = khi + 1u, pv = klo;
+        int al = 0, ah = nk, bsave = 0;
+        int done = 0;                 // 1: pv has bsave in {t - 1, t, t + 1} keys below it, 2: both ranks equal pl
+        if (!ok || t <= 1) { done = 1; pv = klo; bsave = 0; }
+        else if (t >= nk - 1) { done = 1; pv = khi + 1u; bsave = nk; }
+        for (int pass = 0; pass < kThMaxPasses; ++pass) {
+            if (__all_sync(0xFFFFFFFFu, done != 0)) break;
+            if (!done) {
+                if (ph - pl < 2u) {
+                    done = 2;
+                } else if (pass % 3 == 2) {
+                    pv = pl + ((ph - pl) >> 1);
+                } else {   // aim between the ends in proportion to the missing count
+                    const float fr = (float)(t - al) / (float)(ah - al);
+                    pv = pl + (uint32_t)((float)(ph - pl) * fr);
+                    pv = pv <= pl ? pl + 1u : (pv >= ph ? ph - 1u : pv);
+                }
+            }
+            int below = 0;
+            for (int j = 0; j < nkr; j += 4) {
+                const uint4 v = th_lds4(kbase + 4u * j);
+                below += (v.x < pv) + (v.y < pv) + (v.z < pv) + (v.w < pv);
+            }
+            if (!done) {
+                if (below >= t - 1 && below <= t + 1) { done = 1; bsave = below; }
+                else if (below < t) { pl = pv; al = below; }
+                else { ph = pv; ah = below; }
+            }
+        }
+        if (ok && !done) {
+            if (ph - pl < 2u) done = 2; else ok = false;
+        }
+        // the two largest keys below the pivot (b1 >= b2), the two smallest keys not below it (u1 <= u2)
+        uint32_t b1 = 0u, b2 = 0u, u1 = 0xFFFFFFFFu, u2 = 0xFFFFFFFFu;
+        for (int j = 0; j < nkr; j += 4) {
+            const uint4 v4 = th_lds4(kbase + 4u * j);
+            const uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const bool lt = v[u] < pv;
+                const uint32_t lo_v = lt ? v[u] : 0u, hi_v = lt ? 0xFFFFFFFFu : v[u];   // neutral on the other side
+                b2 = max(b2, min(b1, lo_v));
+                b1 = max(b1, lo_v);
+                u2 = min(u2, max(u1, hi_v));
+                u1 = min(u1, hi_v);
+            }
+        }
+        uint32_t vb = b1, vu = u1;                       // bsave == t
+        if (bsave == t + 1) { vb = b2; vu = b1; }
+        if (bsave == t - 1) { vb = u1; vu = u2; }
+        if (done == 2) { vb = pl; vu = pl; }
+        if (ok) med = median_from_keys(even ? vb : vu, vu, even);
+    }
+    if (active && ok) {
+        a.wmed[c] = med;
+        if (a.wmed_user) a.wmed_user[c] = med;
+        // re-tune the half-width so that the interval catches about kThTarget keys next time
+        // (half of the way: one window's count is a noisy estimate of the density)
+        const float f = fminf(2.0f, fmaxf(0.5f, (float)kThTarget / (float)max(nk, 1)));
+        a.spread[c] = h * (0.5f + 0.5f * f);
+        a.centre[c] = hint + kThSmooth * (med - hint);
+    }
+    // ---- series the interval did not serve: the whole warp finishes them one by one ------------
+    unsigned todo = __ballot_sync(0xFFFFFFFFu, active && !ok);
+    // why (diagnostic): 0 no usable interval, 1 more keys than slots, 2 median below the interval,
+    // 3 above it, 4 selection did not converge
+    const int why = !usable ? 0 : (nk > kThSlots ? 1 : ((int)clt > k1 ? 2 : (k2 >= (int)clt + nk ? 3 : 4)));
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int series = __shfl_sync(0xFFFFFFFFu, c, src);
+        const int why_src = __shfl_sync(0xFFFFFFFFu, why, src);
+        uint32_t kv[VPL];
+        int nreal = 0;
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int row = lane + 32 * j;
+            kv[j] = 0xFFFFFFFFu;
+            if (row < n) {
+                int slot = first + row;
+                if (slot >= a.capacity) slot -= a.capacity;
+                kv[j] = f2key(__ldg(a.ring + (size_t)slot * a.row_stride + series));
+                ++nreal;
+            }
+        }
+        lane_sort<VPL>(kv);
+        float m2 = 0.0f;
+        const bool ok2 = warp_median<VPL>(kv, nreal, n, 0u, m2);
+        const float h0 = warp_spread_guess<VPL>(kv, n, m2);
+        if (lane == 0) {
+            if (!ok2) atomicOr(a.status, kStatInternal);
+            a.wmed[series] = m2;
+            if (a.wmed_user) a.wmed_user[series] = m2;
+            a.spread[series] = h0;
+            a.centre[series] = m2;
+            if (a.fb_count) { atomicAdd(a.fb_count, 1u); atomicAdd(a.fb_count + 1 + why_src, 1u); }
+        }
+    }
+}
+
+template <int VPL>
+cudaError_t launch_thread_path(const WindowArgs &a, cudaStream_t st) {
+    const size_t smem = (size_t)kThSlots * kThCols * 4;
+    cudaError_t e = cudaFuncSetAttribute(window_thread_kernel<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(window_thread_kernel<VPL>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    window_thread_kernel<VPL><<<(a.series + kThCols - 1) / kThCols, kThCols, smem, st>>>(a);
+    return cudaGetLastError();
+}
+
 // Fallback for windows too long to stage: one thread per series, bit-by-bit counting
 // selection straight from global memory (32 sweeps of the column).
 __global__ void window_select_global_kernel(const WindowArgs a) {
@@ -609,6 +832,7 @@ cudaError_t launch_staged(const WindowArgs &a, int use_bulk, cudaStream_t st) {
 }  // namespace
 
 int window_launch_count(const WindowArgs &a) {
+    if (GUARD_WIN_THREAD && a.use_hint && a.spread && a.centre && a.n <= 256) return 1;
     const bool bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
     return (a.use_hint && bulk && a.spread && a.fb_list && a.n <= 256) ? 2 : 1;
 }
@@ -618,6 +842,14 @@ cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st) {
     // bulk copies need 16-byte aligned sources and sizes
     const int use_bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
     const size_t n = (size_t)a.n;
+#ifndef GUARD_WIN_THREAD
+#define GUARD_WIN_THREAD 1
+#endif
+    if (GUARD_WIN_THREAD && a.use_hint && a.spread && a.centre && n <= 256) {
+        if (n <= 64) return launch_thread_path<2>(a, st);
+        if (n <= 128) return launch_thread_path<4>(a, st);
+        return launch_thread_path<8>(a, st);
+    }
     if (a.use_hint && use_bulk && a.spread && a.fb_list && n <= 256) {
         if (n <= 64) return launch_bracket_path<2>(a, st);
         if (n <= 128) return launch_bracket_path<4>(a, st);
