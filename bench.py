@@ -35,9 +35,13 @@ if ROOT not in sys.path:
 METRIC = "rank-step-metric cells scored/s"
 UNIT = "cells/s"
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum of one xrank_fused_kernel launch on this workload, from the
-# ncu capture summarised under profiles/ (None once the kernel has changed since the capture)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 113.1e6
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this workload, from
+# the ncu capture summarised under profiles/ (None once the kernel has changed since the capture)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# which kernel the roofline object describes: 2 = window_thread_kernel (guard_score), 1 = the MAD sweep (guard_ingest)
+PROFILE_MODE = 2
+PROFILE_KERNEL = ("window_thread_kernel (windowed per-rank medians of one evaluation)" if PROFILE_MODE == 2 else
+                  "xsplit_sweep_kernel<2,1> (cross-rank MAD / exceedance sweep of one ingested block)")
 FALLBACK_HBM_GBS = 6650.0   # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
 
 
@@ -252,6 +256,10 @@ def main():
 
     ev_pairs = []
 
+    # Deferred evaluations: an evaluation runs beside the next block's ingest; its outputs are
+    # complete once the stream has passed the next score() or join().  Every pass ends with a join.
+    g.set_deferred(True)
+
     def one_pass(time_ingest=False):
         g.reset()
         for j in range(n_blocks):
@@ -265,12 +273,13 @@ def main():
             else:
                 g.ingest(blk)
             g.score(out)
+        g.join()
 
     for _ in range(warm):
         one_pass()
     g.sync_status()
     sampler = ClockSampler(local_rank)
-    g.profile_enable(True)
+    g.profile_enable(PROFILE_MODE)
     launches0 = g.kernel_launches
     gd.barrier()
     torch.cuda.synchronize()
@@ -292,16 +301,17 @@ def main():
     value, tmax = gd.aggregate_throughput(cells_per_step * args.steps, secs, device=dev)
     flagged = int(out["flags"].sum().item())
 
-    # roofline of the dominant kernel: the fused cross-rank sweep behind guard_ingest, timed by
-    # the library with CUDA events recorded on the launching stream right around that kernel.
-    # One launch reads a block of 200 steps once from HBM (4 B per cell; its second sweep is
-    # served by L2) and writes one exceedance byte per (step, rank) (1/8 B per cell).
+    # roofline of the dominant kernel, timed by the library with CUDA events recorded right around
+    # it on the stream it is launched on (while the other kernels of the pipeline share the GPU).
+    # The window-median kernel reads the W x ranks x metrics window once (4 B per cell covered);
+    # the MAD / exceedance sweep reads a block of 200 steps once (4 B per cell) and writes one
+    # exceedance byte per (step, rank).
     ingest_ms = [a.elapsed_time(b) for a, b in ev_pairs]
     launch_s = (kern_ms / kern_n / 1e3) if kern_n else statistics.fmean(ingest_ms) / 1e3
-    algo_bytes = B * R * M * 4 + B * R * 1
+    algo_bytes = (cfg.W * R * M * 4) if PROFILE_MODE == 2 else (B * R * M * 4 + B * R * 1)
     peak, peak_kind = measured_hbm_peak()
     achieved = algo_bytes / launch_s / 1e9
-    roofline = {"bound": "hbm", "kernel": "xrank_fused_kernel (cross-rank median / MAD / exceedance of one ingested block)",
+    roofline = {"bound": "hbm", "kernel": PROFILE_KERNEL,
                 "achieved": achieved, "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes_per_launch": algo_bytes,
                 "avg_launch_ms": launch_s * 1e3, "launches_timed": kern_n,
@@ -320,6 +330,8 @@ def main():
     h_idx = torch.empty(cfg.topk, dtype=torch.int32, pin_memory=True)
     h_sc = torch.empty(cfg.topk, dtype=torch.float32, pin_memory=True)
     torch.cuda.synchronize()
+
+    g.set_deferred(False)   # the end-to-end pass reads every evaluation's flags back at once
 
     def one_pass_e2e():
         g.reset()
@@ -373,6 +385,8 @@ def main():
             "config": {"workload": "large fleet: 16384 ranks x 20000 steps x 8 metrics (10.49 GB), W=200 k=120 top-64, "
                                    "100 blocks of 200 steps, one evaluation per block",
                        "ingest": "in place (telemetry written into the ring before timing)",
+                       "evaluation": "deferred (guard_set_deferred): each evaluation runs beside the next block's ingest, "
+                                     "joined before its outputs are reused and at the end of every pass",
                        "l2": "inputs (10.49 GB) larger than L2", "parallelism": "replicas only",
                        "flagged_last_evaluation": flagged, "direct_path_fallback_rows_last_pass": fallback_rows},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,

@@ -218,11 +218,13 @@ int guard_set_deferred(guard_ctx *ctx, int on);
  * synchronisation). */
 int guard_join(guard_ctx *ctx, void *stream);
 
-/* Kernel timing for benchmarks: while enabled, guard_ingest records a pair of CUDA events on
- * the stream right around its main kernel (the fused cross-rank sweep; contexts whose sizes
- * take another path record nothing).  guard_profile_read waits for the recorded events, returns
- * the sum of the kernel durations in milliseconds and their number, and forgets them.
- * Disabling destroys any events not yet read.  Off by default; do not leave it on in a
+/* Kernel timing for benchmarks.  on = 1: guard_ingest records a pair of CUDA events on its
+ * stream right around the longest of its kernels (the MAD / exceedance sweep of the split
+ * cross-rank path; contexts whose sizes take another path record around their main kernel or
+ * nothing).  on = 2: guard_score records the pair around its window-median kernel, on the
+ * stream that kernel runs on.  guard_profile_read waits for the recorded events, returns the
+ * sum of the kernel durations in milliseconds and their number, and forgets them.  on = 0
+ * (default) switches it off and destroys any events not yet read; do not leave it on in a
  * long-running service without reading (events accumulate in host memory). */
 int guard_profile_enable(guard_ctx *ctx, int on);
 int guard_profile_read(guard_ctx *ctx, double *total_ms, int64_t *launches);

@@ -17,9 +17,8 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, wlist, xr_big, mask, ring, total;
+    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, xr_big, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
-    int xr_fused;   // the single-launch fused cross-rank path applies
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
 };
@@ -34,18 +33,15 @@ Layout make_layout(int R, int M, int C, int K) {
     L.consec = off;    off = align_up(off + (size_t)R);
     L.xr_split = xrank_split_supported(R, M) ? 1 : 0;
     L.xr_cluster = (!L.xr_split && xrank_cluster_supported(R, M)) ? 1 : 0;
-    L.xr_fused = (!L.xr_split && !L.xr_cluster && xrank_fused_supported(R, M)) ? 1 : 0;
-    L.xr_steps = (!L.xr_split && !L.xr_cluster && !L.xr_fused && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
+    L.xr_steps = (!L.xr_split && !L.xr_cluster && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
     L.xr_small = off;  off = align_up(off + (L.xr_steps ? xrank_scratch_small_bytes(M, L.xr_steps) : 0));
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
     L.wspread = off;   off = align_up(off + (size_t)R * M * sizeof(float));
     L.wcentre = off;   off = align_up(off + (size_t)R * M * sizeof(float));
-    L.wlist = off;     off = align_up(off + (size_t)R * M * sizeof(uint32_t));
     L.xr_big = off;    off = align_up(off + (L.xr_split ? xrank_split_scratch_bytes(R, M, C < kSplitMaxSteps ? C : kSplitMaxSteps)
-                                             : L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps)
-                                                          : (L.xr_fused ? (size_t)kFusedMaxSteps * M * 8 * sizeof(uint32_t) : 0)));
+                                             : L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps) : 0));
     L.mask = off;      off = align_up(off + (size_t)C * R * (M <= 8 ? 1 : 4));
     L.ring = off;      off = align_up(off + (size_t)C * R * M * sizeof(float));
     L.total = off;
@@ -166,7 +162,7 @@ struct guard_ctx {
         if (e == cudaSuccess) pending = false;
         return e;
     }
-    bool profiling = false;                                   // record events around the main ingest kernel
+    int profiling = 0;                                        // 1: time the MAD sweep of every ingest, 2: the window kernel of every evaluation
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof;    // recorded, not yet read
     char error[256];
 
@@ -202,7 +198,7 @@ struct guard_ctx {
                 if (a.med_user) g.med_user = a.med_user + (size_t)s0 * M;
                 if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
                 cudaError_t e = launch_xrank_split(g, p, n, ws + L.xr_big, status() + 2, st,
-                                                   (profiling && a.mask_base) ? &prof : nullptr);
+                                                   (profiling == 1 && a.mask_base) ? &prof : nullptr);
                 if (e != cudaSuccess) return e;
                 launches += 6;
             }
@@ -211,25 +207,7 @@ struct guard_ctx {
         if (L.xr_cluster && a.mask_bytes == 1) {
             a.fallbacks = status() + 1;
             launches += 1;
-            return launch_xrank_cluster(a, p, S, status() + 2, st, (profiling && a.mask_base) ? &prof : nullptr);
-        }
-        if (L.xr_fused) {
-            a.fallbacks = status() + 1;
-            const int first = a.first_slot;
-            for (int s0 = 0; s0 < S; s0 += kFusedMaxSteps) {
-                const int n = (S - s0 < kFusedMaxSteps) ? (S - s0) : kFusedMaxSteps;
-                XrankArgs g = a;
-                g.first_slot = (int)(((long long)first + s0) % a.capacity);
-                g.med = a.med + (size_t)s0 * M;
-                g.mad = a.mad + (size_t)s0 * M;
-                if (a.med_user) g.med_user = a.med_user + (size_t)s0 * M;
-                if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
-                cudaError_t e = launch_xrank_fused(g, p, n, status() + 2, (uint32_t *)(ws + L.xr_big), st,
-                                                   (profiling && a.mask_base) ? &prof : nullptr);
-                if (e != cudaSuccess) return e;
-                launches += 2;
-            }
-            return cudaSuccess;
+            return launch_xrank_cluster(a, p, S, status() + 2, st, (profiling == 1 && a.mask_base) ? &prof : nullptr);
         }
         if (L.xr_steps == 0) { launches += 1; return launch_xrank_direct(a, p, S, st); }
         XrankScratch sc = carve_xrank_scratch(ws + L.xr_small, ws + L.xr_big, R, M, L.xr_steps);
@@ -249,6 +227,17 @@ struct guard_ctx {
             launches += 6;
         }
         return cudaSuccess;
+    }
+    // The window kernel, with a pair of events around it on its stream while profiling mode 2 is on.
+    cudaError_t window(const WindowArgs &w, cudaStream_t ws_) {
+        if (profiling != 2) return launch_window_select(w, ws_);
+        cudaEvent_t e0 = nullptr, e1 = nullptr;
+        if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return cudaGetLastError();
+        cudaEventRecord(e0, ws_);
+        const cudaError_t e = launch_window_select(w, ws_);
+        cudaEventRecord(e1, ws_);
+        prof.emplace_back(e0, e1);
+        return e;
     }
     int fail(int code, const char *fmt, ...) {
         va_list ap;
@@ -378,7 +367,6 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     w.use_hint = c->evals > 0 ? 1 : 0;
     w.spread = (float *)(c->ws + c->L.wspread);
     w.centre = (float *)(c->ws + c->L.wcentre);
-    w.fb_list = (uint32_t *)(c->ws + c->L.wlist);
     w.fb_count = c->status() + 8;
     w.status = c->status();
     // The window medians read only the ring: run them on the internal stream, forked where the
@@ -404,7 +392,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         }
         e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
         if (e == cudaSuccess && had_pending) e = cudaStreamWaitEvent(c->side, c->ev_e, 0);
-        if (e == cudaSuccess) e = launch_window_select(w, c->side);
+        if (e == cudaSuccess) e = c->window(w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_x, st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_w, 0);
@@ -412,11 +400,11 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         ts = c->tail;
     } else if (forked) {
         e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
-        if (e == cudaSuccess) e = launch_window_select(w, c->side);
+        if (e == cudaSuccess) e = c->window(w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_join, c->side);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_join, 0);
     } else {
-        e = launch_window_select(w, st);
+        e = c->window(w, st);
     }
     if (e != cudaSuccess) return c->cuda_fail(e, "window_select launch");
 
@@ -602,7 +590,7 @@ int guard_reset(guard_ctx *c, void *stream) {
 
 int guard_profile_enable(guard_ctx *c, int on) {
     if (!c) return GUARD_ERR_ARG;
-    c->profiling = on != 0;
+    c->profiling = on;
     if (!on) {
         for (auto &pr : c->prof) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
         c->prof.clear();

@@ -47,11 +47,6 @@ enum { kWhyCtaList = 0, kWhyStepList = 1, kWhyAmbList = 2, kWhyMedianMiss = 3, k
 // One CTA per (row, metric) column with the column in registers: for a few rows at a time.
 bool xrank_column_supported(int R);
 cudaError_t launch_xrank_column(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st);
-bool xrank_fused_supported(int R, int M);
-// qscratch: S * M * 8 words.
-// prof: if not NULL, a pair of events recorded on st right around the main kernel is appended.
-cudaError_t launch_xrank_fused(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, uint32_t *qscratch,
-                               cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof = nullptr);
 // One cluster of four CTAs per step (4 or 8 metrics, a few thousand ranks and more).
 bool xrank_cluster_supported(int R, int M);
 cudaError_t launch_xrank_cluster(const XrankArgs &a, const MetricParams &p, int S, uint32_t *reasons, cudaStream_t st,
@@ -63,7 +58,6 @@ constexpr int kSplitMaxSteps = 256;   // steps per launch group of the split pat
 size_t xrank_split_scratch_bytes(int R, int M, int S_max);
 cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S, void *scratch, uint32_t *reasons,
                                cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof = nullptr);
-constexpr int kFusedMaxSteps = 1024;   // steps per launch of the fused path (sizes its scratch)
 bool xrank_bracket_supported(int R, int M);
 int xrank_scratch_steps(int R, int M, int want);
 size_t xrank_scratch_small_bytes(int M, int S_max);   // must be zero before first use
@@ -85,13 +79,12 @@ struct WindowArgs {
     float *wmed;            // [series] (never NULL)
     int use_hint;           // wmed holds the previous evaluation's medians: use them as first pivots
     float *wmed_user;       // or NULL
-    float *spread;          // [series] tuned half-width of the bracket path's interval (state), or NULL
+    float *spread;          // [series] tuned half-width of the thread path's interval (state), or NULL
     float *centre;          // [series] smoothed median: the centre of the thread path's interval (state), or NULL
-    uint32_t *fb_list;      // [series] series the bracket path hands to the list kernel, or NULL
-    uint32_t *fb_count;     // their number
+    uint32_t *fb_count;     // [6] series the thread path's interval did not serve, in total and by reason (diagnostic), or NULL
     uint32_t *status;
 };
-// Launches 1 kernel (warp or staged path) or 2 (bracket path + list kernel).
+// Launches one kernel (thread, warp or staged path).
 cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st);
 int window_launch_count(const WindowArgs &a);
 

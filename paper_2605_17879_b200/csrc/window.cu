@@ -7,10 +7,6 @@
 #include "colselect.cuh"
 #include "kernels.h"
 
-#ifndef GUARD_WIN_THREAD
-#define GUARD_WIN_THREAD 1
-#endif
-
 namespace guard {
 
 namespace {
@@ -238,10 +234,10 @@ __device__ __forceinline__ bool warp_median(const uint32_t (&kv)[VPL], const int
     return false;
 }
 
-// A first guess of the half-width the bracket path should search around a series' previous
-// median: 0.45 x the mean absolute deviation of the window about its median (for Gaussian
-// noise that spans about +-0.36 sigma, some 3 standard errors of a 200-step median and ~28 %
-// of the window).  Only a starting point: the bracket path re-tunes it from its own counts.
+// A first guess of the half-width the thread path should search around a series' smoothed
+// median: 0.36 x the mean absolute deviation of the window about its median (for Gaussian
+// noise that spans about +-0.29 sigma, some 3 standard errors of a 200-step median and ~22 %
+// of the window).  Only a starting point: the thread path re-tunes it from its own counts.
 template <int VPL>
 __device__ __forceinline__ float warp_spread_guess(const uint32_t (&kv)[VPL], const int n, const float med) {
     float s = 0.0f;
@@ -250,7 +246,7 @@ __device__ __forceinline__ float warp_spread_guess(const uint32_t (&kv)[VPL], co
         if (kv[i] != 0xFFFFFFFFu) s += fabsf(key2f(kv[i]) - med);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-    return (GUARD_WIN_THREAD ? 0.36f : 0.45f) * s / (float)n;
+    return 0.36f * s / (float)n;
 }
 
 template <int VPL>
@@ -352,215 +348,10 @@ cudaError_t launch_warp_path(const WindowArgs &a, int use_bulk, cudaStream_t st)
 }
 
 // ---------------------------------------------------------------------------------------
-// Bracket path: from the second evaluation on, a series' previous median and a tuned
-// half-width h give an interval [hint - h, hint + h] that almost always holds the new middle
-// elements.  One THREAD per series then suffices: the window's rows stream through a small
-// TMA-fed ring of shared-memory stages (8 rows x 256 series each), every thread counts its
-// keys below the interval and keeps those inside it (a few dozen) in its own shared-memory
-// column, checks from the counts that the middle ranks are among them and selects them there.
-// That is ~10 instructions per element and thread instead of a warp's cooperative walk.
-// Series whose interval missed (or overflowed) go to a list that a warp-per-series kernel
-// finishes exactly; h is re-tuned every time from the number of keys the interval caught.
-// ---------------------------------------------------------------------------------------
-constexpr int kBrCols = 256;     // series per CTA = threads per CTA
-constexpr int kBrRows = 8;       // rows per stage (one per warp)
-constexpr int kBrStages = 4;
-constexpr int kBrSlots = 72;     // kept keys per series
-constexpr int kBrTarget = 52;    // number of keys the interval is tuned to catch
-
-// Ranks t - 1 and t among the nk keys a thread kept (column `col`, pitch kBrCols), all inside
-// [klo, khi].  Kept keys of a narrow interval are close to evenly spread, so the pivot is
-// interpolated in key space (regula falsi on the count below the pivot): a pass counts the
-// keys below the pivot and tracks the two largest keys below it and the two smallest keys not
-// below it; when t - 1, t or t + 1 keys are below, two of those four ARE ranks t - 1 and t.
-// Every thread runs the same fixed-length scans, so a warp does not diverge the way per-thread
-// partitioning does.  Returns false after a few passes (e.g. when the ranks sit inside a long
-// run of equal keys) to let the caller fall back to partitioning.
-__device__ __forceinline__ bool kept_rank_pair(const uint32_t *col, int nk, int t, uint32_t klo, uint32_t khi,
-                                               uint32_t &v_prev, uint32_t &v_t) {
-    unsigned long long pl = klo, ph = (unsigned long long)khi + 1ull;   // counts below: al at pl, ah at ph
-    int al = 0, ah = nk;
-    for (int pass = 0; pass < 8; ++pass) {
-        if (ph - pl < 2ull) return false;
-        // aim between the bracket's ends in proportion to the missing count
-        unsigned long long p = pl + (unsigned long long)((float)(ph - pl) * (((float)(t - al) + 0.5f) / (float)(ah - al)));
-        p = p <= pl ? pl + 1ull : (p >= ph ? ph - 1ull : p);
-        const uint32_t pv = (uint32_t)p;
-        int below = 0;
-        uint32_t b1 = 0u, b2 = 0u, u1 = 0xFFFFFFFFu, u2 = 0xFFFFFFFFu;
-        for (int i = 0; i < nk; i += kSelBatch) {
-            uint32_t v[kSelBatch];
-#pragma unroll
-            for (int q = 0; q < kSelBatch; ++q) v[q] = (i + q < nk) ? col[(size_t)(i + q) * kBrCols] : 0xFFFFFFFFu;
-#pragma unroll
-            for (int q = 0; q < kSelBatch; ++q) {
-                const bool lt = v[q] < pv;
-                below += lt;
-                const uint32_t lo_v = lt ? v[q] : 0u, hi_v = lt ? 0xFFFFFFFFu : v[q];   // neutral on the other side
-                b2 = max(b2, min(b1, lo_v));
-                b1 = max(b1, lo_v);
-                u2 = min(u2, max(u1, hi_v));
-                u1 = min(u1, hi_v);
-            }
-        }
-        if (below == t) { v_prev = b1; v_t = u1; return true; }
-        if (below == t + 1) { v_prev = b2; v_t = b1; return true; }
-        if (below == t - 1) { v_prev = u1; v_t = u2; return true; }
-        if (below < t) { pl = p; al = below; } else { ph = p; ah = below; }
-    }
-    return false;
-}
-
-__global__ void __launch_bounds__(kBrCols, 2) window_bracket_kernel(const WindowArgs a) {
-    extern __shared__ __align__(128) uint32_t bsm[];
-    uint32_t *tile = bsm;                                        // [kBrStages][kBrRows][kBrCols]
-    uint32_t *kept = bsm + kBrStages * kBrRows * kBrCols;        // [kBrSlots][kBrCols]
-    __shared__ __align__(8) uint64_t bar[kBrStages];
-    const int tid = threadIdx.x, lane = lane_id(), w = warp_id();
-    const int n = a.n;
-    const int col0 = blockIdx.x * kBrCols;
-    const int ncols = min(kBrCols, a.series - col0);
-    const int c = col0 + tid;
-    const bool active = tid < ncols;
-    const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;
-    const int nchunks = (n + kBrRows - 1) / kBrRows;
-
-    if (tid == 0)
-        for (int s = 0; s < kBrStages; ++s) mbar_init(&bar[s], kBrRows);
-    __syncthreads();
-    // lane 0 of warp w feeds row w of every chunk (or just arrives when the chunk has no such row)
-    auto feed = [&](int chunk) {
-        if (lane != 0) return;
-        const int stage = chunk % kBrStages;
-        const int row = chunk * kBrRows + w;
-        if (row < n) {
-            int slot = first + row;
-            if (slot >= a.capacity) slot -= a.capacity;
-            mbar_arrive_expect_tx(&bar[stage], (uint32_t)ncols * 4u);
-            bulk_g2s(tile + (stage * kBrRows + w) * kBrCols, a.ring + (size_t)slot * a.row_stride + col0, (uint32_t)ncols * 4u,
-                     &bar[stage]);
-        } else {
-            mbar_arrive(&bar[stage]);
-        }
-    };
-    for (int ch = 0; ch < kBrStages && ch < nchunks; ++ch) feed(ch);
-
-    float hint = 0.0f, h = 0.0f;
-    if (active) { hint = a.wmed[c]; h = a.spread[c]; }
-    const bool usable = active && (h > 0.0f) && (h < 3.0e38f) && (fabsf(hint) < 3.0e38f);
-    // The interval is tested with float compares (keys are made only of what is kept).  That
-    // agrees with the key order as long as an end that is zero admits both zeros: -0 as lower
-    // end, +0 as upper end.  An unusable interval keeps nothing and counts nothing below it, so
-    // it fails the check after the loop.
-    float flo = hint - h, fhi = hint + h;
-    if (flo == 0.0f) flo = -0.0f;
-    if (fhi == 0.0f) fhi = 0.0f;
-    if (!usable) { flo = CUDART_INF_F; fhi = -CUDART_INF_F; }
-    const uint32_t klo = usable ? f2key(flo) : 0xFFFFFFFFu, khi = usable ? f2key(fhi) : 0u;
-    int clt = 0, nk = 0;
-    for (int ch = 0; ch < nchunks; ++ch) {
-        const int stage = ch % kBrStages;
-        if (!mbar_wait_bounded(&bar[stage], (uint32_t)((ch / kBrStages) & 1), kWaitLimitCycles)) {
-            atomicOr(a.status, kStatTimeout);
-            for (int s2 = 0; s2 < kBrStages; ++s2) {   // let copies in flight land before leaving
-                const int fed = ch + ((s2 - stage + kBrStages) % kBrStages);   // the chunk stage s2 is waiting for
-                if (fed < nchunks) mbar_wait_bounded(&bar[s2], (uint32_t)((fed / kBrStages) & 1), kWaitLimitCycles);
-            }
-            return;
-        }
-        const int rows = min(kBrRows, n - ch * kBrRows);
-        const uint32_t *t = tile + stage * kBrRows * kBrCols + tid;
-        float x[kBrRows];
-#pragma unroll
-        for (int r = 0; r < kBrRows; ++r) x[r] = __uint_as_float(t[r * kBrCols]);
-#pragma unroll
-        for (int r = 0; r < kBrRows; ++r) {
-            if (r < rows) {   // rows beyond the window's end hold stale data
-                clt += (x[r] < flo);
-                if (x[r] >= flo && x[r] <= fhi) {
-                    if (nk < kBrSlots) kept[nk * kBrCols + tid] = f2key(x[r]);
-                    ++nk;
-                }
-            }
-        }
-        __syncthreads();   // the stage is free again
-        if (ch + kBrStages < nchunks) feed(ch + kBrStages);
-    }
-    if (!active) return;
-    const bool even = !(n & 1);
-    const int k1 = (n - 1) >> 1, k2 = n >> 1;
-    const bool ok = usable && clt <= k1 && k2 < clt + nk && nk <= kBrSlots;
-    if (ok) {
-        uint32_t v1, v2;
-        const int t = k2 - clt;   // rank of the upper middle among the kept keys (t >= 1 when even)
-        if (!kept_rank_pair(kept + tid, nk, t, klo, khi, v1, v2)) col_rank_pair(kept + tid, kBrCols, nk, t, even, v1, v2);
-        const float med = median_from_keys(even ? v1 : v2, v2, even);
-        a.wmed[c] = med;
-        if (a.wmed_user) a.wmed_user[c] = med;
-        // re-tune the half-width so that the interval catches about kBrTarget keys next time
-        // (half of the way: one window's count is a noisy estimate of the density)
-        const float f = fminf(2.0f, fmaxf(0.5f, (float)kBrTarget / (float)max(nk, 1)));
-        a.spread[c] = h * (0.5f + 0.5f * f);
-    } else {
-        a.fb_list[atomicAdd(a.fb_count, 1u)] = (uint32_t)c;   // the list kernel finishes this series
-    }
-}
-
-// Finishes the series the bracket path could not: one warp per listed series, window read
-// straight from the ring (few series, so the scattered loads do not matter).
-template <int VPL>
-__global__ void __launch_bounds__(256) window_list_kernel(const WindowArgs a) {
-    const int lane = lane_id();
-    const int wglobal = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, wtotal = (gridDim.x * blockDim.x) >> 5;
-    const int n = a.n;
-    const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;
-    const uint32_t count = *a.fb_count;
-    for (uint32_t i = wglobal; i < count; i += wtotal) {
-        const int series = (int)a.fb_list[i];
-        uint32_t kv[VPL];
-        int nreal = 0;
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            const int row = lane + 32 * j;
-            kv[j] = 0xFFFFFFFFu;
-            if (row < n) {
-                int slot = first + row;
-                if (slot >= a.capacity) slot -= a.capacity;
-                kv[j] = f2key(a.ring[(size_t)slot * a.row_stride + series]);
-                ++nreal;
-            }
-        }
-        lane_sort<VPL>(kv);
-        float med = 0.0f;
-        const bool ok = warp_median<VPL>(kv, nreal, n, 0u, med);
-        const float h0 = warp_spread_guess<VPL>(kv, n, med);
-        if (lane == 0) {
-            if (!ok) atomicOr(a.status, kStatInternal);
-            a.wmed[series] = med;
-            if (a.wmed_user) a.wmed_user[series] = med;
-            a.spread[series] = h0;
-        }
-    }
-}
-
-template <int VPL>
-cudaError_t launch_bracket_path(const WindowArgs &a, cudaStream_t st) {
-    const size_t smem = (size_t)(kBrStages * kBrRows + kBrSlots) * kBrCols * 4;
-    cudaError_t e = cudaFuncSetAttribute(window_bracket_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(a.fb_count, 0, sizeof(uint32_t), st);
-    if (e != cudaSuccess) return e;
-    window_bracket_kernel<<<(a.series + kBrCols - 1) / kBrCols, kBrCols, smem, st>>>(a);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    window_list_kernel<VPL><<<sms, 256, 0, st>>>(a);
-    return cudaGetLastError();
-}
-
-// ---------------------------------------------------------------------------------------
-// Thread path: the interval idea without staging.  One thread per series reads its window
+// Thread path: from the second evaluation on, a series' smoothed median and a tuned half-width
+// h give an interval [centre - h, centre + h] that almost always holds the new middle
+// elements, so that counting the values below the interval and selecting among the few dozen
+// inside it replaces sorting the window.  One thread per series reads its window
 // straight from the ring (a warp reads 32 adjacent series of a row: one fully used 128-byte
 // line per load, eight rows in flight per thread), counts the values below the interval and
 // keeps those inside it, as raw bits, in its own shared-memory column.  No thread ever waits
@@ -831,29 +622,17 @@ cudaError_t launch_staged(const WindowArgs &a, int use_bulk, cudaStream_t st) {
 
 }  // namespace
 
-int window_launch_count(const WindowArgs &a) {
-    if (GUARD_WIN_THREAD && a.use_hint && a.spread && a.centre && a.n <= 256) return 1;
-    const bool bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
-    return (a.use_hint && bulk && a.spread && a.fb_list && a.n <= 256) ? 2 : 1;
-}
+int window_launch_count(const WindowArgs &) { return 1; }
 
 cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st) {
     constexpr size_t kMaxTile = 200 * 1024;
     // bulk copies need 16-byte aligned sources and sizes
     const int use_bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
     const size_t n = (size_t)a.n;
-#ifndef GUARD_WIN_THREAD
-#define GUARD_WIN_THREAD 1
-#endif
-    if (GUARD_WIN_THREAD && a.use_hint && a.spread && a.centre && n <= 256) {
+    if (a.use_hint && a.spread && a.centre && n <= 256) {
         if (n <= 64) return launch_thread_path<2>(a, st);
         if (n <= 128) return launch_thread_path<4>(a, st);
         return launch_thread_path<8>(a, st);
-    }
-    if (a.use_hint && use_bulk && a.spread && a.fb_list && n <= 256) {
-        if (n <= 64) return launch_bracket_path<2>(a, st);
-        if (n <= 128) return launch_bracket_path<4>(a, st);
-        return launch_bracket_path<8>(a, st);
     }
     if (n <= 64) return launch_warp_path<2>(a, use_bulk, st);
     if (n <= 128) return launch_warp_path<4>(a, use_bulk, st);

@@ -774,24 +774,20 @@ cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S,
         attr_set = true;
     }
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    if (prof) {
-        if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return cudaGetLastError();
-        cudaEventRecord(ev0, st);
-    }
+    if (prof && (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess)) return cudaGetLastError();
     const dim3 gcol(M, S), gsw(g.chunks, S);
     xsplit_sample_kernel<<<dim3(M / 4, S), kSpSmpThreads, 0, st>>>(a, g, sc, reasons);
     if (M == 8) xsplit_sweep_kernel<2, 0><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
     else xsplit_sweep_kernel<1, 0><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
     xsplit_select_kernel<0><<<gcol, kSpSelThreads, 0, st>>>(a, p, g, sc, reasons);
+    if (prof) cudaEventRecord(ev0, st);   // the MAD / exceedance sweep, the longest kernel of the six
     if (M == 8) xsplit_sweep_kernel<2, 1><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
     else xsplit_sweep_kernel<1, 1><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
+    if (prof) cudaEventRecord(ev1, st);
     xsplit_select_kernel<1><<<gcol, kSpSelThreads, 0, st>>>(a, p, g, sc, reasons);
     xsplit_finish_kernel<<<S, kSpThreads, (size_t)M * 256 * sizeof(uint32_t), st>>>(a, p, sc);
     e = cudaGetLastError();
-    if (prof) {
-        cudaEventRecord(ev1, st);
-        prof->emplace_back(ev0, ev1);
-    }
+    if (prof) prof->emplace_back(ev0, ev1);
     return e;
 }
 

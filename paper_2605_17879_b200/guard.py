@@ -215,11 +215,12 @@ class Guard:
         with torch.cuda.device(self.device):
             self._check(lib().guard_join(self._h, _stream()))
 
-    def profile_enable(self, on: bool = True) -> None:
-        self._check(lib().guard_profile_enable(self._h, 1 if on else 0))
+    def profile_enable(self, on=True) -> None:
+        """0 / False: off; 1 / True: time the MAD sweep of every ingest; 2: the window kernel of every evaluation."""
+        self._check(lib().guard_profile_enable(self._h, int(on)))
 
     def profile_read(self):
-        """(total milliseconds, launches) of the main ingest kernel since the last read."""
+        """(total milliseconds, launches) of the profiled kernel since the last read."""
         ms, n = C.c_double(), C.c_int64()
         self._check(lib().guard_profile_read(self._h, C.byref(ms), C.byref(n)))
         return ms.value, n.value
