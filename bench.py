@@ -226,6 +226,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--streaming-steps", type=int, default=500)
+    ap.add_argument("--blocks", type=int, default=0,
+                    help="profile-sized run: only this many 200-step blocks of the workload (0 = all 100); not a bench value")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -242,6 +244,9 @@ def main():
     warm = max(3, args.warmup)
 
     cfg = workload()
+    if args.blocks > 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, steps=max(2, args.blocks) * cfg.block)
     R, M, T, B = cfg.ranks, cfg.metrics, cfg.steps, cfg.block
     n_blocks = T // B
     dirs = synth.fleet_dir(M)
@@ -382,8 +387,9 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
             "ms_per_step": 1e3 * tmax / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "large fleet: 16384 ranks x 20000 steps x 8 metrics (10.49 GB), W=200 k=120 top-64, "
-                                   "100 blocks of 200 steps, one evaluation per block",
+            "config": {"workload": ("large fleet: 16384 ranks x 20000 steps x 8 metrics (10.49 GB), W=200 k=120 top-64, "
+                                    "100 blocks of 200 steps, one evaluation per block") if args.blocks <= 0 else
+                                   ("PROFILE-SIZED RUN (not a bench value): %d blocks of the large fleet" % (T // B)),
                        "ingest": "in place (telemetry written into the ring before timing)",
                        "evaluation": "deferred (guard_set_deferred): each evaluation runs beside the next block's ingest, "
                                      "joined before its outputs are reused and at the end of every pass",

@@ -475,10 +475,17 @@ __global__ void __launch_bounds__(kThCols, 7) window_thread_kernel(const WindowA
                     pv = pv <= pl ? pl + 1u : (pv >= ph ? ph - 1u : pv);
                 }
             }
+            // the loads of a third of the column are issued before their compares
             int below = 0;
-            for (int j = 0; j < nkr; j += 4) {
-                const uint4 v = th_lds4(kbase + 4u * j);
-                below += (v.x < pv) + (v.y < pv) + (v.z < pv) + (v.w < pv);
+#pragma unroll
+            for (int j0 = 0; j0 < kThSlots / 4; j0 += 5) {
+                uint4 kv4[5];
+#pragma unroll
+                for (int j = 0; j < 5; ++j)
+                    if (4 * (j0 + j) < nkr) kv4[j] = th_lds4(kbase + 16u * (j0 + j));
+#pragma unroll
+                for (int j = 0; j < 5; ++j)
+                    if (4 * (j0 + j) < nkr) below += (kv4[j].x < pv) + (kv4[j].y < pv) + (kv4[j].z < pv) + (kv4[j].w < pv);
             }
             if (!done) {
                 if (below >= t - 1 && below <= t + 1) { done = 1; bsave = below; }

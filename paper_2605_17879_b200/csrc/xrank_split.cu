@@ -143,7 +143,7 @@ struct SpSampleShared {
 // that a warp's 128-bit loads use whole cache lines (a column-wise strided sample costs one
 // line per value).  One CTA handles four metrics: every thread bins the four components of
 // its float4 into the four histograms; then 64 threads per metric scan their histogram.
-__global__ void __launch_bounds__(kSpSmpThreads) xsplit_sample_kernel(const XrankArgs a, const SpGeom g, const SpScratch sc,
+__global__ void __launch_bounds__(kSpSmpThreads, 3) xsplit_sample_kernel(const XrankArgs a, const SpGeom g, const SpScratch sc,
                                                                       uint32_t *reasons) {
     __shared__ SpSampleShared sh;
     const int q = blockIdx.x, t = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
