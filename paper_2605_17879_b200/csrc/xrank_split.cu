@@ -281,39 +281,6 @@ struct SpSweepShared {
     uint32_t fail;
 };
 
-// A rank with a value that is not finite, or that might exceed its threshold (both rare): the
-// finite check, then exact tests against the threshold's possible range [rlo, rhi]; the bit is
-// set at once or the decision deferred until the MAD is known.
-template <int NQ>
-__device__ __noinline__ void sp_slow_row(const float *__restrict__ row, const int r, const int q, SpSweepShared &sh,
-                                         uint32_t *namb, uint32_t *amb, uint8_t *maskrow, uint32_t *status) {
-    constexpr int M = 4 * NQ;
-    const float4 x4 = __ldg(reinterpret_cast<const float4 *>(row + (size_t)r * M) + q);
-    const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
-    uint32_t eb = 0;
-    bool bad = false;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const int m = 4 * q + c;
-        bad |= nonfinite_bits(__float_as_uint(xs[c]));
-        const float sg = sh.sgn[m];
-        const float sdev = __fmaf_rn(xs[c], sg, -sg * sh.med[m]);
-        if (sdev > sh.rlo[m]) {
-            if (sdev > sh.rhi[m]) {
-                eb |= 1u << m;
-            } else {
-                const uint32_t pos = atomicAdd(namb, 1u);
-                if (pos < (uint32_t)kSpAmb) amb[pos] = ((uint32_t)r << 5) | (uint32_t)m;
-            }
-        }
-    }
-    if (bad && status) atomicOr(status, kStatNonFinite);
-    if (eb && maskrow) {
-        unsigned int *w = reinterpret_cast<unsigned int *>(maskrow + (r & ~3));
-        atomicOr(w, eb << (8 * (r & 3)));
-    }
-}
-
 // MODE 0: count x < lo, keep lo <= x <= hi.  MODE 1: the same for d = |x - med| against
 // [dlo, dhi], plus the exceedance bits and the finite check.
 // Kept elements: every batch (kSpU ranks x 4 metrics per thread) the lanes of a metric quad
@@ -392,7 +359,7 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
                     for (int c = 0; c < 4; ++c) v[j][c] = MODE == 0 ? CUDART_NAN_F : __fmul_rn(sg[c], -nsm[c]);   // MODE 1: x = med
                 }
         }
-        uint32_t packed = 0, slowmask = 0;
+        uint32_t packed = 0;
 #pragma unroll
         for (int j = 0; j < kSpU; ++j) {
             if (MODE == 1) {
@@ -401,13 +368,37 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
                 // the threshold's range (a possible exceedance) and values that are not finite (the
                 // comparison is false for NaN).
                 bool slow = false;
+                float sdev[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const float d = fabsf(__fmaf_rn(v[j][c], sg[c], nsm[c]));
+                    sdev[c] = __fmaf_rn(v[j][c], sg[c], nsm[c]);
+                    const float d = fabsf(sdev[c]);
                     v[j][c] = d;
                     slow |= !(d <= rlo[c]);
                 }
-                if (slow) slowmask |= 1u << j;   // handled at the end of the batch, where little else is live
+                // The rare remainder, settled while the signed deviations are at hand (no reload): the
+                // finite check, then exact tests against the threshold's possible range [rlo, rhi]; the
+                // bit is set at once or the decision deferred until the MAD is known.
+                if (slow) {
+                    const int r = base + j * LPI + rl;
+                    if (!guard || r < r1) {
+                        uint32_t eb = 0;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const int m = 4 * q + c;
+                            if (!(fabsf(sdev[c]) <= kFltMax) && a.check_finite) atomicOr(a.status, kStatNonFinite);
+                            if (sdev[c] > rlo[c]) {
+                                if (sdev[c] > sh.rhi[m]) {
+                                    eb |= 1u << m;
+                                } else {
+                                    const uint32_t pos = atomicAdd(sc.namb + t, 1u);
+                                    if (pos < (uint32_t)kSpAmb) sc.amb[(size_t)t * kSpAmb + pos] = ((uint32_t)r << 5) | (uint32_t)m;
+                                }
+                            }
+                        }
+                        if (eb && maskrow) atomicOr(reinterpret_cast<unsigned int *>(maskrow + (r & ~3)), eb << (8 * (r & 3)));
+                    }
+                }
                 if (guard && base + j * LPI + rl >= r1) {
 #pragma unroll
                     for (int c = 0; c < 4; ++c) v[j][c] = CUDART_NAN_F;
@@ -443,15 +434,6 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
         for (int j = 0; j < kSpU; ++j)
 #pragma unroll
             for (int c = 0; c < 4; ++c) sp_cell_keep(v[j][c], lo[c], hi[c], addr[c]);
-        if (MODE == 1 && slowmask) {
-#pragma unroll 1
-            for (int j = 0; j < kSpU; ++j) {
-                const int r = base + j * LPI + rl;
-                if (((slowmask >> j) & 1u) && r < r1)
-                    sp_slow_row<NQ>(row, r, q, sh, sc.namb + t, sc.amb + (size_t)t * kSpAmb, maskrow,
-                                    a.check_finite ? a.status : nullptr);
-            }
-        }
     };
     const int span = LPI * kSpU;
     int base = r0;
