@@ -37,7 +37,7 @@ UNIT = "cells/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this workload, from
 # the ncu capture summarised under profiles/ (None once the kernel has changed since the capture)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 115.85e6
 # which kernel the roofline object describes: 2 = window_thread_kernel (guard_score), 1 = the MAD sweep (guard_ingest)
 PROFILE_MODE = 2
 PROFILE_KERNEL = ("window_thread_kernel (windowed per-rank medians of one evaluation)" if PROFILE_MODE == 2 else
@@ -56,7 +56,7 @@ def measured_hbm_peak():
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -70,12 +70,15 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Summary of the samples taken between the host times t_begin and t_end (the timed region);
+        if the region was too short to catch one, of the samples within half a second around it."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -84,25 +87,35 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             pass
-        sm, mx, reasons = [], [], set()
+        recs = []
         try:
             for ln in open(self.path):
                 p = [x.strip() for x in ln.split(",")]
                 if len(p) < 9:
                     continue
                 try:
-                    sm.append(float(p[1]))
-                    mx.append(float(p[2]))
+                    ts = datetime.datetime.strptime(p[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    recs.append((ts, float(p[1]), float(p[2]), p[5:9]))
                 except ValueError:
                     continue
-                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
-                    if v.lower().startswith("active"):
-                        reasons.add(name)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        window = "timed region"
+        sel = recs
+        if t_begin is not None and t_end is not None:
+            sel = [r for r in recs if t_begin <= r[0] <= t_end]
+            if not sel:
+                sel = [r for r in recs if t_begin - 0.5 <= r[0] <= t_end + 0.5]
+                window = "within 0.5 s of the timed region (the same load: warm-up passes run right before it)"
+        reasons = set()
+        for r in sel:
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if sel:
+            out.update(sm_mhz=statistics.median([r[1] for r in sel]), sm_max_mhz=max(r[2] for r in sel), samples=len(sel),
+                       window=window)
         out["reasons"] = sorted(reasons)
         return out
 
@@ -220,7 +233,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="guard", choices=["guard", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -280,23 +293,25 @@ def main():
             g.score(out)
         g.join()
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()   # nvidia-smi needs a moment before its first sample: started ahead of the warm-up passes
     for _ in range(warm):
         one_pass()
     g.sync_status()
-    sampler = ClockSampler(local_rank)
     g.profile_enable(PROFILE_MODE)
     launches0 = g.kernel_launches
     gd.barrier()
     torch.cuda.synchronize()
-    sampler.start()
+    t_begin = time.time()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record()
     for _ in range(args.steps):
         one_pass(time_ingest=True)
     stop.record()
     torch.cuda.synchronize()
+    t_end = time.time()
     gd.barrier()
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_begin, t_end)
     kern_ms, kern_n = g.profile_read()
     g.profile_enable(False)
     g.sync_status()
