@@ -207,8 +207,11 @@ int guard_set_overlap(guard_ctx *ctx, int on);
  * buffers of that guard_score call are complete, in the order of a stream, only after that
  * stream has passed the next guard_score, guard_join, guard_sync_status or guard_reset on
  * this context; until then the caller must neither read nor reuse them.  At most one
- * evaluation is pending.  The ring slots of the pending evaluation's window must not be
- * overwritten: guard_ingest waits for the evaluation by itself when its block reuses them,
+ * evaluation is pending.  In this mode guard_ingest, too, may run its kernels on streams of the
+ * library's own (two, taken in turn, ordered after everything enqueued on `stream` so far) when
+ * the caller passes no d_step_med / d_step_mad: consecutive blocks then overlap one another;
+ * the same calls as above make `stream` wait for them.  The ring slots of the pending evaluation's window must not be
+ * overwritten, nor those of blocks whose kernels still run: guard_ingest waits by itself when its block reuses them,
  * and guard_ring_reserve refuses (GUARD_ERR_NOT_READY) to hand them out, since it cannot
  * order the caller's writes; with capacity_steps >= W + block size neither ever happens.
  * Results are identical to the default mode. */

@@ -17,7 +17,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, xr_big, mask, ring, total;
+    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, xr_big, xr_big2, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
@@ -42,6 +42,8 @@ Layout make_layout(int R, int M, int C, int K) {
     L.wcentre = off;   off = align_up(off + (size_t)R * M * sizeof(float));
     L.xr_big = off;    off = align_up(off + (L.xr_split ? xrank_split_scratch_bytes(R, M, C < kSplitMaxSteps ? C : kSplitMaxSteps)
                                              : L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps) : 0));
+    // a second scratch: in deferred mode consecutive blocks run their cross-rank kernels on two streams
+    L.xr_big2 = off;   off = align_up(off + (L.xr_split ? xrank_split_scratch_bytes(R, M, C < kSplitMaxSteps ? C : kSplitMaxSteps) : 0));
     L.mask = off;      off = align_up(off + (size_t)C * R * (M <= 8 ? 1 : 4));
     L.ring = off;      off = align_up(off + (size_t)C * R * M * sizeof(float));
     L.total = off;
@@ -140,8 +142,43 @@ struct guard_ctx {
     bool deferred = false;
     bool pending = false;             // an evaluation has been enqueued whose end the caller's stream has not waited for
     int pending_n = 0;                // its window length
+    // In deferred mode the cross-rank kernels of consecutive ingests alternate between two internal
+    // streams (each with its own scratch), so that one block's selections overlap the next block's
+    // sweeps; the caller's stream waits for them only where it joins.
+    cudaStream_t xs[2] = {nullptr, nullptr};
+    cudaEvent_t ev_xs[2] = {nullptr, nullptr}, ev_data = nullptr;
+    bool xs_busy[2] = {false, false};   // stream k has work the caller's stream has not waited for
+    int xs_steps[2] = {0, 0};           // block sizes of that work (ring slots it still reads)
+    int xs_next = 0;
+    int scratch_sel = 0;                // which split scratch the next launch uses
     cudaStream_t tail = nullptr;
     cudaEvent_t ev_x = nullptr, ev_w = nullptr, ev_e = nullptr;
+    bool ensure_xs() {
+        if (xs[0]) return true;
+        if (!ensure_tail()) return false;
+        bool ok = cudaStreamCreateWithFlags(&xs[0], cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&xs[1], cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&ev_xs[0], cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&ev_xs[1], cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&ev_data, cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            for (int k = 0; k < 2; ++k) {
+                if (xs[k]) cudaStreamDestroy(xs[k]);
+                if (ev_xs[k]) cudaEventDestroy(ev_xs[k]);
+                xs[k] = nullptr;
+                ev_xs[k] = nullptr;
+            }
+            if (ev_data) cudaEventDestroy(ev_data);
+            ev_data = nullptr;
+        }
+        return ok;
+    }
+    // Ring slots (in steps, counted back from the newest) that work not yet joined still reads.
+    int protected_steps() const {
+        int n = pending ? pending_n : 0;
+        const int x = (xs_busy[0] ? xs_steps[0] : 0) + (xs_busy[1] ? xs_steps[1] : 0);
+        return n > x ? n : x;
+    }
     bool ensure_tail() {
         if (tail) return true;
         if (!ensure_side()) return false;
@@ -157,10 +194,23 @@ struct guard_ctx {
     }
     // Makes `st` wait for the pending evaluation, if any.
     cudaError_t join(cudaStream_t st) {
-        if (!pending) return cudaSuccess;
-        cudaError_t e = cudaStreamWaitEvent(st, ev_e, 0);
-        if (e == cudaSuccess) pending = false;
+        cudaError_t e = cudaSuccess;
+        if (pending) {
+            e = cudaStreamWaitEvent(st, ev_e, 0);
+            if (e == cudaSuccess) pending = false;
+        }
         return e;
+    }
+    // Makes `st` wait for the cross-rank kernels still running on the internal ingest streams.
+    cudaError_t join_xs(cudaStream_t st) {
+        for (int k = 0; k < 2; ++k)
+            if (xs_busy[k]) {
+                cudaError_t e = cudaStreamWaitEvent(st, ev_xs[k], 0);
+                if (e != cudaSuccess) return e;
+                xs_busy[k] = false;
+                xs_steps[k] = 0;
+            }
+        return cudaSuccess;
     }
     int profiling = 0;                                        // 1: time the MAD sweep of every ingest, 2: the window kernel of every evaluation
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof;    // recorded, not yet read
@@ -197,7 +247,7 @@ struct guard_ctx {
                 g.mad = a.mad + (size_t)s0 * M;
                 if (a.med_user) g.med_user = a.med_user + (size_t)s0 * M;
                 if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
-                cudaError_t e = launch_xrank_split(g, p, n, ws + L.xr_big, status() + 2, st,
+                cudaError_t e = launch_xrank_split(g, p, n, ws + (scratch_sel ? L.xr_big2 : L.xr_big), status() + 2, st,
                                                    (profiling == 1 && a.mask_base) ? &prof : nullptr);
                 if (e != cudaSuccess) return e;
                 launches += 6;
@@ -293,8 +343,8 @@ int guard_ring_reserve(guard_ctx *c, int steps, float **d_slot) {
     if (!d_slot || steps < 1 || steps > c->C) return c->fail(GUARD_ERR_ARG, "steps must be in 1..capacity and d_slot non-NULL");
     const int slot = (int)(c->seen % c->C);
     if (slot + steps > c->C) return c->fail(GUARD_ERR_ARG, "reserved span would wrap around the ring (slot %d + %d > %d)", slot, steps, c->C);
-    if (c->pending && steps + c->pending_n > c->C)
-        return c->fail(GUARD_ERR_NOT_READY, "the reserved slots belong to the window of the deferred evaluation still pending: call guard_join first");
+    if (steps + c->protected_steps() > c->C)
+        return c->fail(GUARD_ERR_NOT_READY, "the reserved slots are still read by deferred work: call guard_join first");
     *d_slot = c->ring() + (size_t)slot * c->R * c->M;
     return GUARD_OK;
 }
@@ -307,9 +357,10 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
     const size_t row = (size_t)c->R * c->M;
     const int slot = (int)(c->seen % c->C);
     const bool in_place = (d_block == c->ring() + (size_t)slot * row) && (slot + B <= c->C);
-    if (c->pending && B + c->pending_n > c->C) {   // this block's slots are read by the pending evaluation
+    if (B + c->protected_steps() > c->C) {   // this block's slots are still read by deferred work
         cudaError_t e = c->join(st);
-        if (e != cudaSuccess) return c->cuda_fail(e, "join of the deferred evaluation");
+        if (e == cudaSuccess) e = c->join_xs(st);
+        if (e != cudaSuccess) return c->cuda_fail(e, "join of deferred work");
     }
     if (!in_place) {
         const int first = (slot + B <= c->C) ? B : (c->C - slot);
@@ -339,7 +390,25 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
     a.mask_bytes = c->mask_bytes();
     a.check_finite = 1;
     a.status = c->status();
-    cudaError_t e = c->xrank(a, B, st);
+    cudaError_t e;
+    const bool piped = c->deferred && c->L.xr_split && a.mask_bytes == 1 && (long long)B * c->M > 64 && !d_step_med &&
+                       !d_step_mad && c->ensure_xs();
+    if (piped) {
+        const int k = c->xs_next;
+        c->xs_next ^= 1;
+        e = cudaEventRecord(c->ev_data, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(c->xs[k], c->ev_data, 0);
+        if (e != cudaSuccess) return c->cuda_fail(e, "fork of the ingest stream");
+        c->scratch_sel = k;
+        e = c->xrank(a, B, c->xs[k]);
+        c->scratch_sel = 0;
+        if (e == cudaSuccess) e = cudaEventRecord(c->ev_xs[k], c->xs[k]);
+        c->xs_busy[k] = true;
+        c->xs_steps[k] = B;
+    } else {
+        e = c->join_xs(st);   // earlier blocks still on the internal streams come first
+        if (e == cudaSuccess) e = c->xrank(a, B, st);
+    }
     if (e != cudaSuccess) return c->cuda_fail(e, "xrank launch");
     c->seen += B;
     return GUARD_OK;
@@ -380,6 +449,10 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     const bool forked = c->overlap && c->fork_fresh && c->side;
     c->fork_fresh = false;
     const bool defer = c->deferred && c->ensure_tail();
+    if (!defer) {
+        e = c->join_xs(st);
+        if (e != cudaSuccess) return c->cuda_fail(e, "join of the ingest streams");
+    }
     cudaStream_t ts = st;   // stream of the evaluation's tail: fleet baseline, scores / flags, top-k
     if (defer) {
         // window medians on the internal stream (after the ring is complete and after the previous
@@ -397,6 +470,8 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_x, st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_w, 0);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_x, 0);
+        for (int k = 0; k < 2 && e == cudaSuccess; ++k)   // cross-rank kernels of the window's blocks on the ingest streams
+            if (c->xs_busy[k]) e = cudaStreamWaitEvent(c->tail, c->ev_xs[k], 0);
         ts = c->tail;
     } else if (forked) {
         e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
@@ -570,6 +645,7 @@ int guard_sync_status(guard_ctx *c, void *stream) {
     if (!c) return GUARD_ERR_ARG;
     uint32_t s = 0;
     cudaError_t e = c->join((cudaStream_t)stream);
+    if (e == cudaSuccess) e = c->join_xs((cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(&s, c->status(), sizeof(s), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "guard_sync_status");
@@ -581,6 +657,7 @@ int guard_sync_status(guard_ctx *c, void *stream) {
 int guard_reset(guard_ctx *c, void *stream) {
     if (!c) return GUARD_ERR_ARG;
     cudaError_t e = c->join((cudaStream_t)stream);
+    if (e == cudaSuccess) e = c->join_xs((cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->ws, 0, c->L.wmed, (cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "cudaMemsetAsync");
     c->seen = 0;
@@ -622,7 +699,9 @@ int64_t guard_kernel_launches(const guard_ctx *c) { return c ? c->launches : 0; 
 
 int guard_fallback_reasons(guard_ctx *c, uint32_t out[6], void *stream) {
     if (!c || !out) return GUARD_ERR_ARG;
-    cudaError_t e = cudaMemcpyAsync(out, c->status() + 2, 6 * sizeof(uint32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    cudaError_t e = c->join((cudaStream_t)stream);
+    if (e == cudaSuccess) e = c->join_xs((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out, c->status() + 2, 6 * sizeof(uint32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "guard_fallback_reasons");
     return GUARD_OK;
@@ -631,7 +710,9 @@ int guard_fallback_reasons(guard_ctx *c, uint32_t out[6], void *stream) {
 int64_t guard_fallback_steps(guard_ctx *c, void *stream) {
     if (!c) return GUARD_ERR_ARG;
     uint32_t n = 0;
-    cudaError_t e = cudaMemcpyAsync(&n, c->status() + 1, sizeof(n), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    cudaError_t e = c->join((cudaStream_t)stream);
+    if (e == cudaSuccess) e = c->join_xs((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&n, c->status() + 1, sizeof(n), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "guard_fallback_steps");
     return (int64_t)n;
@@ -646,6 +727,7 @@ int guard_set_deferred(guard_ctx *c, int on) {
 int guard_join(guard_ctx *c, void *stream) {
     if (!c) return GUARD_ERR_ARG;
     cudaError_t e = c->join((cudaStream_t)stream);
+    if (e == cudaSuccess) e = c->join_xs((cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "guard_join");
     return GUARD_OK;
 }
@@ -660,6 +742,13 @@ int guard_set_overlap(guard_ctx *c, int on) {
 void guard_destroy(guard_ctx *c) {
     if (c) {
         guard_profile_enable(c, 0);
+        for (int k = 0; k < 2; ++k)
+            if (c->xs[k]) {
+                cudaStreamSynchronize(c->xs[k]);
+                cudaStreamDestroy(c->xs[k]);
+                cudaEventDestroy(c->ev_xs[k]);
+            }
+        if (c->ev_data) cudaEventDestroy(c->ev_data);
         if (c->tail) {
             cudaStreamSynchronize(c->tail);
             cudaStreamDestroy(c->tail);
