@@ -253,6 +253,36 @@ def test_large_configuration_sampled_blocks():
         run_both(X, cfg.W, cfg.k, cfg.topk, synth.fleet_dir(cfg.metrics), [cfg.block], capacity=cfg.block, in_place=True)
 
 
+def test_large_configuration_bench_pipeline():
+    """The launch configuration bench.py times: 16 384 ranks x 8 metrics, blocks of 200 steps written
+    in place, deferred mode (evaluations and consecutive ingests on internal streams), a ring of
+    several blocks.  Three consecutive blocks, every evaluation compared in full with the oracle:
+    the second and third run the thread-per-series window kernel at full width."""
+    from paper_2605_17879_b200 import guard
+    cfg = synth.paper_configs()["large"]
+    R, M, B, nb = cfg.ranks, cfg.metrics, cfg.block, 3
+    dirs = synth.fleet_dir(M)
+    g = guard.Guard(R, M, cfg.W, cfg.k, dir=dirs, capacity=nb * B, topk=cfg.topk)
+    g.set_deferred(True)
+    o = go.Oracle(R, M, cfg.W, cfg.k, cfg.topk, dir=dirs)
+    ring = g.ring_reserve(nb * B)
+    for j in range(nb):
+        synth.fleet_block(cfg, j * B, (j + 1) * B, device="cuda", out=ring[j * B:(j + 1) * B])
+    torch.cuda.synchronize()
+    bufs = [g.alloc_outputs() for _ in range(nb)]
+    for j in range(nb):
+        g.ingest(ring[j * B:(j + 1) * B])
+        g.score(bufs[j])
+    g.join()
+    g.sync_status()
+    assert g.fallback_steps() == 0
+    Xh = ring.cpu().numpy()
+    for j in range(nb):
+        o.ingest(Xh[j * B:(j + 1) * B])
+        compare_score(bufs[j], o.score(), "block %d" % j)
+    g.close()
+
+
 def test_streaming_configuration_prefix():
     """32 768 ranks, one step per ingest into a 512-step ring; every step's cross-rank
     statistics are compared, evaluations at a few steps (an oracle evaluation sorts 262 144
