@@ -105,21 +105,32 @@ __global__ void __launch_bounds__(kFastWarps * 32) score_flag_bytes_kernel(const
 #pragma unroll
         for (int m = 0; m < 8; ++m) sums[q][m] = 0;
     int pending = 0;
-    for (int j = w; j < a.n; j += kFastWarps) {
-        int slot = first + j;
-        if (slot >= a.capacity) slot -= a.capacity;
-        const uint8_t *rowp = mask_base + (size_t)slot * a.R;
-        uint32_t word = 0;
-        if (word_ok) {
-            word = *reinterpret_cast<const uint32_t *>(rowp + rq);
-        } else {
+    constexpr int KU = 5;   // window steps whose loads are in flight together
+    for (int j0 = w; j0 < a.n; j0 += kFastWarps * KU) {
+        uint32_t word[KU];
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (rq + q < a.R) word |= (uint32_t)rowp[rq + q] << (8 * q);
+        for (int u = 0; u < KU; ++u) {
+            const int j = j0 + u * kFastWarps;
+            word[u] = 0;
+            if (j < a.n) {
+                int slot = first + j;
+                if (slot >= a.capacity) slot -= a.capacity;
+                const uint8_t *rowp = mask_base + (size_t)slot * a.R;
+                if (word_ok) {
+                    word[u] = __ldg(reinterpret_cast<const uint32_t *>(rowp + rq));
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (rq + q < a.R) word[u] |= (uint32_t)rowp[rq + q] << (8 * q);
+                }
+            }
         }
 #pragma unroll
-        for (int m = 0; m < 8; ++m) acc[m] += (word >> m) & 0x01010101u;
-        if (++pending == 255) {   // byte lanes are about to overflow: spill into the wide sums
+        for (int u = 0; u < KU; ++u)
+#pragma unroll
+            for (int m = 0; m < 8; ++m) acc[m] += (word[u] >> m) & 0x01010101u;
+        pending += KU;
+        if (pending > 255 - KU) {   // byte lanes are about to overflow: spill into the wide sums
 #pragma unroll
             for (int q = 0; q < 4; ++q)
 #pragma unroll
