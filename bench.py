@@ -10,8 +10,8 @@ evaluation (windowed medians, fleet baseline, scores/flags/tiers, top-64) after 
 Prints ONE JSON line.  `value` is cells scored per second with the telemetry already
 resident in HBM (written in place into the library's ring before the timed region);
 `e2e` is the same metric with the telemetry in pinned HOST memory, copied block by block
-into the ring inside the timed region, and the flags / top-k read back to the host after
-every evaluation.  With N > 1 every rank runs an independent replica (the path does not
+into the ring inside the timed region (on a copy stream, one block ahead of the scoring),
+and the flags / top-k of every evaluation read back to the host.  With N > 1 every rank runs an independent replica (the path does not
 shard: a cross-rank median needs all ranks of a step on one GPU).
 
 `--impl reference` times the CPU oracle (oracle/, single thread, as it stands) on a
@@ -339,18 +339,34 @@ def main():
     h_sc = torch.empty(cfg.topk, dtype=torch.float32, pin_memory=True)
     torch.cuda.synchronize()
 
-    g.set_deferred(False)   # the end-to-end pass reads every evaluation's flags back at once
+    # End to end: block j + 1 is copied from pinned host memory on a copy stream while block j is
+    # ingested and evaluated (deferred mode); the flags and top-k of every evaluation are read back to
+    # the host as soon as that evaluation has been joined (by the next score(), or the final join()).
+    copy_stream = torch.cuda.Stream(device=dev)
+    copied = [torch.cuda.Event() for _ in range(n_blocks)]
+    outs2 = [out, g.alloc_outputs()]
+
+    def read_back(o):
+        h_flags.copy_(o["flags"], non_blocking=True)
+        h_idx.copy_(o["topk_idx"], non_blocking=True)
+        h_sc.copy_(o["topk_score"], non_blocking=True)
 
     def one_pass_e2e():
         g.reset()
+        main = torch.cuda.current_stream()
+        copy_stream.wait_stream(main)   # the ring is free again: everything of the previous pass has been joined
+        with torch.cuda.stream(copy_stream):
+            for j in range(n_blocks):
+                ring[j * B:(j + 1) * B].copy_(host[j * B:(j + 1) * B], non_blocking=True)
+                copied[j].record(copy_stream)
         for j in range(n_blocks):
-            slot = g.ring_reserve(B)
-            slot.copy_(host[j * B:(j + 1) * B], non_blocking=True)
-            g.ingest(slot)
-            g.score(out)
-            h_flags.copy_(out["flags"], non_blocking=True)
-            h_idx.copy_(out["topk_idx"], non_blocking=True)
-            h_sc.copy_(out["topk_score"], non_blocking=True)
+            main.wait_event(copied[j])
+            g.ingest(ring[j * B:(j + 1) * B])
+            g.score(outs2[j % 2])       # joins evaluation j - 1
+            if j > 0:
+                read_back(outs2[(j - 1) % 2])
+        g.join()
+        read_back(outs2[(n_blocks - 1) % 2])
 
     e2e = None
     if args.e2e_steps > 0:
