@@ -118,6 +118,7 @@ struct guard_ctx {
     long long seen;
     long long launches;  // kernels enqueued by this context so far
     long long evals;     // evaluations since creation / reset
+    long long seen_at_eval = 0;   // steps seen at the last evaluation
     // overlap of the window medians (which need only the ring) with the cross-rank kernels of the
     // ingest that precedes them: an internal stream forked from and joined into the caller's
     bool overlap = true;
@@ -436,6 +437,10 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     w.use_hint = c->evals > 0 ? 1 : 0;
     w.spread = (float *)(c->ws + c->L.wspread);
     w.centre = (float *)(c->ws + c->L.wcentre);
+    // windows that share at least three quarters of their steps with the previous evaluation's: the
+    // previous median itself is the centre, and a much narrower interval does
+    if (c->evals > 0 && (c->seen - c->seen_at_eval) * 4 <= n) { w.target = kWindowNearTarget; w.smooth = kWindowNearSmooth; }
+    c->seen_at_eval = c->seen;
     w.fb_count = c->status() + 8;
     w.status = c->status();
     // The window medians read only the ring: run them on the internal stream, forked where the
@@ -662,6 +667,7 @@ int guard_reset(guard_ctx *c, void *stream) {
     if (e != cudaSuccess) return c->cuda_fail(e, "cudaMemsetAsync");
     c->seen = 0;
     c->evals = 0;
+    c->seen_at_eval = 0;
     return GUARD_OK;
 }
 

@@ -54,6 +54,10 @@ cudaError_t launch_xrank_cluster(const XrankArgs &a, const MetricParams &p, int 
 // Six uniform kernels per block (sample, sweep, select, sweep, select, finish) with the kept
 // elements in global scratch (4 or 8 metrics, a few thousand to ~20 000 ranks).
 bool xrank_split_supported(int R, int M);
+// Thread path of the window medians when consecutive windows share most of their steps (the median
+// hardly moves): keys the interval is tuned to catch, weight of the newest median in its centre.
+constexpr int kWindowNearTarget = 14;
+constexpr float kWindowNearSmooth = 1.0f;
 constexpr int kSplitMaxSteps = 256;   // steps per launch group of the split path (sizes its scratch)
 size_t xrank_split_scratch_bytes(int R, int M, int S_max);
 cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S, void *scratch, uint32_t *reasons,
@@ -81,6 +85,8 @@ struct WindowArgs {
     float *wmed_user;       // or NULL
     float *spread;          // [series] tuned half-width of the thread path's interval (state), or NULL
     float *centre;          // [series] smoothed median: the centre of the thread path's interval (state), or NULL
+    int target;             // number of keys the thread path's interval is tuned to catch (0: default)
+    float smooth;           // weight of the newest median in the interval's centre (0: default)
     uint32_t *fb_count;     // [6] series the thread path's interval did not serve, in total and by reason (diagnostic), or NULL
     uint32_t *status;
 };

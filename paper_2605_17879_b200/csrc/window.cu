@@ -371,7 +371,7 @@ cudaError_t launch_warp_path(const WindowArgs &a, int use_bulk, cudaStream_t st)
 // ---------------------------------------------------------------------------------------
 constexpr int kThCols = 128;     // series per CTA = threads per CTA
 constexpr int kThSlots = 60;     // kept keys per series
-constexpr int kThTarget = 42;    // number of keys the interval is tuned to catch
+constexpr int kThTarget = 42;    // number of keys the interval is tuned to catch (windows that share few steps)
 constexpr int kThRows = 8;       // rows in flight per thread
 constexpr int kThMaxPasses = 12;
 constexpr float kThSmooth = 0.3f;   // weight of the newest median in the interval's centre
@@ -522,9 +522,9 @@ __global__ void __launch_bounds__(kThCols, 7) window_thread_kernel(const WindowA
         if (a.wmed_user) a.wmed_user[c] = med;
         // re-tune the half-width so that the interval catches about kThTarget keys next time
         // (half of the way: one window's count is a noisy estimate of the density)
-        const float f = fminf(2.0f, fmaxf(0.5f, (float)kThTarget / (float)max(nk, 1)));
+        const float f = fminf(2.0f, fmaxf(0.5f, (float)(a.target > 0 ? a.target : kThTarget) / (float)max(nk, 1)));
         a.spread[c] = h * (0.5f + 0.5f * f);
-        a.centre[c] = hint + kThSmooth * (med - hint);
+        a.centre[c] = hint + (a.smooth > 0.0f ? a.smooth : kThSmooth) * (med - hint);
     }
     // ---- series the interval did not serve: the whole warp finishes them one by one ------------
     unsigned todo = __ballot_sync(0xFFFFFFFFu, active && !ok);
