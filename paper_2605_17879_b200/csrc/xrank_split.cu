@@ -351,12 +351,12 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
             if (!guard || base + j * LPI + rl < r1) x = __ldg(src + (size_t)j * LPI * NQ);
             v[j][0] = x.x; v[j][1] = x.y; v[j][2] = x.z; v[j][3] = x.w;
         }
-        if (guard) {   // ranks beyond the end: neither below nor inside any interval, never "slow"
+        if (guard) {   // ranks beyond the end: +inf is neither below nor inside any interval; never "slow"
 #pragma unroll
             for (int j = 0; j < kSpU; ++j)
                 if (base + j * LPI + rl >= r1) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) v[j][c] = MODE == 0 ? CUDART_NAN_F : __fmul_rn(sg[c], -nsm[c]);   // MODE 1: x = med
+                    for (int c = 0; c < 4; ++c) v[j][c] = MODE == 0 ? CUDART_INF_F : __fmul_rn(sg[c], -nsm[c]);   // MODE 1: x = med
                 }
         }
         uint32_t packed = 0;
@@ -401,7 +401,7 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
                 }
                 if (guard && base + j * LPI + rl >= r1) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) v[j][c] = CUDART_NAN_F;
+                    for (int c = 0; c < 4; ++c) v[j][c] = CUDART_INF_F;
                 }
             }
             sp_cell_count<1u>(v[j][0], lo[0], hi[0], cnt[0], packed);

@@ -61,7 +61,7 @@ def compare_score(gout, oout, what=""):
         assert_scores_close(to_np(gout["topk_score"]), oout["topk_score"], what + " topk_score")
 
 
-def run_both(X, W, k, K, dirs, blocks, capacity=None, score_every=1, in_place=False, **kw):
+def run_both(X, W, k, K, dirs, blocks, capacity=None, score_every=1, in_place=False, max_fallback_steps=None, **kw):
     """Feeds X [T, R, M] (numpy float32) to both sides in the given block sizes and
     compares after every `score_every`-th block.  Returns the last oracle result."""
     from paper_2605_17879_b200 import guard
@@ -94,5 +94,8 @@ def run_both(X, W, k, K, dirs, blocks, capacity=None, score_every=1, in_place=Fa
             g.sync_status()
             last = o.score()
             compare_score(gout, last, "t=%d" % t)
+    if max_fallback_steps is not None:
+        # the fast cross-rank paths must have served the steps themselves, not the direct fallback
+        assert g.fallback_steps() <= max_fallback_steps, g.fallback_steps()
     g.close()
     return last

@@ -80,7 +80,9 @@ def test_bracketed_cross_rank_path(R, M, W, T, quant):
 ])
 def test_wide_block_cross_rank_paths(R, M, B, T, quant):
     X, dirs = _rand_fleet(T, R, M, seed=3 * R + M, quant=quant)
-    run_both(X, B, max(1, B // 2), 16, dirs, [B], capacity=2 * B, min_signals=2)
+    # continuous data must be served by the fast path itself (ragged chunks included), not by the fallback
+    run_both(X, B, max(1, B // 2), 16, dirs, [B], capacity=2 * B, min_signals=2,
+             max_fallback_steps=0 if quant is None else None)
 
 
 def test_wide_block_degenerate_columns():
