@@ -594,7 +594,7 @@ __device__ bool sp_select_regs(const uint32_t *__restrict__ list, const int cap,
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(kSpSelThreads) xsplit_select_kernel(const XrankArgs a, const MetricParams p, const SpGeom g,
+__global__ void __launch_bounds__(kSpSelThreads, 12) xsplit_select_kernel(const XrankArgs a, const MetricParams p, const SpGeom g,
                                                                       const SpScratch sc, uint32_t *reasons) {
     __shared__ SpSelShared sh;
     __shared__ uint32_t s_fail;
