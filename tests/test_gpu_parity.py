@@ -75,6 +75,7 @@ def test_bracketed_cross_rank_path(R, M, W, T, quant):
     (4100, 8, 9, 27, None),        # rank count not a multiple of 16: partial batches
     (16384, 8, 10, 20, None),      # width of the large configuration
     (20000, 8, 9, 9, None),        # beyond the split path's kept-list size: cluster path
+    (32768, 8, 9, 9, None),        # cluster path with kept lists too long for its register selection
     (4096, 8, 12, 24, 50),         # quantised: intervals collapse onto tied values
     (8192, 4, 20, 20, 4),          # very coarse: kept lists overflow, every step takes the direct path
 ])
