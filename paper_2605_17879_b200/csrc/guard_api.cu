@@ -14,10 +14,14 @@ using namespace guard;
 namespace {
 
 constexpr size_t kAlign = 256;
+#ifndef GUARD_INGEST_STREAMS
+#define GUARD_INGEST_STREAMS 2
+#endif
+constexpr int kIngestStreams = GUARD_INGEST_STREAMS;   // internal streams the cross-rank kernels of consecutive blocks take turns on (deferred mode)
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, xr_big, xr_big2, mask, ring, total;
+    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, xr_big, xr_big_stride, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
@@ -42,8 +46,9 @@ Layout make_layout(int R, int M, int C, int K) {
     L.wcentre = off;   off = align_up(off + (size_t)R * M * sizeof(float));
     L.xr_big = off;    off = align_up(off + (L.xr_split ? xrank_split_scratch_bytes(R, M, C < kSplitMaxSteps ? C : kSplitMaxSteps)
                                              : L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps) : 0));
-    // a second scratch: in deferred mode consecutive blocks run their cross-rank kernels on two streams
-    L.xr_big2 = off;   off = align_up(off + (L.xr_split ? xrank_split_scratch_bytes(R, M, C < kSplitMaxSteps ? C : kSplitMaxSteps) : 0));
+    // in deferred mode consecutive blocks run their cross-rank kernels on streams of their own
+    L.xr_big_stride = off - L.xr_big;   // further copies of the split scratch, one per internal ingest stream
+    off = align_up(off + (L.xr_split ? (kIngestStreams - 1) * L.xr_big_stride : 0));
     L.mask = off;      off = align_up(off + (size_t)C * R * (M <= 8 ? 1 : 4));
     L.ring = off;      off = align_up(off + (size_t)C * R * M * sizeof(float));
     L.total = off;
@@ -146,10 +151,10 @@ struct guard_ctx {
     // In deferred mode the cross-rank kernels of consecutive ingests alternate between two internal
     // streams (each with its own scratch), so that one block's selections overlap the next block's
     // sweeps; the caller's stream waits for them only where it joins.
-    cudaStream_t xs[2] = {nullptr, nullptr};
-    cudaEvent_t ev_xs[2] = {nullptr, nullptr}, ev_data = nullptr;
-    bool xs_busy[2] = {false, false};   // stream k has work the caller's stream has not waited for
-    int xs_steps[2] = {0, 0};           // block sizes of that work (ring slots it still reads)
+    cudaStream_t xs[kIngestStreams] = {};
+    cudaEvent_t ev_xs[kIngestStreams] = {}, ev_data = nullptr;
+    bool xs_busy[kIngestStreams] = {};   // stream k has work the caller's stream has not waited for
+    int xs_steps[kIngestStreams] = {};   // block sizes of that work (ring slots it still reads)
     int xs_next = 0;
     int scratch_sel = 0;                // which split scratch the next launch uses
     cudaStream_t tail = nullptr;
@@ -157,13 +162,12 @@ struct guard_ctx {
     bool ensure_xs() {
         if (xs[0]) return true;
         if (!ensure_tail()) return false;
-        bool ok = cudaStreamCreateWithFlags(&xs[0], cudaStreamNonBlocking) == cudaSuccess &&
-                  cudaStreamCreateWithFlags(&xs[1], cudaStreamNonBlocking) == cudaSuccess &&
-                  cudaEventCreateWithFlags(&ev_xs[0], cudaEventDisableTiming) == cudaSuccess &&
-                  cudaEventCreateWithFlags(&ev_xs[1], cudaEventDisableTiming) == cudaSuccess &&
-                  cudaEventCreateWithFlags(&ev_data, cudaEventDisableTiming) == cudaSuccess;
+        bool ok = cudaEventCreateWithFlags(&ev_data, cudaEventDisableTiming) == cudaSuccess;
+        for (int k = 0; k < kIngestStreams && ok; ++k)
+            ok = cudaStreamCreateWithFlags(&xs[k], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&ev_xs[k], cudaEventDisableTiming) == cudaSuccess;
         if (!ok) {
-            for (int k = 0; k < 2; ++k) {
+            for (int k = 0; k < kIngestStreams; ++k) {
                 if (xs[k]) cudaStreamDestroy(xs[k]);
                 if (ev_xs[k]) cudaEventDestroy(ev_xs[k]);
                 xs[k] = nullptr;
@@ -177,7 +181,8 @@ struct guard_ctx {
     // Ring slots (in steps, counted back from the newest) that work not yet joined still reads.
     int protected_steps() const {
         int n = pending ? pending_n : 0;
-        const int x = (xs_busy[0] ? xs_steps[0] : 0) + (xs_busy[1] ? xs_steps[1] : 0);
+        int x = 0;
+        for (int k = 0; k < kIngestStreams; ++k) x += xs_busy[k] ? xs_steps[k] : 0;
         return n > x ? n : x;
     }
     bool ensure_tail() {
@@ -204,7 +209,7 @@ struct guard_ctx {
     }
     // Makes `st` wait for the cross-rank kernels still running on the internal ingest streams.
     cudaError_t join_xs(cudaStream_t st) {
-        for (int k = 0; k < 2; ++k)
+        for (int k = 0; k < kIngestStreams; ++k)
             if (xs_busy[k]) {
                 cudaError_t e = cudaStreamWaitEvent(st, ev_xs[k], 0);
                 if (e != cudaSuccess) return e;
@@ -248,7 +253,7 @@ struct guard_ctx {
                 g.mad = a.mad + (size_t)s0 * M;
                 if (a.med_user) g.med_user = a.med_user + (size_t)s0 * M;
                 if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
-                cudaError_t e = launch_xrank_split(g, p, n, ws + (scratch_sel ? L.xr_big2 : L.xr_big), status() + 2, st,
+                cudaError_t e = launch_xrank_split(g, p, n, ws + L.xr_big + (size_t)scratch_sel * L.xr_big_stride, status() + 2, st,
                                                    (profiling == 1 && a.mask_base) ? &prof : nullptr);
                 if (e != cudaSuccess) return e;
                 launches += 6;
@@ -396,7 +401,7 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
                        !d_step_mad && c->ensure_xs();
     if (piped) {
         const int k = c->xs_next;
-        c->xs_next ^= 1;
+        c->xs_next = (k + 1) % kIngestStreams;
         e = cudaEventRecord(c->ev_data, st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(c->xs[k], c->ev_data, 0);
         if (e != cudaSuccess) return c->cuda_fail(e, "fork of the ingest stream");
@@ -475,7 +480,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_x, st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_w, 0);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_x, 0);
-        for (int k = 0; k < 2 && e == cudaSuccess; ++k)   // cross-rank kernels of the window's blocks on the ingest streams
+        for (int k = 0; k < kIngestStreams && e == cudaSuccess; ++k)   // cross-rank kernels of the window's blocks on the ingest streams
             if (c->xs_busy[k]) e = cudaStreamWaitEvent(c->tail, c->ev_xs[k], 0);
         ts = c->tail;
     } else if (forked) {
@@ -748,7 +753,7 @@ int guard_set_overlap(guard_ctx *c, int on) {
 void guard_destroy(guard_ctx *c) {
     if (c) {
         guard_profile_enable(c, 0);
-        for (int k = 0; k < 2; ++k)
+        for (int k = 0; k < kIngestStreams; ++k)
             if (c->xs[k]) {
                 cudaStreamSynchronize(c->xs[k]);
                 cudaStreamDestroy(c->xs[k]);
