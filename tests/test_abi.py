@@ -75,6 +75,8 @@ def test_create_rejects_bad_arguments_on_the_host(glib):
     # NULL context is tolerated everywhere
     assert L.guard_ingest(None, None, 1, None, None, None) == -1
     assert L.guard_sync_status(None, None) == -1
+    assert L.guard_set_deferred(None, 1) == -1
+    assert L.guard_join(None, None) == -1
     L.guard_destroy(None)
     assert L.guard_steps_seen(None) == 0
 
