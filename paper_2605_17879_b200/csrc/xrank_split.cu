@@ -1,5 +1,5 @@
 // Cross-rank selection, split path: six uniform kernels per ingested block, for fleets of a
-// few thousand to some twenty thousand ranks with 4 or 8 metrics.  Every kernel does one kind
+// few thousand to about sixteen thousand ranks with 4 or 8 metrics.  Every kernel does one kind
 // of work on many small CTAs, so that the streaming sweeps run with all their warps streaming
 // and the short, latency-bound selections of hundreds of columns overlap one another:
 //
@@ -49,7 +49,7 @@ constexpr float kFltMax = 3.402823466e+38f;
 struct SpGeom {
     int chunks;     // sweep CTAs per step
     int slice;      // ranks per sweep CTA (a multiple of 16)
-    int cap;        // kept elements per metric and sweep CTA (shared memory)
+    int cap;        // kept elements per metric and sweep CTA (its shared-memory list and its segment in global scratch)
     int stride;     // one run of four consecutive ranks is sampled out of every 4 * stride
     int s;          // number of sampled ranks
     int delta;      // half-width of the median interval in sample ranks
