@@ -14,6 +14,9 @@ using namespace guard;
 namespace {
 
 constexpr size_t kAlign = 256;
+#ifndef GUARD_EVAL_PRIO
+#define GUARD_EVAL_PRIO 1
+#endif
 #ifndef GUARD_INGEST_STREAMS
 #define GUARD_INGEST_STREAMS 2
 #endif
@@ -132,7 +135,10 @@ struct guard_ctx {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     bool ensure_side() {
         if (side) return true;
-        if (cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking) != cudaSuccess) { side = nullptr; return false; }
+        // the evaluation's streams get the highest priority: flags should not queue behind the next blocks' sweeps
+        int prio_lo = 0, prio_hi = 0;
+        cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+        if (cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, GUARD_EVAL_PRIO ? prio_hi : 0) != cudaSuccess) { side = nullptr; return false; }
         if (cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming) != cudaSuccess) {
             cudaStreamDestroy(side);
@@ -188,7 +194,9 @@ struct guard_ctx {
     bool ensure_tail() {
         if (tail) return true;
         if (!ensure_side()) return false;
-        if (cudaStreamCreateWithFlags(&tail, cudaStreamNonBlocking) != cudaSuccess) { tail = nullptr; return false; }
+        int prio_lo = 0, prio_hi = 0;
+        cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+        if (cudaStreamCreateWithPriority(&tail, cudaStreamNonBlocking, GUARD_EVAL_PRIO ? prio_hi : 0) != cudaSuccess) { tail = nullptr; return false; }
         if (cudaEventCreateWithFlags(&ev_x, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&ev_w, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&ev_e, cudaEventDisableTiming) != cudaSuccess) {
