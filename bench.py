@@ -37,7 +37,7 @@ UNIT = "cells/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this workload, from
 # the ncu capture summarised under profiles/ (None once the kernel has changed since the capture)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 116.1e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 116.14e6
 # which kernel the roofline object describes: 2 = window_thread_kernel (guard_score), 1 = the MAD sweep (guard_ingest)
 PROFILE_MODE = 2
 PROFILE_KERNEL = ("window_thread_kernel (windowed per-rank medians of one evaluation)" if PROFILE_MODE == 2 else

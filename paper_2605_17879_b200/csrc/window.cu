@@ -401,7 +401,7 @@ __device__ __forceinline__ void th_sts4(const uint32_t addr, const uint4 v) {
 }
 
 template <int VPL>
-__global__ void __launch_bounds__(kThCols, 7) window_thread_kernel(const WindowArgs a) {
+__global__ void __launch_bounds__(kThCols, 9) window_thread_kernel(const WindowArgs a) {
     extern __shared__ __align__(16) uint32_t tkept[];   // [kThCols][kThSlots]
     const int tid = threadIdx.x, lane = lane_id();
     const int n = a.n;
