@@ -118,6 +118,7 @@ class Brute:
             masks.append(mask)
             flags.append(int(flag))
             tiers.append(t)
+        self.last = (list(flags), list(tiers), n)
         keyf = lambda r: _order_key(F(-wmed[r][p]) if self.dir[p] < 0 else wmed[r][p])
         order = sorted(range(R), key=lambda r: (tuple(-c for c in keyf(r)), r))
         return {
@@ -126,6 +127,29 @@ class Brute:
             "mask": np.array(masks, np.uint32), "flags": np.array(flags, np.uint8),
             "tier": np.array(tiers, np.uint8), "topk_idx": np.array(order[: self.topk], np.int32),
         }
+
+
+def node_verdict(b: "Brute", rpn: int):
+    """Node-level fold of the last Brute.score(): any rank flagged, highest tier, and the number of
+    window steps in which all ranks of the node exceeded on the primary metric together."""
+    flags, tiers, n = b.last
+    wexc = b.exc[-n:]
+    nf, nt, ns = [], [], []
+    for nd in range(b.R // rpn):
+        rs = range(nd * rpn, (nd + 1) * rpn)
+        nf.append(int(any(flags[r] for r in rs)))
+        nt.append(max(tiers[r] for r in rs))
+        ns.append(sum(1 for e in wexc if all(e[r][b.primary] for r in rs)))
+    return {"node_flag": np.array(nf, np.uint8), "node_tier": np.array(nt, np.uint8),
+            "node_stall": np.array(ns, np.uint16)}
+
+
+def triage(times, period, limit):
+    """Per entry: does the node reach `limit` triage entries no more than `period` apart?"""
+    out = []
+    for i, t in enumerate(times):
+        out.append(int(sum(1 for u in times[: i + 1] if t - u <= period) >= limit))
+    return out
 
 
 def sweep(S: np.ndarray, nodes: int, gpn: int, dir, thr, floor_rel, floor_abs, pct_ppm: int):

@@ -52,6 +52,8 @@ typedef struct {
     unsigned char *exc;  /* per-step exceedance of the last W steps: exc[step % W][r][m] */
     long long seen;      /* steps ingested so far */
     unsigned char *consec; /* consecutive evaluations in which rank r was a candidate */
+    unsigned char *last_flag, *last_tier; /* per-rank flag / tier of the last evaluation */
+    long long eval_seen;   /* steps seen when that evaluation ran (-1: none yet) */
 } oracle_t;
 
 /* ---- order statistics -------------------------------------------------------------- */
@@ -152,18 +154,22 @@ oracle_t *oracle_create(int R, int M, int W, int k, int topk, int primary, int m
     o->hist = (float *)calloc((size_t)W * R * M, sizeof(float));
     o->exc = (unsigned char *)calloc((size_t)W * R * M, 1);
     o->consec = (unsigned char *)calloc((size_t)R, 1);
+    o->last_flag = (unsigned char *)calloc((size_t)R, 1);
+    o->last_tier = (unsigned char *)calloc((size_t)R, 1);
+    o->eval_seen = -1;
     return o;
 }
 
 void oracle_destroy(oracle_t *o)
 {
     if (!o) return;
-    free(o->hist); free(o->exc); free(o->consec); free(o);
+    free(o->hist); free(o->exc); free(o->consec); free(o->last_flag); free(o->last_tier); free(o);
 }
 
 void oracle_reset(oracle_t *o)
 {
     o->seen = 0;
+    o->eval_seen = -1;
     memset(o->consec, 0, (size_t)o->R);
     memset(o->exc, 0, (size_t)o->W * o->R * o->M);
 }
@@ -287,6 +293,8 @@ int oracle_score(oracle_t *o, float *wmed_out, float *fleet_med, float *fleet_ma
         if (mask_out) mask_out[r] = mask;
         if (flags) flags[r] = (unsigned char)flag;
         if (tier) tier[r] = (unsigned char)t;
+        o->last_flag[r] = (unsigned char)flag;
+        o->last_tier[r] = (unsigned char)t;
         float key = wmed[(size_t)r * M + p];
         if (o->dir[p] < 0) key = -key;
         keys[r].key = key;
@@ -304,7 +312,72 @@ int oracle_score(oracle_t *o, float *wmed_out, float *fleet_med, float *fleet_ma
             }
         }
     }
+    o->eval_seen = o->seen;
     free(keys); free(wmed); free(tmp); free(tmp2); free(col);
+    return 0;
+}
+
+/* Node-level verdict of the last evaluation.  The paper acts on nodes, not on single
+ * GPUs (Section 4.2: a flagged node leaves the pool; Section 7.1: 8 GPUs per node), so
+ * the per-rank results are folded over each group of ranks_per_node consecutive ranks:
+ *   node_flag[n]  = 1 when any rank of node n is flagged;
+ *   node_tier[n]  = the highest response tier among its ranks (0 none, 1 pending
+ *                   verification, 2 mitigate at the next checkpoint, 3 restart now);
+ *   node_stall[n] = in how many steps of the evaluation's window EVERY rank of the node
+ *                   exceeded the step's peer baseline on the primary metric at once
+ *                   (a correlated whole-node stall, as opposed to one slow GPU).
+ * Must follow oracle_score with no ingest in between; R must be a multiple of
+ * ranks_per_node.  Returns -2 when there is no such evaluation, -1 on bad arguments.
+ * Reading: the paper says only that the node is the unit; OR / max / all-ranks-at-once
+ * are this file's reading of that. */
+int oracle_node_verdict(oracle_t *o, int ranks_per_node, unsigned char *node_flag, unsigned char *node_tier,
+                        uint16_t *node_stall)
+{
+    const int R = o->R, M = o->M, W = o->W;
+    if (ranks_per_node < 1 || R % ranks_per_node != 0) return -1;
+    if (o->eval_seen < 1 || o->eval_seen != o->seen) return -2;
+    const long n = (long)(o->seen < W ? o->seen : W);
+    const int nodes = R / ranks_per_node;
+    for (int nd = 0; nd < nodes; ++nd) {
+        int any = 0, top = 0;
+        for (int q = 0; q < ranks_per_node; ++q) {
+            const int r = nd * ranks_per_node + q;
+            if (o->last_flag[r]) any = 1;
+            if (o->last_tier[r] > top) top = o->last_tier[r];
+        }
+        int stall = 0;
+        for (long j = 0; j < n; ++j) {
+            long long step = o->seen - n + j;
+            int all = 1;
+            for (int q = 0; q < ranks_per_node; ++q) {
+                const int r = nd * ranks_per_node + q;
+                if (!o->exc[((size_t)(step % W) * R + r) * M + o->primary]) all = 0;
+            }
+            stall += all;
+        }
+        if (node_flag) node_flag[nd] = (unsigned char)any;
+        if (node_tier) node_tier[nd] = (unsigned char)top;
+        if (node_stall) node_stall[nd] = (uint16_t)stall;
+    }
+    return 0;
+}
+
+/* Repeat-offender rule of the triage workflow (Section 6): a node that enters triage
+ * `limit` times within `period` (the paper: three times within a week) is marked for
+ * termination instead of going through triage again.  times[0..n) are the entry times
+ * of ONE node in seconds, non-decreasing.  terminate[i] = 1 when entry i is at least
+ * the limit-th entry of the span [times[i] - period, times[i]] (both ends included:
+ * "within a week" is read as at most one period apart). */
+int oracle_triage(const int64_t *times, int n, int64_t period, int limit, unsigned char *terminate)
+{
+    if (n < 0 || period < 0 || limit < 1) return -1;
+    for (int i = 0; i < n; ++i) {
+        if (i > 0 && times[i] < times[i - 1]) return -1;
+        int c = 0;
+        for (int j = 0; j <= i; ++j)
+            if (times[i] - times[j] <= period) ++c;
+        terminate[i] = (unsigned char)(c >= limit);
+    }
     return 0;
 }
 

@@ -53,6 +53,10 @@ def lib():
         L.oracle_score.restype = C.c_int
         L.oracle_score.argtypes = [C.c_void_p, fp, fp, fp, C.POINTER(C.c_double), C.POINTER(C.c_uint16),
                                    C.POINTER(C.c_uint32), u8p, u8p, C.POINTER(C.c_int32), C.POINTER(C.c_double)]
+        L.oracle_node_verdict.restype = C.c_int
+        L.oracle_node_verdict.argtypes = [C.c_void_p, C.c_int, u8p, u8p, C.POINTER(C.c_uint16)]
+        L.oracle_triage.restype = C.c_int
+        L.oracle_triage.argtypes = [C.POINTER(C.c_int64), C.c_int, C.c_int64, C.c_int, u8p]
         L.oracle_sweep.restype = C.c_int
         L.oracle_sweep.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, i8p, fp, fp, fp, C.c_int,
                                    fp, fp, fp, fp, C.POINTER(C.c_uint32), u8p, u8p]
@@ -143,6 +147,29 @@ class Oracle:
         if rc != 0:
             raise RuntimeError("oracle_score: nothing ingested yet")
         return out
+
+    def node_verdict(self, ranks_per_node: int = 8) -> Dict[str, np.ndarray]:
+        """Node-level fold of the last evaluation (call right after score())."""
+        if ranks_per_node < 1 or self.R % ranks_per_node:
+            raise ValueError("ranks must be a multiple of ranks_per_node")
+        N = self.R // ranks_per_node
+        out = {"node_flag": np.empty(N, np.uint8), "node_tier": np.empty(N, np.uint8),
+               "node_stall": np.empty(N, np.uint16)}
+        rc = lib().oracle_node_verdict(self._h, ranks_per_node, _p(out["node_flag"], C.c_ubyte),
+                                       _p(out["node_tier"], C.c_ubyte), _p(out["node_stall"], C.c_uint16))
+        if rc != 0:
+            raise RuntimeError("oracle_node_verdict: no evaluation of the current window (rc %d)" % rc)
+        return out
+
+
+def triage(times, period: int = 7 * 86400, limit: int = 3) -> np.ndarray:
+    """Entry times (seconds, non-decreasing) of one node -> per entry 1 where the node is to be terminated."""
+    t = np.ascontiguousarray(np.asarray(times, dtype=np.int64))
+    out = np.zeros(t.size, np.uint8)
+    rc = lib().oracle_triage(_p(t, C.c_int64), t.size, period, limit, _p(out, C.c_ubyte))
+    if rc != 0:
+        raise ValueError("oracle_triage rejected the input")
+    return out
 
 
 def sweep(S, nodes: int, gpus_per_node: int, *, dir: Sequence[int], thr=3.5, floor_rel=1e-4, floor_abs=0.0,

@@ -387,3 +387,94 @@ def test_sweep_degraded_gpu_fails_its_node_only():
     clk[7] = 1800.0
     res = go.sweep(clk.astype(np.float32), nodes, gpn, dir=[-1], floor_abs=7.5)
     assert res["gpu_pass"].sum() == nodes * gpn - 1 and res["gpu_pass"][7] == 0
+
+
+# ------------------------------------------------------------------ node-level verdicts (Section 4.2 / 7.1)
+
+@pytest.mark.parametrize("seed", range(8))
+def test_node_verdict_matches_brute_force(seed):
+    rng = np.random.default_rng(500 + seed)
+    rpn = int(rng.integers(1, 5))
+    nodes = int(rng.integers(1, 5))
+    R, M = rpn * nodes, int(rng.integers(1, 4))
+    W = int(rng.integers(1, 7))
+    k = int(rng.integers(1, W + 1))
+    T = int(rng.integers(1, 14))
+    d, thr, frel, fab = _tiny_params(M, rng)
+    prim = int(rng.integers(0, M))
+    kw = dict(primary=prim, min_signals=1, n_consec=1)
+    o = go.Oracle(R, M, W, k, 0, dir=d, thr=thr, floor_rel=frel, floor_abs=fab, **kw)
+    b = brute.Brute(R, M, W, k, 0, d, thr, frel, fab, **kw)
+    X = np.round(rng.normal(1.0, 0.05, (T, R, M)) * 40) / 40
+    X[:, 0, :] *= np.where(np.array(d) > 0, 1.5, 0.6)           # one slow rank: its node must be flagged
+    stall = rng.random((T, nodes)) < 0.3                         # whole-node stalls on the primary metric
+    for t in range(T):
+        for nd in np.nonzero(stall[t])[0][: max(1, nodes // 2)]:
+            X[t, nd * rpn:(nd + 1) * rpn, prim] *= 3.0 if d[prim] > 0 else 0.3
+    X = X.astype(np.float32)
+    for t in range(T):
+        o.ingest(X[t:t + 1])
+        b.ingest(X[t:t + 1])
+        ro, rb = o.score(), b.score()
+        assert np.array_equal(ro["flags"], rb["flags"])
+        no, nb = o.node_verdict(rpn), brute.node_verdict(b, rpn)
+        for key in ("node_flag", "node_tier", "node_stall"):
+            assert np.array_equal(no[key], nb[key]), (key, seed, t)
+
+
+def test_node_verdict_flags_the_node_of_a_slow_rank_and_counts_whole_node_stalls():
+    X = _slow(_fleet(R=64, T=50, seed=21), 19, 1.3)              # rank 19 lives on node 2 (8 ranks per node)
+    stalled = [3, 17, 40]
+    for t in stalled:
+        X[t, 40:48, :] *= np.array([2.0, 2.0, 2.0, 0.5], np.float32)   # node 5 stalls as a whole
+    X[10, 8:15, 0] *= 2.0                                        # seven of node 1's eight ranks: not a whole-node stall
+    o = go.Oracle(64, 4, 50, 30, 8, dir=DIR4)
+    o.ingest(X)
+    res = o.score()
+    nv = o.node_verdict(8)
+    assert nv["node_flag"].tolist() == [0, 0, 1, 0, 0, 0, 0, 0]
+    assert nv["node_tier"][2] == res["tier"][19] == 3
+    assert nv["node_stall"].tolist() == [0, 0, 0, 0, 0, len(stalled), 0, 0]
+    # a stall is transient: node 5 is not flagged by three steps out of fifty
+    assert nv["node_flag"][5] == 0
+    # permuting the ranks inside every node changes no node verdict
+    rng = np.random.default_rng(3)
+    perm = np.concatenate([nd * 8 + rng.permutation(8) for nd in range(8)])
+    o2 = go.Oracle(64, 4, 50, 30, 8, dir=DIR4)
+    o2.ingest(X[:, perm])
+    o2.score()
+    nv2 = o2.node_verdict(8)
+    for key in nv:
+        assert np.array_equal(nv[key], nv2[key]), key
+    # one rank per node: the fold is the identity
+    o.ingest(X[:1])
+    with pytest.raises(RuntimeError):
+        o.node_verdict(8)                                        # an ingest since the evaluation: no verdict
+    res = o.score()
+    nv1 = o.node_verdict(1)
+    assert np.array_equal(nv1["node_flag"], res["flags"]) and np.array_equal(nv1["node_tier"], res["tier"])
+    with pytest.raises(ValueError):
+        o.node_verdict(7)
+
+
+# ------------------------------------------------------------------ triage repeat-offender rule (Section 6)
+
+def test_triage_rule_three_entries_within_a_week():
+    day = 86400
+    # the paper's numbers: the third entry inside one week terminates
+    assert go.triage([0, 2 * day, 5 * day]).tolist() == [0, 0, 1]
+    assert go.triage([0, 2 * day, 7 * day]).tolist() == [0, 0, 1]            # exactly a week apart still counts
+    assert go.triage([0, 2 * day, 7 * day + 1]).tolist() == [0, 0, 0]        # the first entry has aged out
+    assert go.triage([0, 6 * day, 8 * day, 12 * day]).tolist() == [0, 0, 0, 1]   # a sliding week, not calendar weeks
+    assert go.triage([5, 5, 5]).tolist() == [0, 0, 1]
+    assert go.triage([]).tolist() == []
+    assert go.triage([0, 1], limit=1).tolist() == [1, 1]
+    with pytest.raises(ValueError):
+        go.triage([10, 5])                                                   # times must not run backwards
+    rng = np.random.default_rng(9)
+    for _ in range(50):
+        n = int(rng.integers(0, 12))
+        times = np.sort(rng.integers(0, 20 * day, n)).tolist()
+        period = int(rng.integers(0, 10 * day))
+        limit = int(rng.integers(1, 5))
+        assert go.triage(times, period, limit).tolist() == brute.triage(times, period, limit)
