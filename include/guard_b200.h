@@ -18,12 +18,15 @@
  *     memory of its own: the caller hands it one workspace (guard_workspace_bytes) that
  *     holds the telemetry ring and all state, and must keep it alive and untouched until
  *     guard_destroy.
- *   - `stream` is a cudaStream_t passed as void*.  All work is ordered on it and no call
- *     synchronises, except guard_sync_status.  (guard_score may run the window medians on an
- *     internal stream forked from and joined back into `stream` with events, so that they
- *     overlap the preceding guard_ingest; to the caller everything behaves as if enqueued on
- *     `stream`.  guard_set_overlap(ctx, 0) turns that off.)  Calls on one context must be
- *     issued in order on streams that are ordered with respect to each other.
+ *   - `stream` is a cudaStream_t passed as void*.  All work is ordered on it.  The calls that
+ *     synchronise `stream` with the host are the ones that hand a value back from the device:
+ *     guard_sync_status, guard_fallback_steps, guard_fallback_reasons and guard_state_import;
+ *     guard_profile_read waits for the events it recorded.  No other call synchronises.
+ *     (guard_score may run the window medians on an internal stream forked from and joined back
+ *     into `stream` with events, so that they overlap the preceding guard_ingest; to the caller
+ *     everything behaves as if enqueued on `stream`.  guard_set_overlap(ctx, 0) turns that off.)
+ *     Calls on one context must be issued in order on streams that are ordered with respect to
+ *     each other.
  *   - Every function returns a status (GUARD_OK = 0, errors negative) and never throws,
  *     aborts or traps.  Argument errors are detected on the host before anything is
  *     enqueued.  Data-dependent errors (non-finite telemetry, a bounded wait that ran out)
@@ -66,7 +69,7 @@ typedef struct {
     int32_t primary;        /* index of the primary metric: training-step time (Sec. 4.2) */
     int32_t min_signals;    /* metrics that must deviate persistently, "multiple" (Sec. 4.2); clipped to M */
     int32_t n_consec;       /* consecutive evaluations required before a flag is raised (>= 1) */
-    int32_t ranks_per_node; /* 8 in the paper's cluster (Sec. 7.1); used by guard_node_verdict */
+    int32_t ranks_per_node; /* >= 1; 8 in the paper's cluster (Sec. 7.1): group size of guard_node_verdict */
     float tier_moderate;    /* relative slowdown of the moderate tier, 0.10 (Sec. 4.2) */
     float tier_severe;      /* relative slowdown of the severe tier, 0.20 (Sec. 4.2) */
     const int8_t *dir;      /* [M] +1: larger is worse (durations, temperature); -1: smaller is worse */
@@ -82,8 +85,8 @@ size_t guard_workspace_bytes(int ranks, int metrics, int W, int capacity_steps, 
 /*
  * Create a context for `ranks` peers and `metrics` (1..32) indicators, window W
  * (1..65535 steps), persistence k (1..W): a metric is persistent for a rank when at
- * least k of the last W steps exceeded the per-step peer baseline ("sustained deviation
- * ... across consecutive evaluation windows", Sec. 4.2).  topk in 0..min(ranks, 1024).
+ * least k of the last W steps exceeded the per-step peer baseline (the temporal filter of
+ * Sec. 4.2).  topk in 0..min(ranks, 1024).
  * d_workspace: device memory, 256-byte aligned, >= guard_workspace_bytes(...); its state
  * part is zeroed on `stream`.  Errors: GUARD_ERR_ARG, GUARD_ERR_WORKSPACE, GUARD_ERR_CUDA.
  */
@@ -145,8 +148,8 @@ size_t guard_sweep_workspace_bytes(int gpus, int reps, int metrics);
  * and the nearest-rank percentile cut of the bad tail (j = ceil(pct_ppm * G / 1e6)
  * clipped to [1, G]; the j-th worst value).  Metric m fails GPU g when it is a robust-z
  * outlier in the bad direction AND strictly beyond the cut.  A GPU passes when no metric
- * fails; a node passes when all its GPUs pass ("nodes that pass both ... are returned to
- * the healthy pool", Sec. 5.4).  th->dir/thr/floor_rel/floor_abs are used; the other
+ * fails; a node passes when all its GPUs pass (the pass rule of Sec. 5.4).
+ * th->dir/thr/floor_rel/floor_abs are used; the other
  * fields are ignored.  Outputs ("or NULL"): d_gpu_med[G][M], d_fleet_med/mad/cut[M],
  * d_fail_mask[G], d_gpu_pass[G], d_node_pass[nodes].  d_status: device uint32 or NULL,
  * receives sticky status bits (1 = non-finite input, 2 = wait ran out, 4 = internal).
@@ -189,6 +192,67 @@ int guard_sweep_qualify(const float *d_S, int nodes, int gpus_per_node, int reps
 #define GUARD_TOPK_STATIC_MAX_RANKS (1 << 24)
 int guard_topk_static(const float *d_wmed, const float *d_fleet_med, const float *d_fleet_mad, int ranks, int metrics,
                       const guard_thresholds *th, int topk, int32_t *d_topk_idx, float *d_topk_score, void *stream);
+
+/*
+ * Node-level fold of the last evaluation.  The paper acts on nodes (Sec. 4.2: a flagged node
+ * leaves the healthy pool; Sec. 7.1: 8 GPUs per node; the three response classes of
+ * Sec. 4.2), so the per-rank results are folded over groups of ranks_per_node consecutive
+ * ranks, nodes = ranks / ranks_per_node:
+ *   d_node_flag[nodes]   1 when any rank of the node is flagged
+ *   d_node_tier[nodes]   highest tier among its ranks: 0 none, 1 pending verification,
+ *                        2 mitigate at the next checkpoint, 3 restart now
+ *   d_node_stall[nodes]  steps of the evaluation's window in which EVERY rank of the node
+ *                        exceeded the step's peer baseline on the primary metric at once
+ *                        (a correlated whole-node stall, as opposed to one slow GPU)
+ * Every output is "or NULL".  Must follow guard_score with no guard_ingest in between
+ * (GUARD_ERR_NOT_READY otherwise); ranks must be a multiple of ranks_per_node
+ * (GUARD_ERR_ARG).  After a deferred guard_score the fold becomes part of that pending
+ * evaluation: its outputs are complete where the evaluation's are.
+ */
+int guard_node_verdict(guard_ctx *ctx, uint8_t *d_node_flag, uint8_t *d_node_tier, uint16_t *d_node_stall, void *stream);
+
+/*
+ * Checkpoint / resume of a context (the monitor of Sec. 4.2 runs for the months of a
+ * training job and must survive its own restarts).  The state is the telemetry and the
+ * exceedance bits of the last min(W, steps seen) steps, the consecutive-evaluation counters,
+ * the last evaluation's medians, per-rank verdicts and search intervals, the status words
+ * and the step / evaluation counters: everything later results depend on.
+ * guard_state_bytes: size of the state of this context (fixed by its sizes).
+ * guard_state_export: waits (on `stream`, not on the host) for deferred work, then copies the
+ *   state into d_state (DEVICE memory, 16-byte aligned, >= guard_state_bytes).
+ * guard_state_import: loads a state exported by a context of the same ranks, metrics, W, k and
+ *   topk (capacity_steps may differ) into this context, replacing what it held; it reads the
+ *   state's header back and therefore synchronises `stream`.  A context that imports and then
+ *   sees the same steps gives bit-identical results to the one that never stopped.
+ * Errors: GUARD_ERR_WORKSPACE (buffer NULL, misaligned or too small), GUARD_ERR_ARG (not a
+ * state, or one of other sizes), GUARD_ERR_CUDA.
+ */
+size_t guard_state_bytes(const guard_ctx *ctx);
+int guard_state_export(guard_ctx *ctx, void *d_state, size_t state_bytes, void *stream);
+int guard_state_import(guard_ctx *ctx, const void *d_state, size_t state_bytes, void *stream);
+
+/*
+ * Repeat-offender rule of the triage workflow (Sec. 6: a node that enters triage three times
+ * within a week is replaced instead of being triaged again).  Host-only bookkeeping, no GPU
+ * work.  guard_triage_create: `nodes` node ids 0..nodes-1, `limit` entries (the paper: 3)
+ * within `period_s` seconds (the paper: one week = 604800).  guard_triage_record: node
+ * `node` enters triage at `time_s` (seconds, not before the node's previous entry); returns
+ * 1 when this is at least the limit-th entry no more than period_s old (both ends counted),
+ * i.e. the node is to be terminated, 0 when it goes through triage, GUARD_ERR_ARG on a bad
+ * node id or a time that runs backwards.  *entries_in_period (or NULL) receives the number
+ * of entries, this one included, inside that span, counted up to `limit`.
+ */
+typedef struct guard_triage guard_triage;
+int guard_triage_create(guard_triage **out, int nodes, int limit, int64_t period_s);
+int guard_triage_record(guard_triage *t, int node, int64_t time_s, int *entries_in_period);
+void guard_triage_destroy(guard_triage *t);
+
+/* Test hook: limit, in clock cycles, of the first wait for a staged tile in the warp-per-series
+ * window kernel (0 restores the default of about a second).  With a limit of a few cycles that
+ * wait runs out while the copies are still in flight; the kernel then records
+ * GUARD_ERR_TIMEOUT in the status word, lets the copies land and returns, leaving the context
+ * usable after guard_reset.  Exists so that the bounded-wait path can be exercised. */
+int guard_debug_set_wait_limit(guard_ctx *ctx, long long cycles);
 
 /* Synchronises `stream` and returns the sticky device status of the context
  * (GUARD_OK, GUARD_ERR_NONFINITE, GUARD_ERR_TIMEOUT, GUARD_ERR_INTERNAL, GUARD_ERR_CUDA). */
@@ -251,6 +315,13 @@ int64_t guard_fallback_steps(guard_ctx *ctx, void *stream);
  * step's candidate list overflowed, 2 the deferred-exceedance list overflowed, 3 the sampled
  * interval missed the median, 4 candidate selection inconsistent, 5 the interval missed the MAD. */
 int guard_fallback_reasons(guard_ctx *ctx, uint32_t out[6], void *stream);
+
+/* Diagnostic: synchronises `stream` and fills out[6] (HOST) with counts, since creation / reset,
+ * of the series whose windowed median the one-thread-per-series kernel handed to its whole-warp
+ * fallback: 0 in total, 1 no usable search interval, 2 more values inside the interval than it
+ * keeps, 3 the median lay below the interval, 4 above it, 5 the selection did not converge.
+ * Results are exact either way. */
+int guard_window_fallbacks(guard_ctx *ctx, uint32_t out[6], void *stream);
 
 /* Frees the host object (the workspace stays the caller's). NULL is allowed. */
 void guard_destroy(guard_ctx *ctx);

@@ -116,9 +116,29 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Waits for the phase with a time limit (in clock cycles); false if it ran out.
+// Non-blocking probe of the phase (try_wait may suspend the thread for a while before it answers).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+constexpr long long kShortWaitCycles = 100000;   // limits below this poll without suspending
+// Waits for the phase with a time limit (in clock cycles); false if it ran out.  Short limits
+// (test hooks) poll with the non-blocking probe, so that the limit and nothing else ends the wait.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, long long limit_cycles) {
     const long long t0 = clock64();
+    if (limit_cycles < kShortWaitCycles) {
+        while (!mbar_test_wait(bar, parity)) {
+            if (clock64() - t0 > limit_cycles) return false;
+        }
+        return true;
+    }
     while (!mbar_try_wait(bar, parity)) {
         if (clock64() - t0 > limit_cycles) return false;
     }

@@ -24,7 +24,7 @@ constexpr int kIngestStreams = GUARD_INGEST_STREAMS;   // internal streams the c
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, xr_big, xr_big_stride, mask, ring, total;
+    size_t status, consec, lastflag, lasttier, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, xr_big, xr_big_stride, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
@@ -38,6 +38,8 @@ Layout make_layout(int R, int M, int C, int K) {
     L.ticket = off;    off = align_up(off + 64);
     L.fleet = off;     off = align_up(off + 3 * kMaxMetrics * sizeof(float));
     L.consec = off;    off = align_up(off + (size_t)R);
+    L.lastflag = off;  off = align_up(off + (size_t)R);
+    L.lasttier = off;  off = align_up(off + (size_t)R);
     L.xr_split = xrank_split_supported(R, M) ? 1 : 0;
     L.xr_cluster = (!L.xr_split && xrank_cluster_supported(R, M)) ? 1 : 0;
     L.xr_steps = (!L.xr_split && !L.xr_cluster && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
@@ -88,6 +90,7 @@ const char *fill_params(MetricParams &p, const guard_thresholds *th, int M, int 
         if (th->min_signals < 1) return "min_signals must be >= 1";
         if (th->n_consec < 1 || th->n_consec > 255) return "n_consec must be in 1..255";
         if (!(th->tier_moderate >= 0.0f) || !(th->tier_severe >= th->tier_moderate)) return "tier thresholds must satisfy 0 <= moderate <= severe";
+        if (th->ranks_per_node < 1) return "ranks_per_node must be >= 1";
     }
     for (int m = 0; m < M; ++m) {
         if (th->dir[m] != 1 && th->dir[m] != -1) return "dir[m] must be +1 or -1";
@@ -127,6 +130,8 @@ struct guard_ctx {
     long long launches;  // kernels enqueued by this context so far
     long long evals;     // evaluations since creation / reset
     long long seen_at_eval = 0;   // steps seen at the last evaluation
+    int ranks_per_node = 8;
+    long long wait_limit = 0;     // test hook: limit of the warp window path's first wait (0: default)
     // overlap of the window medians (which need only the ring) with the cross-rank kernels of the
     // ingest that precedes them: an internal stream forked from and joined into the caller's
     bool overlap = true;
@@ -154,13 +159,14 @@ struct guard_ctx {
     bool deferred = false;
     bool pending = false;             // an evaluation has been enqueued whose end the caller's stream has not waited for
     int pending_n = 0;                // its window length
+    long long pending_seen = 0;       // steps seen when it was enqueued (its window ends there)
     // In deferred mode the cross-rank kernels of consecutive ingests alternate between two internal
     // streams (each with its own scratch), so that one block's selections overlap the next block's
     // sweeps; the caller's stream waits for them only where it joins.
     cudaStream_t xs[kIngestStreams] = {};
     cudaEvent_t ev_xs[kIngestStreams] = {}, ev_data = nullptr;
     bool xs_busy[kIngestStreams] = {};   // stream k has work the caller's stream has not waited for
-    int xs_steps[kIngestStreams] = {};   // block sizes of that work (ring slots it still reads)
+    long long xs_first[kIngestStreams] = {};   // first step (counted from creation / reset) of the oldest such block
     int xs_next = 0;
     int scratch_sel = 0;                // which split scratch the next launch uses
     cudaStream_t tail = nullptr;
@@ -185,11 +191,20 @@ struct guard_ctx {
         return ok;
     }
     // Ring slots (in steps, counted back from the newest) that work not yet joined still reads.
-    int protected_steps() const {
-        int n = pending ? pending_n : 0;
-        int x = 0;
-        for (int k = 0; k < kIngestStreams; ++k) x += xs_busy[k] ? xs_steps[k] : 0;
-        return n > x ? n : x;
+    // Oldest step that work not yet joined may still read: a pending evaluation reads the pending_n
+    // steps that ended where `seen` stood when it was enqueued; an internal ingest stream reads the
+    // blocks enqueued on it since it was last joined.  Everything from that step on is protected.
+    // Work whose end event has already completed (a host-side query, no waiting) reads nothing any more.
+    long long protected_steps() {
+        long long first = seen;
+        if (pending && pending_seen - pending_n < first && cudaEventQuery(ev_e) != cudaSuccess) first = pending_seen - pending_n;
+        for (int k = 0; k < kIngestStreams; ++k)
+            if (xs_busy[k] && xs_first[k] < first) {
+                if (cudaEventQuery(ev_xs[k]) == cudaSuccess) { xs_busy[k] = false; continue; }   // finished: nothing left to wait for
+                first = xs_first[k];
+            }
+        (void)cudaGetLastError();   // cudaErrorNotReady is an answer, not an error
+        return seen - first;
     }
     bool ensure_tail() {
         if (tail) return true;
@@ -222,7 +237,6 @@ struct guard_ctx {
                 cudaError_t e = cudaStreamWaitEvent(st, ev_xs[k], 0);
                 if (e != cudaSuccess) return e;
                 xs_busy[k] = false;
-                xs_steps[k] = 0;
             }
         return cudaSuccess;
     }
@@ -235,6 +249,8 @@ struct guard_ctx {
     float *fleet_med() const { return (float *)(ws + L.fleet); }
     float *fleet_mad() const { return fleet_med() + kMaxMetrics; }
     uint8_t *consec() const { return (uint8_t *)(ws + L.consec); }
+    uint8_t *lastflag() const { return (uint8_t *)(ws + L.lastflag); }
+    uint8_t *lasttier() const { return (uint8_t *)(ws + L.lasttier); }
     float *wmed() const { return (float *)(ws + L.wmed); }
     float *step_med() const { return (float *)(ws + L.stepstat); }
     float *step_mad() const { return step_med() + (size_t)C * M; }
@@ -243,7 +259,10 @@ struct guard_ctx {
     float *ring() const { return (float *)(ws + L.ring); }
     int mask_bytes() const { return M <= 8 ? 1 : 4; }
     // Cross-rank statistics of S rows: the bracketed path where it applies, else the direct one.
-    cudaError_t xrank(XrankArgs a, int S, cudaStream_t st) {
+    // own_scratch = false: the call may run beside another cross-rank call of this context (the fleet
+    // baseline of a deferred evaluation beside the next ingest), so it must not touch the one
+    // scratch of the bracketed path: such rows take the direct selection.
+    cudaError_t xrank(XrankArgs a, int S, cudaStream_t st, bool own_scratch = true) {
         // a few rows at a time: one CTA per column keeps the whole GPU busy
         if (xrank_column_supported(R) && (long long)S * M <= 64 && !a.cut) {
             launches += 1;
@@ -273,7 +292,7 @@ struct guard_ctx {
             launches += 1;
             return launch_xrank_cluster(a, p, S, status() + 2, st, (profiling == 1 && a.mask_base) ? &prof : nullptr);
         }
-        if (L.xr_steps == 0) { launches += 1; return launch_xrank_direct(a, p, S, st); }
+        if (L.xr_steps == 0 || !own_scratch) { launches += 1; return launch_xrank_direct(a, p, S, st); }
         XrankScratch sc = carve_xrank_scratch(ws + L.xr_small, ws + L.xr_big, R, M, L.xr_steps);
         sc.reasons = status() + 2;
         const int first = a.first_slot;
@@ -341,6 +360,7 @@ int guard_create(guard_ctx **out, int ranks, int metrics, int W, int k, const gu
     if (!c) { set_error(g_error, "out of host memory"); return GUARD_ERR_ARG; }
     c->R = ranks; c->M = metrics; c->W = W; c->k = k; c->C = capacity_steps; c->K = topk;
     c->p = p; c->L = L; c->ws = (char *)d_workspace; c->seen = 0; c->launches = 0; c->evals = 0; c->error[0] = 0;
+    c->ranks_per_node = th->ranks_per_node;
     // state: status word, ticket, fleet statistics, consecutive counters
     cudaError_t e = cudaMemsetAsync(c->ws, 0, L.wmed, (cudaStream_t)stream);
     if (e != cudaSuccess) {
@@ -417,8 +437,8 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
         e = c->xrank(a, B, c->xs[k]);
         c->scratch_sel = 0;
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_xs[k], c->xs[k]);
+        if (!c->xs_busy[k]) c->xs_first[k] = c->seen;
         c->xs_busy[k] = true;
-        c->xs_steps[k] = B;
     } else {
         e = c->join_xs(st);   // earlier blocks still on the internal streams come first
         if (e == cudaSuccess) e = c->xrank(a, B, st);
@@ -456,6 +476,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     c->seen_at_eval = c->seen;
     w.fb_count = c->status() + 8;
     w.status = c->status();
+    w.first_wait_cycles = c->wait_limit;
     // The window medians read only the ring: run them on the internal stream, forked where the
     // ring became complete, so that they overlap the cross-rank kernels of the preceding ingest;
     // the caller's stream waits for them before anything that uses them.
@@ -513,7 +534,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     x.med_user = d_fleet_med;
     x.mad_user = d_fleet_mad;
     x.status = c->status();
-    e = c->xrank(x, 1, ts);
+    e = c->xrank(x, 1, ts, !defer);
     if (e != cudaSuccess) return c->cuda_fail(e, "fleet baseline launch");
 
     ScoreArgs s{};
@@ -533,6 +554,8 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     s.metric_mask = d_metric_mask;
     s.flags = d_flags;
     s.tier = d_tier;
+    s.flags_keep = c->lastflag();
+    s.tier_keep = c->lasttier();
     // top-k and the score pass are independent of each other: top-k goes to the internal stream
     const bool want_topk = c->K > 0 && (d_topk_idx || d_topk_score);
     bool topk_forked = false;
@@ -575,6 +598,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         if (e != cudaSuccess) return c->cuda_fail(e, "event record");
         c->pending = true;
         c->pending_n = n;
+        c->pending_seen = c->seen;
     }
     return GUARD_OK;
 }
@@ -659,6 +683,172 @@ int guard_sweep_qualify(const float *d_S, int nodes, int gpus_per_node, int reps
     return GUARD_OK;
 }
 
+int guard_node_verdict(guard_ctx *c, uint8_t *d_node_flag, uint8_t *d_node_tier, uint16_t *d_node_stall, void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    if (c->R % c->ranks_per_node != 0)
+        return c->fail(GUARD_ERR_ARG, "ranks (%d) is not a multiple of ranks_per_node (%d)", c->R, c->ranks_per_node);
+    if (c->evals < 1 || c->seen_at_eval != c->seen)
+        return c->fail(GUARD_ERR_NOT_READY, "guard_node_verdict must follow guard_score with no ingest in between");
+    NodeArgs a{};
+    a.R = c->R;
+    a.ranks_per_node = c->ranks_per_node;
+    a.nodes = c->R / c->ranks_per_node;
+    a.primary = c->p.primary;
+    a.flags = c->lastflag();
+    a.tier = c->lasttier();
+    a.mask_base = c->mask();
+    a.mask_bytes = c->mask_bytes();
+    a.capacity = c->C;
+    a.last_slot = (int)((c->seen - 1) % c->C);
+    a.n = (int)(c->seen < c->W ? c->seen : c->W);
+    a.node_flag = d_node_flag;
+    a.node_tier = d_node_tier;
+    a.node_stall = d_node_stall;
+    // a deferred evaluation still pending: the fold joins it on the evaluation's own stream
+    const bool on_tail = c->pending && c->tail;
+    cudaStream_t ts = on_tail ? c->tail : (cudaStream_t)stream;
+    cudaError_t e = launch_node_verdict(a, ts);
+    if (e == cudaSuccess && on_tail) e = cudaEventRecord(c->ev_e, c->tail);
+    if (e != cudaSuccess) return c->cuda_fail(e, "node verdict launch");
+    c->launches += 1;
+    return GUARD_OK;
+}
+
+// ---- state export / import -----------------------------------------------------------------------
+namespace {
+struct StateHeader {
+    uint32_t magic, version;
+    int32_t R, M, W, k, K, mask_bytes;
+    int64_t seen, evals, seen_at_eval;
+    int32_t steps;      // ring steps stored: min(seen, W)
+    int32_t pad;
+};
+constexpr uint32_t kStateMagic = 0x47524453u;   // "GRDS"
+constexpr size_t kStateHeaderBytes = 256;
+
+struct StateLayout { size_t status, fleet, consec, lastflag, lasttier, wmed, wspread, wcentre, mask, ring, total; };
+StateLayout state_layout(const guard_ctx *c) {
+    StateLayout s{};
+    const size_t RM = (size_t)c->R * c->M * sizeof(float);
+    size_t off = kStateHeaderBytes;
+    s.status = off;   off = align_up(off + 64);
+    s.fleet = off;    off = align_up(off + 3 * kMaxMetrics * sizeof(float));
+    s.consec = off;   off = align_up(off + (size_t)c->R);
+    s.lastflag = off; off = align_up(off + (size_t)c->R);
+    s.lasttier = off; off = align_up(off + (size_t)c->R);
+    s.wmed = off;     off = align_up(off + RM);
+    s.wspread = off;  off = align_up(off + RM);
+    s.wcentre = off;  off = align_up(off + RM);
+    s.mask = off;     off = align_up(off + (size_t)c->W * c->R * c->mask_bytes());
+    s.ring = off;     off = align_up(off + (size_t)c->W * RM);
+    s.total = off;
+    return s;
+}
+
+// Copies the last `steps` ring rows (row_bytes each) between the ring at `ring` (capacity C, newest
+// row at step index seen - 1) and a compact buffer holding them oldest first.
+cudaError_t copy_rows(char *ring, char *compact, size_t row_bytes, long long seen, int steps, int C, bool to_compact,
+                      cudaStream_t st) {
+    long long step = seen - steps;
+    int done = 0;
+    while (done < steps) {
+        const int slot = (int)((step + done) % C);
+        const int run = (steps - done < C - slot) ? (steps - done) : (C - slot);
+        char *r = ring + (size_t)slot * row_bytes, *q = compact + (size_t)done * row_bytes;
+        cudaError_t e = cudaMemcpyAsync(to_compact ? q : r, to_compact ? r : q, (size_t)run * row_bytes, cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) return e;
+        done += run;
+    }
+    return cudaSuccess;
+}
+}  // namespace
+
+size_t guard_state_bytes(const guard_ctx *c) { return c ? state_layout(c).total : 0; }
+
+int guard_state_export(guard_ctx *c, void *d_state, size_t state_bytes, void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    const StateLayout sl = state_layout(c);
+    if (!d_state || ((uintptr_t)d_state % 16) != 0 || state_bytes < sl.total)
+        return c->fail(GUARD_ERR_WORKSPACE, "state buffer must be non-NULL, 16-byte aligned and at least %zu bytes", sl.total);
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = c->join(st);
+    if (e == cudaSuccess) e = c->join_xs(st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "join of deferred work");
+    char *d = (char *)d_state;
+    const size_t RM = (size_t)c->R * c->M * sizeof(float);
+    StateHeader h{};
+    h.magic = kStateMagic; h.version = 1;
+    h.R = c->R; h.M = c->M; h.W = c->W; h.k = c->k; h.K = c->K; h.mask_bytes = c->mask_bytes();
+    h.seen = c->seen; h.evals = c->evals; h.seen_at_eval = c->seen_at_eval;
+    h.steps = (int)(c->seen < c->W ? c->seen : c->W);
+    // pageable host source: the runtime stages it before the call returns
+    e = cudaMemcpyAsync(d, &h, sizeof(h), cudaMemcpyHostToDevice, st);
+    auto dd = [&](size_t dst_off, const void *src, size_t n) {
+        if (e == cudaSuccess) e = cudaMemcpyAsync(d + dst_off, src, n, cudaMemcpyDeviceToDevice, st);
+    };
+    dd(sl.status, c->status(), 64);
+    dd(sl.fleet, c->fleet_med(), 3 * kMaxMetrics * sizeof(float));
+    dd(sl.consec, c->consec(), (size_t)c->R);
+    dd(sl.lastflag, c->lastflag(), (size_t)c->R);
+    dd(sl.lasttier, c->lasttier(), (size_t)c->R);
+    dd(sl.wmed, c->wmed(), RM);
+    dd(sl.wspread, c->ws + c->L.wspread, RM);
+    dd(sl.wcentre, c->ws + c->L.wcentre, RM);
+    if (e == cudaSuccess) e = copy_rows((char *)c->mask(), d + sl.mask, (size_t)c->R * c->mask_bytes(), c->seen, h.steps, c->C, true, st);
+    if (e == cudaSuccess) e = copy_rows((char *)c->ring(), d + sl.ring, RM, c->seen, h.steps, c->C, true, st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_state_export");
+    return GUARD_OK;
+}
+
+int guard_state_import(guard_ctx *c, const void *d_state, size_t state_bytes, void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    const StateLayout sl = state_layout(c);
+    if (!d_state || ((uintptr_t)d_state % 16) != 0 || state_bytes < sl.total)
+        return c->fail(GUARD_ERR_WORKSPACE, "state buffer must be non-NULL, 16-byte aligned and at least %zu bytes", sl.total);
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = c->join(st);
+    if (e == cudaSuccess) e = c->join_xs(st);
+    StateHeader h{};
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&h, d_state, sizeof(h), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_state_import");
+    if (h.magic != kStateMagic || h.version != 1) return c->fail(GUARD_ERR_ARG, "not a state written by guard_state_export");
+    if (h.R != c->R || h.M != c->M || h.W != c->W || h.k != c->k || h.K != c->K || h.mask_bytes != c->mask_bytes())
+        return c->fail(GUARD_ERR_ARG, "state was exported from a context of other sizes (ranks %d metrics %d W %d k %d topk %d)",
+                       h.R, h.M, h.W, h.k, h.K);
+    if (h.seen < 0 || h.steps != (int)(h.seen < h.W ? h.seen : h.W) || h.evals < 0 || h.seen_at_eval > h.seen)
+        return c->fail(GUARD_ERR_ARG, "state header is inconsistent");
+    const char *d = (const char *)d_state;
+    const size_t RM = (size_t)c->R * c->M * sizeof(float);
+    // scratch that must start at zero (ticket, bracketed-path flags) is cleared with the rest of the prefix
+    e = cudaMemsetAsync(c->ws, 0, c->L.wmed, st);
+    auto dd = [&](void *dst, size_t src_off, size_t n) {
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dst, d + src_off, n, cudaMemcpyDeviceToDevice, st);
+    };
+    dd(c->status(), sl.status, 64);
+    dd(c->fleet_med(), sl.fleet, 3 * kMaxMetrics * sizeof(float));
+    dd(c->consec(), sl.consec, (size_t)c->R);
+    dd(c->lastflag(), sl.lastflag, (size_t)c->R);
+    dd(c->lasttier(), sl.lasttier, (size_t)c->R);
+    dd(c->wmed(), sl.wmed, RM);
+    dd(c->ws + c->L.wspread, sl.wspread, RM);
+    dd(c->ws + c->L.wcentre, sl.wcentre, RM);
+    if (e == cudaSuccess) e = copy_rows((char *)c->mask(), const_cast<char *>(d) + sl.mask, (size_t)c->R * c->mask_bytes(), h.seen, h.steps, c->C, false, st);
+    if (e == cudaSuccess) e = copy_rows((char *)c->ring(), const_cast<char *>(d) + sl.ring, RM, h.seen, h.steps, c->C, false, st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_state_import");
+    c->seen = h.seen;
+    c->evals = h.evals;
+    c->seen_at_eval = h.seen_at_eval;
+    c->fork_fresh = false;
+    return GUARD_OK;
+}
+
+int guard_debug_set_wait_limit(guard_ctx *c, long long cycles) {
+    if (!c || cycles < 0) return GUARD_ERR_ARG;
+    c->wait_limit = cycles;
+    return GUARD_OK;
+}
+
 int guard_sync_status(guard_ctx *c, void *stream) {
     if (!c) return GUARD_ERR_ARG;
     uint32_t s = 0;
@@ -723,6 +913,16 @@ int guard_fallback_reasons(guard_ctx *c, uint32_t out[6], void *stream) {
     if (e == cudaSuccess) e = cudaMemcpyAsync(out, c->status() + 2, 6 * sizeof(uint32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "guard_fallback_reasons");
+    return GUARD_OK;
+}
+
+int guard_window_fallbacks(guard_ctx *c, uint32_t out[6], void *stream) {
+    if (!c || !out) return GUARD_ERR_ARG;
+    cudaError_t e = c->join((cudaStream_t)stream);
+    if (e == cudaSuccess) e = c->join_xs((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out, c->status() + 8, 6 * sizeof(uint32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_window_fallbacks");
     return GUARD_OK;
 }
 

@@ -89,6 +89,7 @@ struct WindowArgs {
     float smooth;           // weight of the newest median in the interval's centre (0: default)
     uint32_t *fb_count;     // [6] series the thread path's interval did not serve, in total and by reason (diagnostic), or NULL
     uint32_t *status;
+    long long first_wait_cycles;   // limit of the warp path's wait for a staged tile (0: the default of about a second)
 };
 // Launches one kernel (thread, warp or staged path).
 cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st);
@@ -111,8 +112,23 @@ struct ScoreArgs {
     uint32_t *metric_mask;   // [R] or NULL
     uint8_t *flags;          // [R] or NULL
     uint8_t *tier;           // [R] or NULL
+    uint8_t *flags_keep;     // [R] the context's own copy (input of the node-level fold), never NULL
+    uint8_t *tier_keep;      // [R] likewise
 };
 cudaError_t launch_score_flag(const ScoreArgs &a, const MetricParams &p, cudaStream_t st);
+
+// Node-level fold of an evaluation: any rank flagged, highest tier, and the number of window steps
+// in which every rank of the node exceeded on the primary metric at once.
+struct NodeArgs {
+    int R, ranks_per_node, nodes, primary;
+    const uint8_t *flags, *tier;   // [R] per-rank results of the evaluation
+    const void *mask_base;         // exceedance rows [capacity][R]
+    int mask_bytes, capacity, last_slot, n;
+    uint8_t *node_flag;            // [nodes] or NULL
+    uint8_t *node_tier;            // [nodes] or NULL
+    uint16_t *node_stall;          // [nodes] or NULL
+};
+cudaError_t launch_node_verdict(const NodeArgs &a, cudaStream_t st);
 
 // Block-then-grid top-k of dir * wmed[:, primary].
 struct TopkArgs {

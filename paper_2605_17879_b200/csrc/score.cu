@@ -69,6 +69,8 @@ __global__ void __launch_bounds__(kScoreThreads) score_flag_kernel(const ScoreAr
     if (a.metric_mask) a.metric_mask[r] = mask;
     if (a.flags) a.flags[r] = (uint8_t)flag;
     if (a.tier) a.tier[r] = (uint8_t)t;
+    a.flags_keep[r] = (uint8_t)flag;
+    a.tier_keep[r] = (uint8_t)t;
 }
 
 
@@ -187,9 +189,67 @@ __global__ void __launch_bounds__(kFastWarps * 32) score_flag_bytes_kernel(const
     if (a.metric_mask) a.metric_mask[r] = mask;
     if (a.flags) a.flags[r] = (uint8_t)flag;
     if (a.tier) a.tier[r] = (uint8_t)t;
+    a.flags_keep[r] = (uint8_t)flag;
+    a.tier_keep[r] = (uint8_t)t;
+}
+
+// Node-level fold.  A CTA takes 32 nodes; its eight warps split the window's steps (warp w takes
+// steps w, w + 8, ...), lane l owns node l of the CTA's 32.  "All ranks of the node exceeded on the
+// primary metric in this step" is an AND over the node's exceedance entries; with eight ranks per
+// node and byte-wide entries that is one 64-bit load and one mask test.
+constexpr int kNodeWarps = 8;
+
+template <typename MaskT>
+__global__ void __launch_bounds__(kNodeWarps * 32) node_verdict_kernel(const NodeArgs a) {
+    __shared__ uint32_t s_stall[32];
+    const int lane = lane_id(), w = warp_id();
+    const int node = blockIdx.x * 32 + lane;
+    if (threadIdx.x < 32) s_stall[threadIdx.x] = 0;
+    __syncthreads();
+    const bool live = node < a.nodes;
+    const int rpn = a.ranks_per_node;
+    const size_t r0 = (size_t)node * rpn;
+    const MaskT *mask_base = (const MaskT *)a.mask_base;
+    const int first = ((a.last_slot - (a.n - 1)) % a.capacity + a.capacity) % a.capacity;
+    const bool wide = sizeof(MaskT) == 1 && rpn == 8 && (a.R & 7) == 0;
+    const unsigned long long want = 0x0101010101010101ull << a.primary;
+    uint32_t stall = 0;
+    if (live) {
+        for (int j = w; j < a.n; j += kNodeWarps) {
+            int slot = first + j;
+            if (slot >= a.capacity) slot -= a.capacity;
+            const MaskT *rowp = mask_base + (size_t)slot * a.R + r0;
+            bool all = true;
+            if (wide) {
+                all = (__ldg(reinterpret_cast<const unsigned long long *>(rowp)) & want) == want;
+            } else {
+                for (int q = 0; q < rpn; ++q) all = all && (((uint32_t)rowp[q] >> a.primary) & 1u);
+            }
+            stall += all;
+        }
+        if (stall) atomicAdd(&s_stall[lane], stall);
+    }
+    __syncthreads();
+    if (w == 0 && live) {
+        int any = 0, top = 0;
+        for (int q = 0; q < rpn; ++q) {
+            any |= a.flags[r0 + q];
+            top = max(top, (int)a.tier[r0 + q]);
+        }
+        if (a.node_flag) a.node_flag[node] = (uint8_t)(any != 0);
+        if (a.node_tier) a.node_tier[node] = (uint8_t)top;
+        if (a.node_stall) a.node_stall[node] = (uint16_t)s_stall[lane];
+    }
 }
 
 }  // namespace
+
+cudaError_t launch_node_verdict(const NodeArgs &a, cudaStream_t st) {
+    const int grid = (a.nodes + 31) / 32;
+    if (a.mask_bytes == 1) node_verdict_kernel<uint8_t><<<grid, kNodeWarps * 32, 0, st>>>(a);
+    else node_verdict_kernel<uint32_t><<<grid, kNodeWarps * 32, 0, st>>>(a);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_score_flag(const ScoreArgs &a, const MetricParams &p, cudaStream_t st) {
     const int grid = (a.R + kScoreThreads - 1) / kScoreThreads;

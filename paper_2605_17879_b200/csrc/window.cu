@@ -4,12 +4,16 @@
 // then every thread selects inside its own column.
 #include <math_constants.h>
 
+#include <mutex>
+
 #include "colselect.cuh"
 #include "kernels.h"
 
 namespace guard {
 
 namespace {
+
+constexpr size_t kMaxStagedTile = 200 * 1024;   // largest staged tile (dynamic shared memory of the staged path)
 
 // Staged path.  blockDim.x == TC; dynamic shared memory = n * TC * 4 bytes.
 template <int TC>
@@ -294,8 +298,13 @@ __global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a
         const int next = tile + gridDim.x;
         if (next < ntiles) stage(next, cur ^ 1);
         if (use_bulk) {
-            if (!mbar_wait_bounded(&bar[cur], (uint32_t)((it >> 1) & 1), kWaitLimitCycles)) {
-                atomicOr(a.status, kStatTimeout);
+            // only this first wait takes the caller's (test) limit: the waits below, which let the copies
+            // in flight land before the CTA leaves, always get the full one.  The CTA decides as one:
+            // if the wait ran out for any thread, all of them leave.
+            const bool arrived = mbar_wait_bounded(&bar[cur], (uint32_t)((it >> 1) & 1),
+                                                   a.first_wait_cycles > 0 ? a.first_wait_cycles : kWaitLimitCycles);
+            if (__syncthreads_or(!arrived)) {
+                if (!arrived) atomicOr(a.status, kStatTimeout);
                 mbar_wait_bounded(&bar[cur], (uint32_t)((it >> 1) & 1), kWaitLimitCycles);   // let copies in flight land
                 if (next < ntiles) mbar_wait_bounded(&bar[cur ^ 1], (uint32_t)(((it + 1) >> 1) & 1), kWaitLimitCycles);
                 return;
@@ -334,13 +343,39 @@ __global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a
     }
 }
 
+// Function attributes are set once per device and kernel (the calls go to the driver: two of them
+// per evaluation showed in the per-step latency of the streaming configuration).
+struct AttrOnce {
+    std::mutex mu;
+    bool done[64] = {};
+    int sms[64] = {};
+    template <typename F>
+    cudaError_t operator()(int &dev_out, F &&set) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        dev_out = dev & 63;
+        std::lock_guard<std::mutex> lock(mu);
+        if (!done[dev_out]) {
+            e = set();
+            if (e != cudaSuccess) return e;
+            if (cudaDeviceGetAttribute(&sms[dev_out], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms[dev_out] = 148;
+            done[dev_out] = true;
+        }
+        return cudaSuccess;
+    }
+};
+
 template <int VPL>
 cudaError_t launch_warp_path(const WindowArgs &a, int use_bulk, cudaStream_t st) {
     const size_t smem = 2 * (size_t)a.n * kWarpPitch * 4;
-    cudaError_t e = cudaFuncSetAttribute(window_warp_kernel<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static AttrOnce once;
+    int dev = 0;
+    cudaError_t e = once(dev, [] {
+        return cudaFuncSetAttribute(window_warp_kernel<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 32 * VPL * kWarpPitch * 4);
+    });
     if (e != cudaSuccess) return e;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = once.sms[dev];
     const int ntiles = (a.series + kWarpTileCols - 1) / kWarpTileCols;
     const int grid = ntiles < 2 * sms ? ntiles : 2 * sms;
     window_warp_kernel<VPL><<<grid, 1024, smem, st>>>(a, ntiles, use_bulk);
@@ -567,9 +602,14 @@ __global__ void __launch_bounds__(kThCols, 9) window_thread_kernel(const WindowA
 template <int VPL>
 cudaError_t launch_thread_path(const WindowArgs &a, cudaStream_t st) {
     const size_t smem = (size_t)kThSlots * kThCols * 4;
-    cudaError_t e = cudaFuncSetAttribute(window_thread_kernel<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(window_thread_kernel<VPL>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    static AttrOnce once;
+    int dev = 0;
+    cudaError_t e = once(dev, [] {
+        cudaError_t e2 = cudaFuncSetAttribute(window_thread_kernel<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kThSlots * kThCols * 4);
+        if (e2 == cudaSuccess)
+            e2 = cudaFuncSetAttribute(window_thread_kernel<VPL>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        return e2;
+    });
     if (e != cudaSuccess) return e;
     window_thread_kernel<VPL><<<(a.series + kThCols - 1) / kThCols, kThCols, smem, st>>>(a);
     return cudaGetLastError();
@@ -620,7 +660,11 @@ __global__ void window_select_global_kernel(const WindowArgs a) {
 template <int TC>
 cudaError_t launch_staged(const WindowArgs &a, int use_bulk, cudaStream_t st) {
     const size_t smem = (size_t)a.n * TC * 4;
-    cudaError_t e = cudaFuncSetAttribute(window_select_kernel<TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static AttrOnce once;
+    int dev = 0;
+    cudaError_t e = once(dev, [] {
+        return cudaFuncSetAttribute(window_select_kernel<TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxStagedTile);
+    });
     if (e != cudaSuccess) return e;
     const int grid = (a.series + TC - 1) / TC;
     window_select_kernel<TC><<<grid, TC, smem, st>>>(a, use_bulk);
@@ -632,7 +676,7 @@ cudaError_t launch_staged(const WindowArgs &a, int use_bulk, cudaStream_t st) {
 int window_launch_count(const WindowArgs &) { return 1; }
 
 cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st) {
-    constexpr size_t kMaxTile = 200 * 1024;
+    constexpr size_t kMaxTile = kMaxStagedTile;
     // bulk copies need 16-byte aligned sources and sizes
     const int use_bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
     const size_t n = (size_t)a.n;

@@ -430,12 +430,15 @@ __device__ __forceinline__ void cl_sweep(const float *__restrict__ row, const in
                 float z[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
+                    // the finite check looks at the value itself: the deviation of two finite values of
+                    // opposite sign may overflow
+                    const bool nf = nonfinite_bits(__float_as_uint(v[j][c]));
                     const float sdev = __fmaf_rn(v[j][c], sg[c], nsm[c]);
                     const float d = fabsf(sdev);
                     v[j][c] = d;
                     z[c] = sdev * irlo[c];
-                    if (guard) bad |= (base + j * LPI + rl < r1) && !(d <= kFltMax);
-                    else bad |= !(d <= kFltMax);
+                    if (guard) bad |= (base + j * LPI + rl < r1) && nf;
+                    else bad |= nf;
                 }
                 // conservative test for "some metric of this rank may exceed": exact tests follow
                 if (fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])) > 0.99f && (!guard || base + j * LPI + rl < r1))

@@ -25,6 +25,8 @@
 // The scratch (intervals, counters, kept lists: ~80 KB per step) stays in L2 between kernels.
 #include <math_constants.h>
 
+#include <mutex>
+
 #include "xrank_common.cuh"
 #include "xrank_direct.cuh"
 
@@ -386,7 +388,11 @@ __global__ void __launch_bounds__(kSpThreads, 4) xsplit_sweep_kernel(const Xrank
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             const int m = 4 * q + c;
-                            if (!(fabsf(sdev[c]) <= kFltMax) && a.check_finite) atomicOr(a.status, kStatNonFinite);
+                            // a deviation that is not finite: the value itself (re-read, this is rare) decides,
+                            // since two finite values of opposite sign may differ by more than the largest float
+                            if (!(fabsf(sdev[c]) <= kFltMax) && a.check_finite &&
+                                nonfinite_bits(__float_as_uint(__ldg(row + (size_t)r * M + m))))
+                                atomicOr(a.status, kStatNonFinite);
                             if (sdev[c] > rlo[c]) {
                                 if (sdev[c] > sh.rhi[m]) {
                                     eb |= 1u << m;
@@ -742,10 +748,12 @@ cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S,
     sc.nseg = (uint32_t *)b;  b += align256((size_t)S * M * g.chunks * sizeof(uint32_t));
     sc.list = (uint32_t *)b;
     const size_t smem = split_sweep_smem(g, M);
+    static std::mutex attr_mutex;
     static bool attr_set_dev[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(attr_mutex);
     bool &attr_set = attr_set_dev[dev & 63];
     if (!attr_set) {
         e = cudaFuncSetAttribute(xsplit_sweep_kernel<2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);

@@ -65,6 +65,22 @@ def lib():
                                           vp, C.c_size_t] + [fp] * 8 + [vp]
         L.guard_topk_static.restype = C.c_int
         L.guard_topk_static.argtypes = [fp, fp, fp, C.c_int, C.c_int, C.POINTER(_Thresholds), C.c_int, fp, fp, vp]
+        L.guard_node_verdict.restype = C.c_int
+        L.guard_node_verdict.argtypes = [vp, fp, fp, fp, vp]
+        L.guard_state_bytes.restype = C.c_size_t
+        L.guard_state_bytes.argtypes = [vp]
+        L.guard_state_export.restype = C.c_int
+        L.guard_state_export.argtypes = [vp, vp, C.c_size_t, vp]
+        L.guard_state_import.restype = C.c_int
+        L.guard_state_import.argtypes = [vp, vp, C.c_size_t, vp]
+        L.guard_triage_create.restype = C.c_int
+        L.guard_triage_create.argtypes = [C.POINTER(vp), C.c_int, C.c_int, C.c_int64]
+        L.guard_triage_record.restype = C.c_int
+        L.guard_triage_record.argtypes = [vp, C.c_int, C.c_int64, C.POINTER(C.c_int)]
+        L.guard_triage_destroy.restype = None
+        L.guard_triage_destroy.argtypes = [vp]
+        L.guard_debug_set_wait_limit.restype = C.c_int
+        L.guard_debug_set_wait_limit.argtypes = [vp, C.c_longlong]
         L.guard_sync_status.restype = C.c_int
         L.guard_sync_status.argtypes = [vp, vp]
         L.guard_reset.restype = C.c_int
@@ -77,6 +93,8 @@ def lib():
         L.guard_fallback_steps.argtypes = [vp, vp]
         L.guard_fallback_reasons.restype = C.c_int
         L.guard_fallback_reasons.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        L.guard_window_fallbacks.restype = C.c_int
+        L.guard_window_fallbacks.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.guard_set_overlap.restype = C.c_int
         L.guard_set_overlap.argtypes = [vp, C.c_int]
         L.guard_set_deferred.restype = C.c_int
@@ -145,6 +163,7 @@ class Guard:
                  tier_moderate: float = 0.10, tier_severe: float = 0.20, capacity: Optional[int] = None, topk: int = 0,
                  device="cuda", workspace: Optional[torch.Tensor] = None):
         self.R, self.M, self.W, self.k, self.K = ranks, metrics, W, k, topk
+        self.ranks_per_node = ranks_per_node
         self.C = capacity if capacity is not None else W
         self.device = torch.device(device)
         self._h = C.c_void_p()
@@ -199,6 +218,14 @@ class Guard:
         with torch.cuda.device(self.device):
             self._check(lib().guard_fallback_reasons(self._h, out, _stream()))
         names = ("cta_list", "step_list", "deferred_list", "median_miss", "select", "mad_miss")
+        return dict(zip(names, [int(v) for v in out]))
+
+    def window_fallbacks(self):
+        """Series the thread-per-series window kernel handed to its whole-warp fallback (synchronises)."""
+        out = (C.c_uint32 * 6)()
+        with torch.cuda.device(self.device):
+            self._check(lib().guard_window_fallbacks(self._h, out, _stream()))
+        names = ("total", "no_interval", "overflow", "below", "above", "no_convergence")
         return dict(zip(names, [int(v) for v in out]))
 
     def set_overlap(self, on: bool) -> None:
@@ -274,6 +301,39 @@ class Guard:
                 _ptr(g("topk_score"), torch.float32, K) if K else None, _stream()))
         return out
 
+    def node_verdict(self, out: Optional[Dict[str, Optional[torch.Tensor]]] = None) -> Dict[str, Optional[torch.Tensor]]:
+        """Node-level fold of the evaluation just made (call right after score())."""
+        N = self.R // self.ranks_per_node
+        if out is None:
+            out = {"node_flag": torch.empty(N, dtype=torch.uint8, device=self.device),
+                   "node_tier": torch.empty(N, dtype=torch.uint8, device=self.device),
+                   "node_stall": torch.empty(N, dtype=torch.uint16, device=self.device)}
+        g = out.get
+        with torch.cuda.device(self.device):
+            self._check(lib().guard_node_verdict(self._h, _ptr(g("node_flag"), torch.uint8, N),
+                                                 _ptr(g("node_tier"), torch.uint8, N),
+                                                 _ptr(g("node_stall"), torch.uint16, N), _stream()))
+        return out
+
+    def state_bytes(self) -> int:
+        return int(lib().guard_state_bytes(self._h))
+
+    def state_export(self, state: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Copies the context's state into `state` (a uint8 CUDA tensor of state_bytes(), allocated if None)."""
+        if state is None:
+            state = torch.empty(self.state_bytes(), dtype=torch.uint8, device=self.device)
+        with torch.cuda.device(self.device):
+            self._check(lib().guard_state_export(self._h, _ptr(state, torch.uint8), state.numel(), _stream()))
+        return state
+
+    def state_import(self, state: torch.Tensor) -> None:
+        """Loads a state written by state_export of a context of the same sizes (synchronises)."""
+        with torch.cuda.device(self.device):
+            self._check(lib().guard_state_import(self._h, _ptr(state, torch.uint8), state.numel(), _stream()))
+
+    def debug_set_wait_limit(self, cycles: int) -> None:
+        self._check(lib().guard_debug_set_wait_limit(self._h, int(cycles)))
+
     def sync_status(self) -> int:
         """Synchronises the current stream; raises GuardError on a sticky device error."""
         with torch.cuda.device(self.device):
@@ -323,6 +383,35 @@ def sweep_qualify(S: torch.Tensor, nodes: int, gpus_per_node: int, *, dir: Seque
     if rc != GUARD_OK:
         raise GuardError(rc, lib().guard_last_error(None).decode())
     return out
+
+
+class Triage:
+    """Repeat-offender bookkeeping of the triage workflow: record(node, time_s) -> True when the
+    node has entered triage `limit` times within `period_s` seconds and is to be terminated."""
+
+    def __init__(self, nodes: int, limit: int = 3, period_s: int = 7 * 86400):
+        self._h = C.c_void_p()
+        rc = lib().guard_triage_create(C.byref(self._h), nodes, limit, period_s)
+        if rc != GUARD_OK:
+            raise GuardError(rc, lib().guard_last_error(None).decode())
+
+    def record(self, node: int, time_s: int):
+        n = C.c_int(0)
+        rc = lib().guard_triage_record(self._h, node, int(time_s), C.byref(n))
+        if rc < 0:
+            raise GuardError(rc, "bad node id, or a time before the node's previous entry")
+        return bool(rc), n.value
+
+    def close(self):
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.guard_triage_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 TOPK_STATIC_MAX_K = 256

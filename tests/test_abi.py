@@ -107,3 +107,40 @@ def test_key_map_is_order_preserving_and_invertible(glib):
     assert np.all(sb[:-1] >= sb[1:])                       # -0 before +0
     assert glib.key_from_float(-0.0) + 1 == glib.key_from_float(0.0)
     assert glib.key_from_float(-math.inf) < glib.key_from_float(-3e38) < glib.key_from_float(3e38) < glib.key_from_float(math.inf)
+
+
+def test_triage_counter_matches_the_oracle_rule(glib):
+    """Section 6's repeat-offender rule through the C ABI (host-only code) against the oracle's
+    statement of it, node by node, on interleaved entries."""
+    from oracle import guard_oracle as go
+    rng = np.random.default_rng(17)
+    day = 86400
+    for limit, period in ((3, 7 * day), (1, 0), (4, 3 * day), (2, 10)):
+        nodes = 6
+        t = glib.Triage(nodes, limit, period)
+        entries = sorted((int(rng.integers(0, 30 * day)), int(rng.integers(0, nodes))) for _ in range(80))
+        entries += [(entries[-1][0], 2)] * 3                     # repeated entries at the same second
+        per_node = {n: [] for n in range(nodes)}
+        got = {n: [] for n in range(nodes)}
+        for ts, n in entries:
+            term, within = t.record(n, ts)
+            per_node[n].append(ts)
+            got[n].append(int(term))
+            want_within = sum(1 for u in per_node[n] if ts - u <= period)
+            assert within == min(want_within, limit)
+        for n in range(nodes):
+            assert got[n] == go.triage(per_node[n], period, limit).tolist(), (limit, period, n)
+        with pytest.raises(glib.GuardError):
+            t.record(nodes, 0)                                   # unknown node
+        with pytest.raises(glib.GuardError):
+            t.record(2, entries[-1][0] - 1)                      # time runs backwards for node 2
+        t.close()
+    # the paper's numbers
+    t = glib.Triage(4)
+    assert [t.record(1, d * day)[0] for d in (0, 2, 5)] == [False, False, True]
+    assert [t.record(3, d * day)[0] for d in (0, 2, 8)] == [False, False, False]
+    h = C.c_void_p()
+    assert glib.lib().guard_triage_create(C.byref(h), 0, 3, 10) == -1
+    assert glib.lib().guard_triage_create(C.byref(h), 4, 0, 10) == -1
+    assert glib.lib().guard_triage_record(None, 0, 0, None) == -1
+    glib.lib().guard_triage_destroy(None)

@@ -5,9 +5,8 @@ on a GPU whose memory the training job's allocator already owns, where cudaMallo
 also stall the job by synchronising the device.  Its scratch is a fixed array inside the
 library, shared by every call on the device, so the check runs it twice in a row on
 different data: the second call must not be disturbed by what the first one left behind.
-Both results must equal guard_score's top-k bit for bit (indices) and value for value
-(scores; same kernel arithmetic, so the 1e-6 relative tolerance of the other tests is met
-with room to spare).  This file sorts last so that a stop-at-first-failure run has already
+Every result must equal the CPU oracle's top-k of the same telemetry (indices bit for bit,
+scores within the 1e-6 relative tolerance of the other tests) and guard_score's.  This file sorts last so that a stop-at-first-failure run has already
 run every other test.
 """
 import numpy as np
@@ -23,11 +22,17 @@ def _evaluation(R, M, K, seed):
     dirs = [1, 1, -1, 1][:M]
     X = np.exp(0.03 * rng.normal(size=(12, R, M)))
     X[:, rng.integers(0, R, 5), 0] *= 1.3
+    X = X.astype(np.float32)
     g = guard.Guard(R, M, 12, 6, dir=dirs, topk=K)
-    g.ingest(torch.from_numpy(X.astype(np.float32)).cuda())
+    g.ingest(torch.from_numpy(X).cuda())
     out = g.score()
     g.sync_status()
     g.close()
+    from oracle import guard_oracle as go
+    o = go.Oracle(R, M, 12, 6, K, dir=dirs)
+    o.ingest(X)
+    ref = o.score()
+    out["oracle_topk_idx"], out["oracle_topk_score"] = ref["topk_idx"], ref["topk_score"]
     return out, dirs
 
 
@@ -48,9 +53,11 @@ def test_static_scratch_topk_matches_score_twice_in_a_row():
         torch.cuda.synchronize()
         # the call itself went nowhere near torch's device allocator either
         assert torch.cuda.memory_stats()["allocation.all.allocated"] == before
+        assert np.array_equal(idx.cpu().numpy(), ref["oracle_topk_idx"])
+        got = sc.cpu().numpy().astype(np.float64)
+        assert np.allclose(got, ref["oracle_topk_score"], rtol=1e-6, atol=1e-30)
         assert torch.equal(idx, ref["topk_idx"])
-        got, want = sc.cpu().numpy().astype(np.float64), ref["topk_score"].cpu().numpy().astype(np.float64)
-        assert np.allclose(got, want, rtol=1e-6, atol=1e-30)
+        assert np.allclose(got, ref["topk_score"].cpu().numpy().astype(np.float64), rtol=1e-6, atol=1e-30)
 
 
 def test_static_scratch_limits_are_rejected():
