@@ -113,7 +113,7 @@ def test_large_configuration_ten_blocks_around_a_ramp_onset():
     wf = g.window_fallbacks()
     # ramp ranks drift away from their previous medians and carry heavy-tailed noise: a few series per
     # evaluation leave the predicted interval and are finished by the whole-warp fallback, at full width
-    assert 0 < wf["total"] < 0.01 * R * M * (nb - 1), wf
+    assert 0 < wf["total"] < 0.05 * R * M * (nb - 1), wf
     o = go.Oracle(R, M, cfg.W, cfg.k, cfg.topk, dir=dirs)
     Xh = ring.cpu().numpy()
     for j in range(nb):

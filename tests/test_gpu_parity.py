@@ -86,6 +86,93 @@ def test_wide_block_cross_rank_paths(R, M, B, T, quant):
              max_fallback_steps=0 if quant is None else None)
 
 
+@pytest.mark.parametrize("R,M,B,W,nblk,cap,quant,deferred", [
+    (4096, 8, 50, 50, 4, 100, None, False),     # block = window: window medians fused into the median pass from the 2nd block on
+    (4096, 8, 50, 50, 4, 100, None, True),      # the same in the deferred pipeline (alternating internal streams)
+    (4100, 8, 64, 64, 3, 135, None, False),     # last tile of 4 ranks; ring wraps inside a block
+    (5000, 4, 70, 70, 3, 140, None, True),      # four metrics: 64-rank tiles, last one of 8 ranks; last stage of 6 steps
+    (4096, 8, 60, 40, 3, 120, None, False),     # window shorter than the block: the fused medians skip the block's first steps
+    (4096, 8, 50, 80, 4, 160, None, False),     # window longer than the block: tile kernels without fusion
+    (4096, 8, 48, 48, 3, 96, 50, False),        # quantised: intervals collapse onto tied values, steps fall back
+    (8192, 4, 48, 48, 2, 96, 4, False),         # very coarse: kept lists overflow, every step takes the direct path
+    (16384, 8, 48, 48, 2, 96, None, True),      # width of the large configuration
+])
+def test_tile_kernels_match_oracle(R, M, B, W, nblk, cap, quant, deferred):
+    """Blocks of 48 steps and more take the tile kernels (one CTA per tile of ranks over all steps of the
+    block) for both cross-rank passes."""
+    from paper_2605_17879_b200 import guard
+    T = nblk * B
+    X, dirs = _rand_fleet(T, R, M, seed=11 * R + B + W, quant=quant)
+    Xd = torch.from_numpy(X).cuda()
+    k = max(1, W // 2)
+    o = go.Oracle(R, M, W, k, 16, dir=dirs)
+    results = {}
+    for fusion in (True, False):
+        g = guard.Guard(R, M, W, k, dir=dirs, capacity=cap, topk=16)
+        g.set_fusion(fusion)
+        g.set_deferred(deferred)
+        bufs = [g.alloc_outputs() for _ in range(nblk)]
+        stats = []
+        for j in range(nblk):
+            smed = torch.empty((B, M), dtype=torch.float32, device="cuda")
+            smad = torch.empty((B, M), dtype=torch.float32, device="cuda")
+            if deferred and j % 2 == 1:
+                g.ingest(Xd[j * B:(j + 1) * B])               # no per-step outputs: the block goes to an internal stream
+                stats.append(None)
+            else:
+                g.ingest(Xd[j * B:(j + 1) * B], smed, smad)
+                stats.append((smed, smad))
+            g.score(bufs[j])
+        g.join()
+        assert g.sync_status() == 0
+        if quant is None:
+            assert g.fallback_steps() == 0
+        results[fusion] = (bufs, stats)
+        g.close()
+    for j in range(nblk):
+        ref_i = o.ingest(X[j * B:(j + 1) * B])
+        ref = o.score()
+        for fusion in (True, False):
+            bufs, stats = results[fusion]
+            if stats[j] is not None:
+                assert_bit_equal(to_np(stats[j][0]), ref_i["step_med"], "step_med block %d" % j)
+                assert_bit_equal(to_np(stats[j][1]), ref_i["step_mad"], "step_mad block %d" % j)
+            compare_score(bufs[j], ref, "fusion=%s block %d" % (fusion, j))
+
+
+def test_tile_kernels_nonfinite_and_overflowing_deviation():
+    from paper_2605_17879_b200 import guard
+    R, M, B = 4096, 8, 48
+    X, dirs = _rand_fleet(2 * B, R, M, seed=123)
+    for m in (2, 7):
+        X[..., m] = (X[..., m] / np.median(X[..., m])) * np.float32(1e38)
+        for t in range(2 * B):
+            X[t, (37 * t + 5) % 997:R:997, m] = np.float32(-3e38)
+    g = guard.Guard(R, M, B, B // 2, dir=dirs, capacity=2 * B, topk=8)
+    o = go.Oracle(R, M, B, B // 2, 8, dir=dirs)
+    Xd = torch.from_numpy(X).cuda()
+    for t in range(0, 2 * B, B):
+        smed = torch.empty((B, M), dtype=torch.float32, device="cuda")
+        smad = torch.empty((B, M), dtype=torch.float32, device="cuda")
+        g.ingest(Xd[t:t + B], smed, smad)
+        ref_i = o.ingest(X[t:t + B])
+        out = g.score()
+        assert g.sync_status() == 0                      # finite input whose deviation overflows is not an error
+        assert_bit_equal(to_np(smed), ref_i["step_med"], "step_med")
+        assert_bit_equal(to_np(smad), ref_i["step_mad"], "step_mad")
+        compare_score(out, o.score(), "t=%d" % t)
+    assert g.fallback_steps() == 0
+    g.reset()
+    Xd[B + 7, 4000, 5] = float("inf")                    # a value that is not finite, in the last tile
+    g.ingest(Xd[:B])
+    assert g.sync_status() == 0
+    g.ingest(Xd[B:])
+    with pytest.raises(guard.GuardError) as ei:
+        g.sync_status()
+    assert ei.value.code == -4
+    g.close()
+
+
 def test_wide_block_degenerate_columns():
     # constant, two-valued and single-valued steps inside a wide block: the sample cannot
     # bracket anything, the direct path must take over for those steps only
