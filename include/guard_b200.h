@@ -264,14 +264,6 @@ int guard_reset(guard_ctx *ctx, void *stream);
 /* Enables (default) or disables the internal fork/join stream described under Conventions. */
 int guard_set_overlap(guard_ctx *ctx, int on);
 
-/* Fused window medians (on by default).  When an ingested block is the whole window of the next
- * evaluation (B >= W, after at least one earlier evaluation, fleets the tile kernels serve),
- * guard_ingest computes that evaluation's windowed per-rank medians in the same pass over the
- * block that counts for the cross-rank medians, so the block crosses HBM once for both; the
- * following guard_score then starts from those medians.  Results are identical either way;
- * guard_set_fusion(ctx, 0) makes every evaluation run its own window kernel. */
-int guard_set_fusion(guard_ctx *ctx, int on);
-
 /* Deferred evaluations (off by default).  While on, guard_score enqueues the evaluation on
  * streams of the library's own, ordered after everything enqueued on `stream` so far, and
  * `stream` does NOT wait for it: the evaluation (Section 4.2's peer comparison over the last
@@ -297,8 +289,7 @@ int guard_join(guard_ctx *ctx, void *stream);
  * stream right around the longest of its kernels (the MAD / exceedance sweep of the split
  * cross-rank path; contexts whose sizes take another path record around their main kernel or
  * nothing).  on = 2: guard_score records the pair around its window-median kernel, on the
- * stream that kernel runs on.  on = 3: guard_ingest records the pair around the median pass of a large
- * block (the tile kernel, with the window medians when they are fused into it).  guard_profile_read waits for the recorded events, returns the
+ * stream that kernel runs on.  guard_profile_read waits for the recorded events, returns the
  * sum of the kernel durations in milliseconds and their number, and forgets them.  on = 0
  * (default) switches it off and destroys any events not yet read; do not leave it on in a
  * long-running service without reading (events accumulate in host memory). */

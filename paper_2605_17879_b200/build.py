@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libguard_b200.so")
-SOURCES = ["guard_api.cu", "xrank.cu", "xrank_bracket.cu", "xrank_cluster.cu", "xrank_split.cu", "xrank_tile.cu", "xrank_column.cu", "window.cu", "score.cu", "topk.cu", "sweep.cu", "triage.cu"]
+SOURCES = ["guard_api.cu", "xrank.cu", "xrank_bracket.cu", "xrank_cluster.cu", "xrank_split.cu", "xrank_column.cu", "window.cu", "score.cu", "topk.cu", "sweep.cu", "triage.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--fmad=false",            # every decision is defined on unfused float32 operations

@@ -8,7 +8,6 @@
 
 #include "../../include/guard_b200.h"
 #include "kernels.h"
-#include "xsplit_common.cuh"
 
 using namespace guard;
 
@@ -25,7 +24,7 @@ constexpr int kIngestStreams = GUARD_INGEST_STREAMS;   // internal streams the c
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, lastflag, lasttier, ticket, fleet, xr_small, wmed, wmed_stride, stepstat, topk_cand, wspread, wcentre, xr_big, xr_big_stride, mask, ring, total;
+    size_t status, consec, lastflag, lasttier, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, xr_big, xr_big_stride, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
@@ -46,8 +45,6 @@ Layout make_layout(int R, int M, int C, int K) {
     L.xr_steps = (!L.xr_split && !L.xr_cluster && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
     L.xr_small = off;  off = align_up(off + (L.xr_steps ? xrank_scratch_small_bytes(M, L.xr_steps) : 0));
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
-    L.wmed_stride = off - L.wmed;   // a second copy: medians fused into an ingest are written beside the ones a pending evaluation reads
-    off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
     L.wspread = off;   off = align_up(off + (size_t)R * M * sizeof(float));
@@ -134,19 +131,6 @@ struct guard_ctx {
     long long evals;     // evaluations since creation / reset
     long long seen_at_eval = 0;   // steps seen at the last evaluation
     int ranks_per_node = 8;
-    // Windowed medians are kept twice.  wcur is the copy the last evaluation used (and the next one that
-    // runs a window kernel of its own overwrites).  An ingest whose block is the whole window of the next
-    // evaluation computes that evaluation's medians in its median pass, into the other copy, and notes for
-    // which step count they hold; guard_score then switches to that copy instead of launching a window kernel.
-    int wcur = 0;
-    bool fuse = true;                 // guard_set_fusion
-    long long fused_seen = -1;        // the other copy holds the medians of the window ending at this step count
-    cudaEvent_t ev_hint = nullptr;    // after the last kernel that wrote the per-series search intervals
-    bool hint_recorded = false;
-    bool ensure_hint_event() {
-        if (ev_hint) return true;
-        return cudaEventCreateWithFlags(&ev_hint, cudaEventDisableTiming) == cudaSuccess;
-    }
     long long wait_limit = 0;     // test hook: limit of the warp window path's first wait (0: default)
     // overlap of the window medians (which need only the ring) with the cross-rank kernels of the
     // ingest that precedes them: an internal stream forked from and joined into the caller's
@@ -267,8 +251,7 @@ struct guard_ctx {
     uint8_t *consec() const { return (uint8_t *)(ws + L.consec); }
     uint8_t *lastflag() const { return (uint8_t *)(ws + L.lastflag); }
     uint8_t *lasttier() const { return (uint8_t *)(ws + L.lasttier); }
-    float *wmed(int which) const { return (float *)(ws + L.wmed + (size_t)(which & 1) * L.wmed_stride); }
-    float *wmed() const { return wmed(wcur); }
+    float *wmed() const { return (float *)(ws + L.wmed); }
     float *step_med() const { return (float *)(ws + L.stepstat); }
     float *step_mad() const { return step_med() + (size_t)C * M; }
     unsigned long long *topk_cand() const { return (unsigned long long *)(ws + L.topk_cand); }
@@ -279,9 +262,7 @@ struct guard_ctx {
     // own_scratch = false: the call may run beside another cross-rank call of this context (the fleet
     // baseline of a deferred evaluation beside the next ingest), so it must not touch the one
     // scratch of the bracketed path: such rows take the direct selection.
-    // win: window medians to fuse into the median pass (only honoured where the whole call is one launch
-    // group of the tile kernels; the caller checks that with xrank_split_uses_tiles).
-    cudaError_t xrank(XrankArgs a, int S, cudaStream_t st, bool own_scratch = true, const TileWindow *win = nullptr) {
+    cudaError_t xrank(XrankArgs a, int S, cudaStream_t st, bool own_scratch = true) {
         // a few rows at a time: one CTA per column keeps the whole GPU busy
         if (xrank_column_supported(R) && (long long)S * M <= 64 && !a.cut) {
             launches += 1;
@@ -299,10 +280,8 @@ struct guard_ctx {
                 g.mad = a.mad + (size_t)s0 * M;
                 if (a.med_user) g.med_user = a.med_user + (size_t)s0 * M;
                 if (a.mad_user) g.mad_user = a.mad_user + (size_t)s0 * M;
-                const bool fuse_here = win && S <= smax;
                 cudaError_t e = launch_xrank_split(g, p, n, ws + L.xr_big + (size_t)scratch_sel * L.xr_big_stride, status() + 2, st,
-                                                   ((profiling == 1 || profiling == 3) && a.mask_base) ? &prof : nullptr, profiling,
-                                                   fuse_here ? win : nullptr, fuse_here ? ev_hint : nullptr);
+                                                   (profiling == 1 && a.mask_base) ? &prof : nullptr);
                 if (e != cudaSuccess) return e;
                 launches += 6;
             }
@@ -341,18 +320,6 @@ struct guard_ctx {
         const cudaError_t e = launch_window_select(w, ws_);
         cudaEventRecord(e1, ws_);
         prof.emplace_back(e0, e1);
-        return e;
-    }
-    // A window kernel reads and rewrites the per-series search intervals: it runs behind their last
-    // writer (possibly an ingest on another stream) and becomes the last writer itself.
-    cudaError_t window_after_hints(const WindowArgs &w, cudaStream_t ws_) {
-        cudaError_t e = cudaSuccess;
-        if (hint_recorded) e = cudaStreamWaitEvent(ws_, ev_hint, 0);
-        if (e == cudaSuccess) e = window(w, ws_);
-        if (e == cudaSuccess && ensure_hint_event()) {
-            e = cudaEventRecord(ev_hint, ws_);
-            hint_recorded = e == cudaSuccess;
-        }
         return e;
     }
     int fail(int code, const char *fmt, ...) {
@@ -458,51 +425,25 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
     a.check_finite = 1;
     a.status = c->status();
     cudaError_t e;
-    // The block is the whole window of the next evaluation (and the per-series search intervals of an
-    // earlier evaluation exist): its median pass computes that evaluation's windowed medians as well.
-    const long long seen_after = c->seen + B;
-    const int n_after = (int)(seen_after < c->W ? seen_after : c->W);
-    const bool fuse = c->fuse && c->L.xr_split && a.mask_bytes == 1 && c->evals > 0 && n_after <= B && n_after <= 256 &&
-                      B <= kSplitMaxSteps && xrank_split_uses_tiles(c->R, c->M, B) && c->ensure_hint_event();
-    TileWindow tw{};
-    if (fuse) {
-        tw.enabled = 1;
-        tw.n = n_after;
-        tw.wmed = c->wmed(c->wcur ^ 1);
-        tw.spread = (float *)(c->ws + c->L.wspread);
-        tw.centre = (float *)(c->ws + c->L.wcentre);
-        tw.fb_count = c->status() + 8;
-    }
     const bool piped = c->deferred && c->L.xr_split && a.mask_bytes == 1 && (long long)B * c->M > 64 && !d_step_med &&
                        !d_step_mad && c->ensure_xs();
-    cudaStream_t run = piped ? c->xs[c->xs_next] : st;
-    if (piped) {
-        e = cudaEventRecord(c->ev_data, st);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(run, c->ev_data, 0);
-        if (e != cudaSuccess) return c->cuda_fail(e, "fork of the ingest stream");
-    }
-    if (fuse && c->hint_recorded) {   // the intervals' last writer may have run on another stream
-        e = cudaStreamWaitEvent(run, c->ev_hint, 0);
-        if (e != cudaSuccess) return c->cuda_fail(e, "wait for the search intervals");
-    }
     if (piped) {
         const int k = c->xs_next;
         c->xs_next = (k + 1) % kIngestStreams;
+        e = cudaEventRecord(c->ev_data, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(c->xs[k], c->ev_data, 0);
+        if (e != cudaSuccess) return c->cuda_fail(e, "fork of the ingest stream");
         c->scratch_sel = k;
-        e = c->xrank(a, B, c->xs[k], true, fuse ? &tw : nullptr);
+        e = c->xrank(a, B, c->xs[k]);
         c->scratch_sel = 0;
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_xs[k], c->xs[k]);
         if (!c->xs_busy[k]) c->xs_first[k] = c->seen;
         c->xs_busy[k] = true;
     } else {
         e = c->join_xs(st);   // earlier blocks still on the internal streams come first
-        if (e == cudaSuccess) e = c->xrank(a, B, st, true, fuse ? &tw : nullptr);
+        if (e == cudaSuccess) e = c->xrank(a, B, st);
     }
     if (e != cudaSuccess) return c->cuda_fail(e, "xrank launch");
-    if (fuse) {
-        c->fused_seen = seen_after;
-        c->hint_recorded = true;
-    }
     c->seen += B;
     return GUARD_OK;
 }
@@ -517,10 +458,6 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     const int last = (int)((c->seen - 1) % c->C);
     const size_t row = (size_t)c->R * c->M;
 
-    // medians an ingest has already computed for exactly this window: switch to their copy
-    const bool fused = c->fused_seen == c->seen;
-    if (fused) c->wcur ^= 1;
-    c->fused_seen = -1;
     WindowArgs w{};
     w.ring = c->ring();
     w.row_stride = (long long)row;
@@ -565,27 +502,23 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
             e = cudaEventRecord(c->ev_fork, st);
             if (e != cudaSuccess) return c->cuda_fail(e, "event record");
         }
-        if (!fused) {
-            e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
-            if (e == cudaSuccess && had_pending) e = cudaStreamWaitEvent(c->side, c->ev_e, 0);
-            if (e == cudaSuccess) e = c->window_after_hints(w, c->side);
-            if (e == cudaSuccess) e = cudaEventRecord(c->ev_w, c->side);
-            if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_w, 0);
-        }
+        e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
+        if (e == cudaSuccess && had_pending) e = cudaStreamWaitEvent(c->side, c->ev_e, 0);
+        if (e == cudaSuccess) e = c->window(w, c->side);
+        if (e == cudaSuccess) e = cudaEventRecord(c->ev_w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_x, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_w, 0);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(c->tail, c->ev_x, 0);
         for (int k = 0; k < kIngestStreams && e == cudaSuccess; ++k)   // cross-rank kernels of the window's blocks on the ingest streams
             if (c->xs_busy[k]) e = cudaStreamWaitEvent(c->tail, c->ev_xs[k], 0);
         ts = c->tail;
-    } else if (fused) {
-        e = cudaSuccess;   // the medians were enqueued with the ingest, which `st` is ordered behind
     } else if (forked) {
         e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
-        if (e == cudaSuccess) e = c->window_after_hints(w, c->side);
+        if (e == cudaSuccess) e = c->window(w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_join, c->side);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_join, 0);
     } else {
-        e = c->window_after_hints(w, st);
+        e = c->window(w, st);
     }
     if (e != cudaSuccess) return c->cuda_fail(e, "window_select launch");
 
@@ -608,7 +541,6 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     s.R = c->R;
     s.M = c->M;
     s.wmed = c->wmed();
-    s.wmed_user = fused ? d_wmed : nullptr;   // a window kernel writes the caller's copy itself
     s.fleet_med = c->fleet_med();
     s.fleet_mad = c->fleet_mad();
     s.mask_base = c->mask();
@@ -652,7 +584,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     e = launch_score_flag(s, c->p, ts);
     if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
     c->evals += 1;
-    c->launches += 1 + (fused ? 0 : window_launch_count(w));
+    c->launches += 1 + window_launch_count(w);
     if (topk_forked) {
         e = cudaStreamWaitEvent(ts, c->ev_join, 0);
         if (e != cudaSuccess) return c->cuda_fail(e, "topk join");
@@ -907,7 +839,6 @@ int guard_state_import(guard_ctx *c, const void *d_state, size_t state_bytes, vo
     c->seen = h.seen;
     c->evals = h.evals;
     c->seen_at_eval = h.seen_at_eval;
-    c->fused_seen = -1;
     c->fork_fresh = false;
     return GUARD_OK;
 }
@@ -940,7 +871,6 @@ int guard_reset(guard_ctx *c, void *stream) {
     c->seen = 0;
     c->evals = 0;
     c->seen_at_eval = 0;
-    c->fused_seen = -1;
     return GUARD_OK;
 }
 
@@ -1007,12 +937,6 @@ int64_t guard_fallback_steps(guard_ctx *c, void *stream) {
     return (int64_t)n;
 }
 
-int guard_set_fusion(guard_ctx *c, int on) {
-    if (!c) return GUARD_ERR_ARG;
-    c->fuse = on != 0;
-    return GUARD_OK;
-}
-
 int guard_set_deferred(guard_ctx *c, int on) {
     if (!c) return GUARD_ERR_ARG;
     c->deferred = on != 0;
@@ -1051,7 +975,6 @@ void guard_destroy(guard_ctx *c) {
             cudaEventDestroy(c->ev_w);
             cudaEventDestroy(c->ev_e);
         }
-        if (c->ev_hint) cudaEventDestroy(c->ev_hint);
         if (c->side) {
             cudaStreamDestroy(c->side);
             cudaEventDestroy(c->ev_fork);

@@ -60,14 +60,8 @@ constexpr int kWindowNearTarget = 14;
 constexpr float kWindowNearSmooth = 1.0f;
 constexpr int kSplitMaxSteps = 256;   // steps per launch group of the split path (sizes its scratch)
 size_t xrank_split_scratch_bytes(int R, int M, int S_max);
-struct TileWindow;   // window medians fused into the median pass of a large block (xsplit_common.cuh)
-// prof_mode 1: the events go around the MAD / exceedance pass, 3: around the median pass.  after_median (or
-// nullptr) is recorded once the median pass, and with it any fused window medians, has been enqueued.
 cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S, void *scratch, uint32_t *reasons,
-                               cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof = nullptr,
-                               int prof_mode = 1, const TileWindow *win = nullptr, cudaEvent_t after_median = nullptr);
-// True when a block of S steps takes the tile kernels (then window medians can be fused into its median pass).
-bool xrank_split_uses_tiles(int R, int M, int S);
+                               cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof = nullptr);
 bool xrank_bracket_supported(int R, int M);
 int xrank_scratch_steps(int R, int M, int want);
 size_t xrank_scratch_small_bytes(int M, int S_max);   // must be zero before first use
@@ -105,7 +99,6 @@ int window_launch_count(const WindowArgs &a);
 struct ScoreArgs {
     int R, M;
     const float *wmed;       // [R][M]
-    float *wmed_user;        // [R][M] copy for the caller, or NULL (medians that no window kernel of this evaluation wrote out)
     const float *fleet_med;  // [M]
     const float *fleet_mad;  // [M]
     const void *mask_base;   // exceedance rows [capacity][R]

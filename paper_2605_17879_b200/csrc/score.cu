@@ -44,7 +44,6 @@ __global__ void __launch_bounds__(kScoreThreads) score_flag_kernel(const ScoreAr
     for (int m = 0; m < NM; ++m) {
         if (m < M) {
             const float x = w[m];
-            if (a.wmed_user) a.wmed_user[(size_t)r * M + m] = x;
             float dev = __fsub_rn(x, s_B[m]);
             if (p.dir[m] < 0) dev = -dev;
             const bool zflag = dev > s_rhs[m];
@@ -166,7 +165,6 @@ __global__ void __launch_bounds__(kFastWarps * 32) score_flag_bytes_kernel(const
     for (int m = 0; m < 8; ++m) {
         if (m < M) {
             const int cnt = (int)s_cnt[tid][m];
-            if (a.wmed_user) a.wmed_user[(size_t)r * M + m] = wv[m];
             float dev = __fsub_rn(wv[m], s_B[m]);
             if (p.dir[m] < 0) dev = -dev;
             if (dev > s_rhs[m] && cnt >= p.k) mask |= 1u << m;

@@ -27,12 +27,53 @@
 
 #include <mutex>
 
-#include "xsplit_common.cuh"
+#include "xrank_common.cuh"
 #include "xrank_direct.cuh"
 
 namespace guard {
 
 namespace {
+
+constexpr int kSpThreads = 256;     // sweep CTA
+constexpr int kSpU = 4;             // ranks per thread and sweep batch
+constexpr int kSpSlice = 4096;      // ranks per sweep CTA
+constexpr int kSpSlack = 128;       // words behind each shared-memory list that absorb the stores of a full list
+constexpr int kSpAmb = 1024;        // deferred exceedance decisions per step
+constexpr int kSpSample = 4096;     // target number of sampled ranks per column
+constexpr int kSpSBins = 2048;      // sample histogram bins (16-bit counters, two per word)
+constexpr int kSpBins = 1024;       // selection histogram bins
+constexpr int kSpSelThreads = 128;  // sample / select CTA
+constexpr int kSpJmax = 20;         // kept elements per thread the register selection can hold
+constexpr int kSpSegs = 4;          // sweep CTAs per step the selection can gather from
+constexpr int kSpMaxM = 8;
+constexpr float kFltMax = 3.402823466e+38f;
+
+struct SpGeom {
+    int chunks;     // sweep CTAs per step
+    int slice;      // ranks per sweep CTA (a multiple of 16)
+    int cap;        // kept elements per metric and sweep CTA (its shared-memory list and its segment in global scratch)
+    int stride;     // one run of four consecutive ranks is sampled out of every 4 * stride
+    int s;          // number of sampled ranks
+    int delta;      // half-width of the median interval in sample ranks
+    int delta_q;    // half-width of the quartile intervals in sample ranks
+};
+
+// Per-column record in global scratch.
+struct SpCol {
+    float lo, hi, dlo, dhi;   // intervals of the median and of the MAD
+    float med, rlo, rhi, rhs; // median; range of the exceedance threshold over [dlo, dhi]; exact threshold
+    uint32_t cnt;             // elements below the current interval
+    uint32_t pad[3];
+};
+
+struct SpScratch {
+    SpCol *col;       // [S][M]
+    uint32_t *fail;   // [S] the step goes to the direct path
+    uint32_t *namb;   // [S] deferred exceedance decisions
+    uint32_t *amb;    // [S][kSpAmb] (rank << 5 | metric)
+    uint32_t *nseg;   // [S][M][chunks] kept elements of each sweep CTA
+    uint32_t *list;   // [S][M][chunks][cap] kept elements (raw bits), one segment per sweep CTA
+};
 
 // ---- per-element operations of the sweeps, written out so that each is a fixed handful of
 // instructions (compare, predicated add / predicated store) ---------------------------------
@@ -129,11 +170,6 @@ __global__ void __launch_bounds__(kSpSmpThreads, 3) xsplit_sample_kernel(const X
         col.cnt = 0;
     }
     if (tid == 0 && q == 0) { sc.fail[t] = 0; sc.namb[t] = 0; }
-    if (sc.tile && tid < 2) {   // the tile kernels' packed counters of this (step, quad), both passes
-        const size_t i = ((size_t)tid * gridDim.y + t) * gridDim.x + q;
-        sc.cnt64[i] = 0ull;
-        sc.nk64[i] = 0ull;
-    }
     if (tid == 0) {
         const int mid = g.s / 2, q1 = g.s / 4, q3 = (3 * g.s) / 4;
         const int tk[6] = {mid - g.delta, mid + g.delta, q1 - g.delta_q, q1 + g.delta_q, q3 - g.delta_q, q3 + g.delta_q};
@@ -232,10 +268,6 @@ __global__ void __launch_bounds__(kSpSmpThreads, 3) xsplit_sample_kernel(const X
             if (dhi > kFltMax) dhi = kFltMax;
         }
         col.lo = lo; col.hi = hi; col.dlo = dlo; col.dhi = dhi;
-        if (sc.tile) {
-            const size_t i = (size_t)t * M + 4 * q + cc;
-            sc.blo[i] = lo; sc.bhi[i] = hi; sc.bdlo[i] = dlo; sc.bdhi[i] = dhi;
-        }
         if (!ok) {
             atomicOr(&sc.fail[t], 1u);
             if (reasons) atomicAdd(reasons + kWhySelect, 1u);
@@ -472,28 +504,19 @@ __device__ __forceinline__ void sp_find_bin(SpSelShared &sh, uint32_t k) {
 // narrower range; then the bin's keys are gathered and one warp ranks them.  The next order
 // statistic is the following gathered key or, if the bin ends there, the smallest key above it.
 template <int JMAX>
-__device__ bool sp_select_regs(const uint32_t *__restrict__ list, const int cap, const bool contig, const uint32_t (&nseg)[kSpSegs], uint32_t k,
+__device__ bool sp_select_regs(const uint32_t *__restrict__ list, const int cap, const uint32_t (&nseg)[kSpSegs], uint32_t k,
                                bool want_next, uint32_t base, uint32_t width, SpSelShared &sh, uint32_t &v1, uint32_t &v2) {
     constexpr int G = kSpSelThreads, JS = JMAX / kSpSegs;   // registers per segment
     const int tid = threadIdx.x;
     uint32_t off[JMAX];   // key - base; 0xFFFFFFFF (beyond any width) where there is no element
-    if (contig) {         // one list of nseg[0] elements
 #pragma unroll
-        for (int j = 0; j < JMAX; ++j) {
+    for (int sg = 0; sg < kSpSegs; ++sg)
+#pragma unroll
+        for (int j = 0; j < JS; ++j) {
             const uint32_t i = (uint32_t)(tid + j * G);
-            off[j] = 0x7F800000u;
-            if (i < nseg[0]) off[j] = list[i];
+            off[sg * JS + j] = 0x7F800000u;   // bits of +inf: its key lies above every finite key
+            if (i < nseg[sg]) off[sg * JS + j] = list[(size_t)sg * cap + i];
         }
-    } else {
-#pragma unroll
-        for (int sg = 0; sg < kSpSegs; ++sg)
-#pragma unroll
-            for (int j = 0; j < JS; ++j) {
-                const uint32_t i = (uint32_t)(tid + j * G);
-                off[sg * JS + j] = 0x7F800000u;   // bits of +inf: its key lies above every finite key
-                if (i < nseg[sg]) off[sg * JS + j] = list[(size_t)sg * cap + i];
-            }
-    }
 #pragma unroll
     for (int j = 0; j < JMAX; ++j) {
         const uint32_t key = key_of_bits(off[j]);
@@ -590,22 +613,14 @@ __global__ void __launch_bounds__(kSpSelThreads, 12) xsplit_select_kernel(const 
     SpCol &col = sc.col[so + m];
     const bool even = (R & 1) == 0;
     const uint32_t k1 = (uint32_t)((R - 1) / 2), k2 = (uint32_t)(R / 2);
-    uint32_t clt = col.cnt;
+    const uint32_t clt = col.cnt;
     uint32_t nseg[kSpSegs], n = 0;
     bool over = false;
-    if (sc.tile) {   // packed counters of the tile kernels: 16 bits per metric of the quad
-        const size_t i = ((size_t)MODE * gridDim.y + t) * (M / 4) + (m >> 2);
-        clt = (uint32_t)(sc.cnt64[i] >> (16 * (m & 3))) & 0xFFFFu;
-        n = (uint32_t)(sc.nk64[i] >> (16 * (m & 3))) & 0xFFFFu;
-        nseg[0] = n; nseg[1] = nseg[2] = nseg[3] = 0u;
-        over = n > (uint32_t)kTileCap;
-    } else {
 #pragma unroll
-        for (int sg = 0; sg < kSpSegs; ++sg) {
-            nseg[sg] = sg < g.chunks ? sc.nseg[(so + m) * g.chunks + sg] : 0u;
-            over |= nseg[sg] > (uint32_t)g.cap;
-            n += nseg[sg];
-        }
+    for (int sg = 0; sg < kSpSegs; ++sg) {
+        nseg[sg] = sg < g.chunks ? sc.nseg[(so + m) * g.chunks + sg] : 0u;
+        over |= nseg[sg] > (uint32_t)g.cap;
+        n += nseg[sg];
     }
     const float flo = MODE == 0 ? col.lo : col.dlo, fhi = MODE == 0 ? col.hi : col.dhi;
     int why = -1;
@@ -616,8 +631,7 @@ __global__ void __launch_bounds__(kSpSelThreads, 12) xsplit_select_kernel(const 
     if (why < 0) {
         const uint32_t base = f2key((MODE == 0 && flo == 0.0f) ? -0.0f : flo);
         const uint32_t width = f2key((MODE == 0 && fhi == 0.0f) ? 0.0f : fhi) - base;
-        const uint32_t *lst = sc.tile ? sc.clist + (so + m) * kTileCap : sc.list + (so + m) * g.chunks * g.cap;
-        if (!sp_select_regs<kSpJmax>(lst, g.cap, sc.tile != 0, nseg, k1 - clt, even, base, width, sh, v1, v2))
+        if (!sp_select_regs<kSpJmax>(sc.list + (so + m) * g.chunks * g.cap, g.cap, nseg, k1 - clt, even, base, width, sh, v1, v2))
             why = kWhySelect;
     }
     if (tid == 0) {
@@ -631,7 +645,6 @@ __global__ void __launch_bounds__(kSpSelThreads, 12) xsplit_select_kernel(const 
                 col.rlo = __fmul_rn(p.thrp[m], fmaxf(fmaxf(col.dlo, rel), p.floor_abs[m]));
                 col.rhi = __fmul_rn(p.thrp[m], fmaxf(fmaxf(col.dhi, rel), p.floor_abs[m]));
                 col.cnt = 0;   // the MAD sweep counts anew
-                if (sc.tile) { sc.bmed[so + m] = val; sc.brlo[so + m] = col.rlo; }
             } else {
                 a.mad[so + m] = val;
                 if (a.mad_user) a.mad_user[so + m] = val;
@@ -710,10 +723,6 @@ bool xrank_split_supported(int R, int M) {
     return split_sweep_smem(g, M) <= 64 * 1024;
 }
 
-bool xrank_split_uses_tiles(int R, int M, int S) {
-    return xrank_split_supported(R, M) && xrank_tile_supported(R, M, S) && S >= kTileMinSteps && S <= kSplitMaxSteps;
-}
-
 size_t xrank_split_scratch_bytes(int R, int M, int S_max) {
     const SpGeom g = split_geometry(R);
     size_t b = 0;
@@ -722,17 +731,11 @@ size_t xrank_split_scratch_bytes(int R, int M, int S_max) {
     b += align256((size_t)S_max * kSpAmb * sizeof(uint32_t));
     b += align256((size_t)S_max * M * g.chunks * sizeof(uint32_t));
     b += align256((size_t)S_max * M * g.chunks * g.cap * sizeof(uint32_t));
-    if (xrank_tile_supported(R, M, S_max)) {
-        b += 2 * align256((size_t)2 * S_max * (M / 4) * sizeof(unsigned long long));
-        b += 6 * align256((size_t)S_max * M * sizeof(float));
-        b += align256((size_t)S_max * M * kTileCap * sizeof(uint32_t));
-    }
     return b;
 }
 
 cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S, void *scratch, uint32_t *reasons,
-                               cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof, int prof_mode,
-                               const TileWindow *win, cudaEvent_t after_median) {
+                               cudaStream_t st, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> *prof) {
     if (S <= 0) return cudaSuccess;
     const int M = a.M;
     const SpGeom g = split_geometry(a.R);
@@ -743,19 +746,7 @@ cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S,
     sc.namb = (uint32_t *)b;  b += align256((size_t)S * sizeof(uint32_t));
     sc.amb = (uint32_t *)b;   b += align256((size_t)S * kSpAmb * sizeof(uint32_t));
     sc.nseg = (uint32_t *)b;  b += align256((size_t)S * M * g.chunks * sizeof(uint32_t));
-    sc.list = (uint32_t *)b;  b += align256((size_t)S * M * g.chunks * g.cap * sizeof(uint32_t));
-    // Blocks of many steps take the tile kernels (one CTA per tile of ranks over all steps) instead of
-    // the chunked sweeps (one CTA per step and chunk of ranks): their grid does not depend on the
-    // number of steps, so short blocks stay with the sweeps.
-    const bool tile = xrank_tile_supported(a.R, M, S) && S >= kTileMinSteps && a.mask_base != nullptr;
-    sc.tile = tile ? 1 : 0;
-    if (tile) {
-        sc.cnt64 = (unsigned long long *)b;  b += align256((size_t)2 * S * (M / 4) * sizeof(unsigned long long));
-        sc.nk64 = (unsigned long long *)b;   b += align256((size_t)2 * S * (M / 4) * sizeof(unsigned long long));
-        float **soa[6] = {&sc.blo, &sc.bhi, &sc.bdlo, &sc.bdhi, &sc.bmed, &sc.brlo};
-        for (int i = 0; i < 6; ++i) { *soa[i] = (float *)b; b += align256((size_t)S * M * sizeof(float)); }
-        sc.clist = (uint32_t *)b;
-    }
+    sc.list = (uint32_t *)b;
     const size_t smem = split_sweep_smem(g, M);
     static std::mutex attr_mutex;
     static bool attr_set_dev[64] = {};
@@ -775,25 +766,14 @@ cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S,
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     if (prof && (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess)) return cudaGetLastError();
     const dim3 gcol(M, S), gsw(g.chunks, S);
-    TileWindow nowin{};
     xsplit_sample_kernel<<<dim3(M / 4, S), kSpSmpThreads, 0, st>>>(a, g, sc, reasons);
-    if (prof && prof_mode == 3) cudaEventRecord(ev0, st);   // the median pass (with the fused window medians)
-    if (tile) e = launch_xtile_sweep(0, a, p, sc, S, win ? *win : nowin, st);
-    else if (M == 8) xsplit_sweep_kernel<2, 0><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
+    if (M == 8) xsplit_sweep_kernel<2, 0><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
     else xsplit_sweep_kernel<1, 0><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
-    if (prof && prof_mode == 3) cudaEventRecord(ev1, st);
-    if (e != cudaSuccess) return e;
-    if (after_median) {   // the windowed medians (if fused) are complete from here on
-        e = cudaEventRecord(after_median, st);
-        if (e != cudaSuccess) return e;
-    }
     xsplit_select_kernel<0><<<gcol, kSpSelThreads, 0, st>>>(a, p, g, sc, reasons);
-    if (prof && prof_mode != 3) cudaEventRecord(ev0, st);   // the MAD / exceedance pass
-    if (tile) e = launch_xtile_sweep(1, a, p, sc, S, nowin, st);
-    else if (M == 8) xsplit_sweep_kernel<2, 1><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
+    if (prof) cudaEventRecord(ev0, st);   // the MAD / exceedance sweep, the longest kernel of the six
+    if (M == 8) xsplit_sweep_kernel<2, 1><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
     else xsplit_sweep_kernel<1, 1><<<gsw, kSpThreads, smem, st>>>(a, p, g, sc);
-    if (prof && prof_mode != 3) cudaEventRecord(ev1, st);
-    if (e != cudaSuccess) return e;
+    if (prof) cudaEventRecord(ev1, st);
     xsplit_select_kernel<1><<<gcol, kSpSelThreads, 0, st>>>(a, p, g, sc, reasons);
     xsplit_finish_kernel<<<S, kSpThreads, (size_t)M * 256 * sizeof(uint32_t), st>>>(a, p, sc);
     e = cudaGetLastError();

@@ -97,8 +97,6 @@ def lib():
         L.guard_window_fallbacks.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.guard_set_overlap.restype = C.c_int
         L.guard_set_overlap.argtypes = [vp, C.c_int]
-        L.guard_set_fusion.restype = C.c_int
-        L.guard_set_fusion.argtypes = [vp, C.c_int]
         L.guard_set_deferred.restype = C.c_int
         L.guard_set_deferred.argtypes = [vp, C.c_int]
         L.guard_join.restype = C.c_int
@@ -234,10 +232,6 @@ class Guard:
         """Window medians of an evaluation on an internal stream overlapping the preceding ingest."""
         self._check(lib().guard_set_overlap(self._h, 1 if on else 0))
 
-    def set_fusion(self, on: bool) -> None:
-        """Window medians fused into the ingest of a block that is the next evaluation's whole window (default on)."""
-        self._check(lib().guard_set_fusion(self._h, 1 if on else 0))
-
     def set_deferred(self, on: bool) -> None:
         """Deferred evaluations: score() does not make the current stream wait for its results; they
         are complete after the next score(), join(), sync_status() or reset()."""
@@ -249,8 +243,7 @@ class Guard:
             self._check(lib().guard_join(self._h, _stream()))
 
     def profile_enable(self, on=True) -> None:
-        """0 / False: off; 1 / True: time the MAD pass of every ingest; 2: the window kernel of every evaluation;
-        3: the median pass of every large ingested block."""
+        """0 / False: off; 1 / True: time the MAD sweep of every ingest; 2: the window kernel of every evaluation."""
         self._check(lib().guard_profile_enable(self._h, int(on)))
 
     def profile_read(self):

@@ -87,60 +87,55 @@ def test_wide_block_cross_rank_paths(R, M, B, T, quant):
 
 
 @pytest.mark.parametrize("R,M,B,W,nblk,cap,quant,deferred", [
-    (4096, 8, 50, 50, 4, 100, None, False),     # block = window: window medians fused into the median pass from the 2nd block on
+    (4096, 8, 50, 50, 4, 100, None, False),     # block = window; two sweep CTAs per step
     (4096, 8, 50, 50, 4, 100, None, True),      # the same in the deferred pipeline (alternating internal streams)
-    (4100, 8, 64, 64, 3, 135, None, False),     # last tile of 4 ranks; ring wraps inside a block
-    (5000, 4, 70, 70, 3, 140, None, True),      # four metrics: 64-rank tiles, last one of 8 ranks; last stage of 6 steps
-    (4096, 8, 60, 40, 3, 120, None, False),     # window shorter than the block: the fused medians skip the block's first steps
-    (4096, 8, 50, 80, 4, 160, None, False),     # window longer than the block: tile kernels without fusion
+    (4100, 8, 64, 64, 3, 135, None, False),     # last sweep CTA of a step holds 4 ranks; ring wraps inside a block
+    (5000, 4, 70, 70, 3, 140, None, True),      # four metrics: 4096-rank slices, ragged second slice
+    (4096, 8, 60, 40, 3, 120, None, False),     # window shorter than the block
+    (4096, 8, 50, 80, 4, 160, None, False),     # window longer than the block
     (4096, 8, 48, 48, 3, 96, 50, False),        # quantised: intervals collapse onto tied values, steps fall back
     (8192, 4, 48, 48, 2, 96, 4, False),         # very coarse: kept lists overflow, every step takes the direct path
     (16384, 8, 48, 48, 2, 96, None, True),      # width of the large configuration
+    (18000, 8, 20, 20, 2, 40, None, False),     # wider than the split path takes: one cluster per step
 ])
-def test_tile_kernels_match_oracle(R, M, B, W, nblk, cap, quant, deferred):
-    """Blocks of 48 steps and more take the tile kernels (one CTA per tile of ranks over all steps of the
-    block) for both cross-rank passes."""
+def test_many_step_blocks_match_oracle(R, M, B, W, nblk, cap, quant, deferred):
+    """Blocks of many steps on the split cross-rank path (per-step statistics, evaluations, with and without
+    per-step outputs, default and deferred mode)."""
     from paper_2605_17879_b200 import guard
     T = nblk * B
     X, dirs = _rand_fleet(T, R, M, seed=11 * R + B + W, quant=quant)
     Xd = torch.from_numpy(X).cuda()
     k = max(1, W // 2)
     o = go.Oracle(R, M, W, k, 16, dir=dirs)
-    results = {}
-    for fusion in (True, False):
-        g = guard.Guard(R, M, W, k, dir=dirs, capacity=cap, topk=16)
-        g.set_fusion(fusion)
-        g.set_deferred(deferred)
-        bufs = [g.alloc_outputs() for _ in range(nblk)]
-        stats = []
-        for j in range(nblk):
-            smed = torch.empty((B, M), dtype=torch.float32, device="cuda")
-            smad = torch.empty((B, M), dtype=torch.float32, device="cuda")
-            if deferred and j % 2 == 1:
-                g.ingest(Xd[j * B:(j + 1) * B])               # no per-step outputs: the block goes to an internal stream
-                stats.append(None)
-            else:
-                g.ingest(Xd[j * B:(j + 1) * B], smed, smad)
-                stats.append((smed, smad))
-            g.score(bufs[j])
-        g.join()
-        assert g.sync_status() == 0
-        if quant is None:
-            assert g.fallback_steps() == 0
-        results[fusion] = (bufs, stats)
-        g.close()
+    g = guard.Guard(R, M, W, k, dir=dirs, capacity=cap, topk=16)
+    g.set_deferred(deferred)
+    bufs = [g.alloc_outputs() for _ in range(nblk)]
+    stats = []
+    for j in range(nblk):
+        smed = torch.empty((B, M), dtype=torch.float32, device="cuda")
+        smad = torch.empty((B, M), dtype=torch.float32, device="cuda")
+        if deferred and j % 2 == 1:
+            g.ingest(Xd[j * B:(j + 1) * B])               # no per-step outputs: the block goes to an internal stream
+            stats.append(None)
+        else:
+            g.ingest(Xd[j * B:(j + 1) * B], smed, smad)
+            stats.append((smed, smad))
+        g.score(bufs[j])
+    g.join()
+    assert g.sync_status() == 0
+    if quant is None:
+        assert g.fallback_steps() == 0
+    g.close()
     for j in range(nblk):
         ref_i = o.ingest(X[j * B:(j + 1) * B])
         ref = o.score()
-        for fusion in (True, False):
-            bufs, stats = results[fusion]
-            if stats[j] is not None:
-                assert_bit_equal(to_np(stats[j][0]), ref_i["step_med"], "step_med block %d" % j)
-                assert_bit_equal(to_np(stats[j][1]), ref_i["step_mad"], "step_mad block %d" % j)
-            compare_score(bufs[j], ref, "fusion=%s block %d" % (fusion, j))
+        if stats[j] is not None:
+            assert_bit_equal(to_np(stats[j][0]), ref_i["step_med"], "step_med block %d" % j)
+            assert_bit_equal(to_np(stats[j][1]), ref_i["step_mad"], "step_mad block %d" % j)
+        compare_score(bufs[j], ref, "block %d" % j)
 
 
-def test_tile_kernels_nonfinite_and_overflowing_deviation():
+def test_split_path_nonfinite_and_overflowing_deviation():
     from paper_2605_17879_b200 import guard
     R, M, B = 4096, 8, 48
     X, dirs = _rand_fleet(2 * B, R, M, seed=123)
