@@ -20,7 +20,8 @@
  *     guard_destroy.
  *   - `stream` is a cudaStream_t passed as void*.  All work is ordered on it.  The calls that
  *     synchronise `stream` with the host are the ones that hand a value back from the device:
- *     guard_sync_status, guard_fallback_steps, guard_fallback_reasons and guard_state_import;
+ *     guard_sync_status, guard_fallback_steps, guard_fallback_reasons, guard_window_fallbacks,
+ *     guard_sliding_rebuilds and guard_state_import;
  *     guard_profile_read waits for the events it recorded.  No other call synchronises.
  *     (guard_score may run the window medians on an internal stream forked from and joined back
  *     into `stream` with events, so that they overlap the preceding guard_ingest; to the caller
@@ -264,6 +265,15 @@ int guard_reset(guard_ctx *ctx, void *stream);
 /* Enables (default) or disables the internal fork/join stream described under Conventions. */
 int guard_set_overlap(guard_ctx *ctx, int on);
 
+/* Sliding evaluations (on by default).  When an evaluation follows the previous one by at most 8
+ * steps (the online monitor of Sec. 4.2 / 7.1 re-evaluates every step or poll), consecutive
+ * windows share almost all their steps; guard_score then updates a small per-series state (an
+ * interval around the series' median, the count of window values below it, the values inside)
+ * from the few steps that entered and left the window instead of reading the whole window again.
+ * Series whose median has left their interval are rebuilt from the window.  Results are identical
+ * either way; guard_set_sliding(ctx, 0) makes every evaluation read its whole window. */
+int guard_set_sliding(guard_ctx *ctx, int on);
+
 /* Deferred evaluations (off by default).  While on, guard_score enqueues the evaluation on
  * streams of the library's own, ordered after everything enqueued on `stream` so far, and
  * `stream` does NOT wait for it: the evaluation (Section 4.2's peer comparison over the last
@@ -322,6 +332,11 @@ int guard_fallback_reasons(guard_ctx *ctx, uint32_t out[6], void *stream);
  * keeps, 3 the median lay below the interval, 4 above it, 5 the selection did not converge.
  * Results are exact either way. */
 int guard_window_fallbacks(guard_ctx *ctx, uint32_t out[6], void *stream);
+
+/* Diagnostic: synchronises `stream` and returns how many series the sliding evaluations
+ * (guard_set_sliding) rebuilt from their whole window since creation / reset (every series once
+ * when sliding starts, afterwards those whose median left its interval).  Negative on error. */
+int64_t guard_sliding_rebuilds(guard_ctx *ctx, void *stream);
 
 /* Frees the host object (the workspace stays the caller's). NULL is allowed. */
 void guard_destroy(guard_ctx *ctx);

@@ -24,7 +24,7 @@ constexpr int kIngestStreams = GUARD_INGEST_STREAMS;   // internal streams the c
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, lastflag, lasttier, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, xr_big, xr_big_stride, mask, ring, total;
+    size_t status, consec, lastflag, lasttier, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, inc_lo, inc_hi, inc_cnt, inc_val, xr_big, xr_big_stride, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
@@ -49,6 +49,11 @@ Layout make_layout(int R, int M, int C, int K) {
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
     L.wspread = off;   off = align_up(off + (size_t)R * M * sizeof(float));
     L.wcentre = off;   off = align_up(off + (size_t)R * M * sizeof(float));
+    // sliding-window state: interval ends, packed counts, listed values
+    L.inc_lo = off;    off = align_up(off + window_inc_bytes(R * M));
+    L.inc_hi = off;    off = align_up(off + window_inc_bytes(R * M));
+    L.inc_cnt = off;   off = align_up(off + window_inc_bytes(R * M));
+    L.inc_val = off;   off = align_up(off + (size_t)kIncSlots * window_inc_bytes(R * M));
     L.xr_big = off;    off = align_up(off + (L.xr_split ? xrank_split_scratch_bytes(R, M, C < kSplitMaxSteps ? C : kSplitMaxSteps)
                                              : L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps) : 0));
     // in deferred mode consecutive blocks run their cross-rank kernels on streams of their own
@@ -132,6 +137,12 @@ struct guard_ctx {
     long long seen_at_eval = 0;   // steps seen at the last evaluation
     int ranks_per_node = 8;
     long long wait_limit = 0;     // test hook: limit of the warp window path's first wait (0: default)
+    // Sliding-window state (window.cu): current for the window of inc_n steps ending at step count inc_seen
+    // (-1: none).  hints_ready: a whole-window kernel has seeded the per-series search intervals.
+    long long inc_seen = -1;
+    int inc_n = 0;
+    bool sliding = true;          // guard_set_sliding
+    bool hints_ready = false;
     // overlap of the window medians (which need only the ring) with the cross-rank kernels of the
     // ingest that precedes them: an internal stream forked from and joined into the caller's
     bool overlap = true;
@@ -312,12 +323,14 @@ struct guard_ctx {
         return cudaSuccess;
     }
     // The window kernel, with a pair of events around it on its stream while profiling mode 2 is on.
+    const IncArgs *inc_now = nullptr;   // set by guard_score while its window medians take the sliding update
     cudaError_t window(const WindowArgs &w, cudaStream_t ws_) {
-        if (profiling != 2) return launch_window_select(w, ws_);
+        auto go = [&]() { return inc_now ? launch_window_incremental(w, *inc_now, ws_) : launch_window_select(w, ws_); };
+        if (profiling != 2) return go();
         cudaEvent_t e0 = nullptr, e1 = nullptr;
         if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return cudaGetLastError();
         cudaEventRecord(e0, ws_);
-        const cudaError_t e = launch_window_select(w, ws_);
+        const cudaError_t e = go();
         cudaEventRecord(e1, ws_);
         prof.emplace_back(e0, e1);
         return e;
@@ -467,12 +480,37 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     w.series = (int)row;
     w.wmed = c->wmed();
     w.wmed_user = d_wmed;
-    w.use_hint = c->evals > 0 ? 1 : 0;
+    w.use_hint = c->hints_ready ? 1 : 0;
     w.spread = (float *)(c->ws + c->L.wspread);
     w.centre = (float *)(c->ws + c->L.wcentre);
     // windows that share at least three quarters of their steps with the previous evaluation's: the
     // previous median itself is the centre, and a much narrower interval does
     if (c->evals > 0 && (c->seen - c->seen_at_eval) * 4 <= n) { w.target = kWindowNearTarget; w.smooth = kWindowNearSmooth; }
+    // Evaluations that follow one another by a few steps: the sliding update reads only the steps that
+    // entered and left the window since its per-series state was current (or rebuilds that state).
+    IncArgs ia{};
+    const bool close = c->evals > 0 ? (c->seen - c->seen_at_eval) <= kIncMaxNew : c->seen <= kIncMaxNew;
+    const bool use_inc = c->sliding && close && window_inc_supported(w);
+    if (use_inc) {
+        ia.lo = (float *)(c->ws + c->L.inc_lo);
+        ia.hi = (float *)(c->ws + c->L.inc_hi);
+        ia.cnt = (uint32_t *)(c->ws + c->L.inc_cnt);
+        ia.val = (float *)(c->ws + c->L.inc_val);
+        ia.rebuilds = c->status() + 14;
+        const long long p1 = c->inc_seen, p0 = p1 - c->inc_n, q1 = c->seen, q0 = q1 - n;
+        // the windows overlap, few steps entered / left, and the steps that left are still in the ring
+        if (p1 >= 0 && q0 < p1 && q1 - p1 <= kIncMaxNew && q0 - p0 <= kIncMaxNew && q1 - p0 <= c->C) {
+            ia.entering = (int)(q1 - p1);
+            ia.leaving = (int)(q0 - p0);
+        } else {
+            ia.rebuild_all = 1;
+        }
+        c->inc_seen = c->seen;
+        c->inc_n = n;
+    } else {
+        c->hints_ready = true;   // a whole-window kernel runs: it seeds (or re-tunes) the per-series search intervals
+    }
+    c->inc_now = use_inc ? &ia : nullptr;
     c->seen_at_eval = c->seen;
     w.fb_count = c->status() + 8;
     w.status = c->status();
@@ -520,6 +558,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     } else {
         e = c->window(w, st);
     }
+    c->inc_now = nullptr;
     if (e != cudaSuccess) return c->cuda_fail(e, "window_select launch");
 
     XrankArgs x{};
@@ -597,7 +636,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         e = cudaEventRecord(c->ev_e, c->tail);
         if (e != cudaSuccess) return c->cuda_fail(e, "event record");
         c->pending = true;
-        c->pending_n = n;
+        c->pending_n = n + (use_inc ? ia.leaving : 0);   // the sliding update also reads the steps that just left the window
         c->pending_seen = c->seen;
     }
     return GUARD_OK;
@@ -721,12 +760,14 @@ struct StateHeader {
     int32_t R, M, W, k, K, mask_bytes;
     int64_t seen, evals, seen_at_eval;
     int32_t steps;      // ring steps stored: min(seen, W)
-    int32_t pad;
+    int32_t inc_n;      // sliding-window state: window length it is current for
+    int64_t inc_seen;   // ... and the step count (-1: none)
+    int32_t hints_ready, pad;
 };
 constexpr uint32_t kStateMagic = 0x47524453u;   // "GRDS"
 constexpr size_t kStateHeaderBytes = 256;
 
-struct StateLayout { size_t status, fleet, consec, lastflag, lasttier, wmed, wspread, wcentre, mask, ring, total; };
+struct StateLayout { size_t status, fleet, consec, lastflag, lasttier, wmed, wspread, wcentre, inc, mask, ring, total; };
 StateLayout state_layout(const guard_ctx *c) {
     StateLayout s{};
     const size_t RM = (size_t)c->R * c->M * sizeof(float);
@@ -739,6 +780,7 @@ StateLayout state_layout(const guard_ctx *c) {
     s.wmed = off;     off = align_up(off + RM);
     s.wspread = off;  off = align_up(off + RM);
     s.wcentre = off;  off = align_up(off + RM);
+    s.inc = off;      off = align_up(off + (3 + kIncSlots) * window_inc_bytes(c->R * c->M));
     s.mask = off;     off = align_up(off + (size_t)c->W * c->R * c->mask_bytes());
     s.ring = off;     off = align_up(off + (size_t)c->W * RM);
     s.total = off;
@@ -781,6 +823,7 @@ int guard_state_export(guard_ctx *c, void *d_state, size_t state_bytes, void *st
     h.R = c->R; h.M = c->M; h.W = c->W; h.k = c->k; h.K = c->K; h.mask_bytes = c->mask_bytes();
     h.seen = c->seen; h.evals = c->evals; h.seen_at_eval = c->seen_at_eval;
     h.steps = (int)(c->seen < c->W ? c->seen : c->W);
+    h.inc_n = c->inc_n; h.inc_seen = c->inc_seen; h.hints_ready = c->hints_ready ? 1 : 0;
     // pageable host source: the runtime stages it before the call returns
     e = cudaMemcpyAsync(d, &h, sizeof(h), cudaMemcpyHostToDevice, st);
     auto dd = [&](size_t dst_off, const void *src, size_t n) {
@@ -794,6 +837,13 @@ int guard_state_export(guard_ctx *c, void *d_state, size_t state_bytes, void *st
     dd(sl.wmed, c->wmed(), RM);
     dd(sl.wspread, c->ws + c->L.wspread, RM);
     dd(sl.wcentre, c->ws + c->L.wcentre, RM);
+    {   // sliding-window state: four arrays, stored back to back
+        const size_t ib = window_inc_bytes(c->R * c->M);
+        dd(sl.inc, c->ws + c->L.inc_lo, ib);
+        dd(sl.inc + ib, c->ws + c->L.inc_hi, ib);
+        dd(sl.inc + 2 * ib, c->ws + c->L.inc_cnt, ib);
+        dd(sl.inc + 3 * ib, c->ws + c->L.inc_val, kIncSlots * ib);
+    }
     if (e == cudaSuccess) e = copy_rows((char *)c->mask(), d + sl.mask, (size_t)c->R * c->mask_bytes(), c->seen, h.steps, c->C, true, st);
     if (e == cudaSuccess) e = copy_rows((char *)c->ring(), d + sl.ring, RM, c->seen, h.steps, c->C, true, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "guard_state_export");
@@ -816,7 +866,8 @@ int guard_state_import(guard_ctx *c, const void *d_state, size_t state_bytes, vo
     if (h.R != c->R || h.M != c->M || h.W != c->W || h.k != c->k || h.K != c->K || h.mask_bytes != c->mask_bytes())
         return c->fail(GUARD_ERR_ARG, "state was exported from a context of other sizes (ranks %d metrics %d W %d k %d topk %d)",
                        h.R, h.M, h.W, h.k, h.K);
-    if (h.seen < 0 || h.steps != (int)(h.seen < h.W ? h.seen : h.W) || h.evals < 0 || h.seen_at_eval > h.seen)
+    if (h.seen < 0 || h.steps != (int)(h.seen < h.W ? h.seen : h.W) || h.evals < 0 || h.seen_at_eval > h.seen ||
+        h.inc_seen > h.seen || h.inc_n < 0 || h.inc_n > h.W)
         return c->fail(GUARD_ERR_ARG, "state header is inconsistent");
     const char *d = (const char *)d_state;
     const size_t RM = (size_t)c->R * c->M * sizeof(float);
@@ -833,12 +884,22 @@ int guard_state_import(guard_ctx *c, const void *d_state, size_t state_bytes, vo
     dd(c->wmed(), sl.wmed, RM);
     dd(c->ws + c->L.wspread, sl.wspread, RM);
     dd(c->ws + c->L.wcentre, sl.wcentre, RM);
+    {
+        const size_t ib = window_inc_bytes(c->R * c->M);
+        dd(c->ws + c->L.inc_lo, sl.inc, ib);
+        dd(c->ws + c->L.inc_hi, sl.inc + ib, ib);
+        dd(c->ws + c->L.inc_cnt, sl.inc + 2 * ib, ib);
+        dd(c->ws + c->L.inc_val, sl.inc + 3 * ib, kIncSlots * ib);
+    }
     if (e == cudaSuccess) e = copy_rows((char *)c->mask(), const_cast<char *>(d) + sl.mask, (size_t)c->R * c->mask_bytes(), h.seen, h.steps, c->C, false, st);
     if (e == cudaSuccess) e = copy_rows((char *)c->ring(), const_cast<char *>(d) + sl.ring, RM, h.seen, h.steps, c->C, false, st);
     if (e != cudaSuccess) return c->cuda_fail(e, "guard_state_import");
     c->seen = h.seen;
     c->evals = h.evals;
     c->seen_at_eval = h.seen_at_eval;
+    c->inc_seen = h.inc_seen;
+    c->inc_n = h.inc_n;
+    c->hints_ready = h.hints_ready != 0;
     c->fork_fresh = false;
     return GUARD_OK;
 }
@@ -871,6 +932,8 @@ int guard_reset(guard_ctx *c, void *stream) {
     c->seen = 0;
     c->evals = 0;
     c->seen_at_eval = 0;
+    c->inc_seen = -1;
+    c->hints_ready = false;
     return GUARD_OK;
 }
 
@@ -926,6 +989,17 @@ int guard_window_fallbacks(guard_ctx *c, uint32_t out[6], void *stream) {
     return GUARD_OK;
 }
 
+int64_t guard_sliding_rebuilds(guard_ctx *c, void *stream) {
+    if (!c) return GUARD_ERR_ARG;
+    uint32_t n = 0;
+    cudaError_t e = c->join((cudaStream_t)stream);
+    if (e == cudaSuccess) e = c->join_xs((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&n, c->status() + 14, sizeof(n), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_sliding_rebuilds");
+    return (int64_t)n;
+}
+
 int64_t guard_fallback_steps(guard_ctx *c, void *stream) {
     if (!c) return GUARD_ERR_ARG;
     uint32_t n = 0;
@@ -935,6 +1009,12 @@ int64_t guard_fallback_steps(guard_ctx *c, void *stream) {
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return c->cuda_fail(e, "guard_fallback_steps");
     return (int64_t)n;
+}
+
+int guard_set_sliding(guard_ctx *c, int on) {
+    if (!c) return GUARD_ERR_ARG;
+    c->sliding = on != 0;
+    return GUARD_OK;
 }
 
 int guard_set_deferred(guard_ctx *c, int on) {

@@ -93,6 +93,27 @@ struct WindowArgs {
 };
 // Launches one kernel (thread, warp or staged path).
 cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st);
+
+// Sliding windows: per-series state that lets an evaluation which follows the previous one by a few
+// steps read only the steps that entered and left the window.  A series keeps an interval [lo, hi]
+// around its median, the number of window values below lo and the values inside the interval; the
+// median is then a rank among those.  A series whose median leaves the interval (or whose interval
+// overflows) rebuilds its state from the whole window.
+constexpr int kIncSlots = 24;     // values a series' interval can hold
+constexpr int kIncHalf = 6;       // ranks the interval reaches beyond the middle ranks when it is (re)built
+constexpr int kIncMaxNew = 8;     // most steps between two evaluations the sliding update is used for
+struct IncArgs {
+    float *lo, *hi;               // [series] interval ends (inclusive)
+    uint32_t *cnt;                // [series] bit 31: state valid; bits 16..23: values inside; bits 0..15: values below lo
+    float *val;                   // [kIncSlots][series] the values inside the interval, in no particular order
+    int rebuild_all;              // ignore the stored state: every series rebuilds
+    int entering;                 // steps that entered the window since the state was current (the newest ones)
+    int leaving;                  // steps that left it (those right before the window's oldest step)
+    uint32_t *rebuilds;           // diagnostic counter or NULL
+};
+size_t window_inc_bytes(int series);   // per array: lo, hi, cnt take series * 4 bytes, val kIncSlots * series * 4
+bool window_inc_supported(const WindowArgs &a);
+cudaError_t launch_window_incremental(const WindowArgs &a, const IncArgs &inc, cudaStream_t st);
 int window_launch_count(const WindowArgs &a);
 
 // Fused k-of-W count, robust score, thresholds, multi-signal flag, tier, consecutive counter.

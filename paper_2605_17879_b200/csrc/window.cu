@@ -8,6 +8,7 @@
 
 #include "colselect.cuh"
 #include "kernels.h"
+#include "xrank_common.cuh"
 
 namespace guard {
 
@@ -615,6 +616,160 @@ cudaError_t launch_thread_path(const WindowArgs &a, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------
+// Sliding-window path: evaluations that follow one another by a few steps (streaming: one step)
+// share all but a few steps of their windows, so a series' median moves by a rank or two.  Each
+// series keeps, across evaluations, an interval [lo, hi] around its median, the number of window
+// values below lo, and the handful of values inside the interval (global memory, one array per
+// slot so that a warp's accesses are contiguous).  An evaluation reads only the steps that
+// entered and left the window: a value below lo moves the count, a value inside the interval is
+// appended to / removed from the series' list; the median is then the rank (middle - count) among
+// the listed values, found by counting (the list holds a dozen values).  One thread per series.
+// A series whose median has left its interval, whose list is full, or that has no state yet is
+// rebuilt by its whole warp: the lanes fetch the window, sort it (bitonic network over registers
+// and shuffles) and take the median, the interval ends kIncHalf ranks beyond the middle ranks, and
+// the values inside.  Exact either way: the interval only decides which values are listed.
+// ---------------------------------------------------------------------------------------
+constexpr int kIncThreads = 128;
+
+template <int VPL>
+__global__ void __launch_bounds__(kIncThreads) window_inc_kernel(const WindowArgs a, const IncArgs s) {
+    __shared__ float sv[kIncSlots][kIncThreads];   // this thread's listed values: column tid
+    const int tid = threadIdx.x, lane = lane_id();
+    const int n = a.n;
+    const int c = blockIdx.x * kIncThreads + tid;
+    const bool active = c < a.series;
+    const int cc = active ? c : a.series - 1;
+    const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;   // slot of the window's oldest step
+    const bool even = !(n & 1);
+    const int k1 = (n - 1) >> 1, k2 = n >> 1;
+
+    const uint32_t w = s.cnt[cc];
+    bool ok = active && (w >> 31) && !s.rebuild_all;
+    int cb = (int)(w & 0xFFFFu), nin = (int)((w >> 16) & 0xFFu);
+    const float lo = s.lo[cc], hi = s.hi[cc];
+    bool dirty = false;
+    if (ok) {
+        for (int j = 0; j < nin; ++j) sv[j][tid] = s.val[(size_t)j * a.series + c];
+        // steps that left the window: the ones right before its oldest step
+        for (int i = 0; i < s.leaving; ++i) {
+            int slot = first - s.leaving + i;
+            if (slot < 0) slot += a.capacity;
+            const float x = __ldg(a.ring + (size_t)slot * a.row_stride + c);
+            if (x < lo) {
+                --cb;
+            } else if (x <= hi) {
+                int at = -1;
+                for (int j = 0; j < nin; ++j)
+                    if (__float_as_uint(sv[j][tid]) == __float_as_uint(x)) at = j;
+                if (at < 0) { ok = false; break; }      // the books do not balance: rebuild
+                sv[at][tid] = sv[nin - 1][tid];
+                --nin;
+                dirty = true;
+            }
+        }
+        // steps that entered it: the newest ones
+        for (int i = 0; ok && i < s.entering; ++i) {
+            int slot = a.last_slot - (s.entering - 1 - i);
+            if (slot < 0) slot += a.capacity;
+            const float x = __ldg(a.ring + (size_t)slot * a.row_stride + c);
+            if (x < lo) {
+                ++cb;
+            } else if (x <= hi) {
+                if (nin >= kIncSlots) { ok = false; break; }
+                sv[nin][tid] = x;
+                ++nin;
+                dirty = true;
+            }
+        }
+        ok = ok && cb >= 0 && cb <= k1 && k2 < cb + nin;
+    }
+    if (ok) {
+        // ranks j1, j2 among the listed values (total order: keys; equal keys by position)
+        const int j1 = k1 - cb, j2 = k2 - cb;
+        uint32_t v1 = 0, v2 = 0;
+        for (int i = 0; i < nin; ++i) {
+            const uint32_t ki = f2key(sv[i][tid]);
+            int rank = 0;
+            for (int j = 0; j < nin; ++j) {
+                const uint32_t kj = f2key(sv[j][tid]);
+                rank += (kj < ki) || (kj == ki && j < i);
+            }
+            if (rank == j1) v1 = ki;
+            if (rank == j2) v2 = ki;
+        }
+        const float med = median_from_keys(v1, v2, even);
+        a.wmed[c] = med;
+        if (a.wmed_user) a.wmed_user[c] = med;
+        s.cnt[c] = 0x80000000u | ((uint32_t)nin << 16) | (uint32_t)cb;
+        if (dirty)
+            for (int j = 0; j < nin; ++j) s.val[(size_t)j * a.series + c] = sv[j][tid];
+    }
+    // ---- series without a usable state: the whole warp rebuilds them one by one ------------------
+    unsigned todo = __ballot_sync(0xFFFFFFFFu, active && !ok);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int series = __shfl_sync(0xFFFFFFFFu, c, src);
+        uint32_t kv[VPL];
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int row = lane + 32 * j;
+            kv[j] = 0xFFFFFFFFu;                 // padding sorts behind every finite value
+            if (row < n) {
+                int slot = first + row;
+                if (slot >= a.capacity) slot -= a.capacity;
+                kv[j] = f2key(__ldg(a.ring + (size_t)slot * a.row_stride + series));
+            }
+        }
+        warp_bitonic_sort<VPL>(kv, lane);        // ascending: element e in lane e / VPL, register e % VPL
+        auto pick = [&](int r) -> uint32_t {
+            uint32_t mine = kv[0];
+#pragma unroll
+            for (int j = 1; j < VPL; ++j) mine = ((r % VPL) == j) ? kv[j] : mine;
+            return __shfl_sync(0xFFFFFFFFu, mine, r / VPL);
+        };
+        const float med = median_from_keys(pick(k1), pick(k2), even);
+        const float flo = key2f(pick(max(0, k1 - kIncHalf))), fhi = key2f(pick(min(n - 1, k2 + kIncHalf)));
+        // values below / inside the interval, by the same float comparisons the sliding update uses
+        int below = 0, in = 0;
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const bool real = lane * VPL + j < n;
+            const float x = key2f(kv[j]);
+            below += real && (x < flo);
+            in += real && !(x < flo) && (x <= fhi);
+        }
+        int incl = in;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int u = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= d) incl += u;
+        }
+        const int nin2 = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        const int cb2 = (int)__reduce_add_sync(0xFFFFFFFFu, (uint32_t)below);
+        const bool fits = nin2 <= kIncSlots;
+        if (fits) {
+            int pos = incl - in;
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) {
+                const bool real = lane * VPL + j < n;
+                const float x = key2f(kv[j]);
+                if (real && !(x < flo) && (x <= fhi)) { s.val[(size_t)pos * a.series + series] = x; ++pos; }
+            }
+        }
+        if (lane == 0) {
+            a.wmed[series] = med;
+            if (a.wmed_user) a.wmed_user[series] = med;
+            s.lo[series] = flo;
+            s.hi[series] = fhi;
+            // an interval with more (tied) values than a list holds stays without state: it rebuilds every time
+            s.cnt[series] = fits ? (0x80000000u | ((uint32_t)nin2 << 16) | (uint32_t)cb2) : 0u;
+            if (s.rebuilds) atomicAdd(s.rebuilds, 1u);
+        }
+    }
+}
+
 // Fallback for windows too long to stage: one thread per series, bit-by-bit counting
 // selection straight from global memory (32 sweeps of the column).
 __global__ void window_select_global_kernel(const WindowArgs a) {
@@ -674,6 +829,18 @@ cudaError_t launch_staged(const WindowArgs &a, int use_bulk, cudaStream_t st) {
 }  // namespace
 
 int window_launch_count(const WindowArgs &) { return 1; }
+
+size_t window_inc_bytes(int series) { return (size_t)series * sizeof(float); }
+
+bool window_inc_supported(const WindowArgs &a) { return a.n >= 1 && a.n <= 256; }
+
+cudaError_t launch_window_incremental(const WindowArgs &a, const IncArgs &inc, cudaStream_t st) {
+    const int grid = (a.series + kIncThreads - 1) / kIncThreads;
+    if (a.n <= 64) window_inc_kernel<2><<<grid, kIncThreads, 0, st>>>(a, inc);
+    else if (a.n <= 128) window_inc_kernel<4><<<grid, kIncThreads, 0, st>>>(a, inc);
+    else window_inc_kernel<8><<<grid, kIncThreads, 0, st>>>(a, inc);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st) {
     constexpr size_t kMaxTile = kMaxStagedTile;

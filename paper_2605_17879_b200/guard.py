@@ -97,6 +97,10 @@ def lib():
         L.guard_window_fallbacks.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.guard_set_overlap.restype = C.c_int
         L.guard_set_overlap.argtypes = [vp, C.c_int]
+        L.guard_set_sliding.restype = C.c_int
+        L.guard_set_sliding.argtypes = [vp, C.c_int]
+        L.guard_sliding_rebuilds.restype = C.c_int64
+        L.guard_sliding_rebuilds.argtypes = [vp, vp]
         L.guard_set_deferred.restype = C.c_int
         L.guard_set_deferred.argtypes = [vp, C.c_int]
         L.guard_join.restype = C.c_int
@@ -231,6 +235,18 @@ class Guard:
     def set_overlap(self, on: bool) -> None:
         """Window medians of an evaluation on an internal stream overlapping the preceding ingest."""
         self._check(lib().guard_set_overlap(self._h, 1 if on else 0))
+
+    def set_sliding(self, on: bool) -> None:
+        """Sliding update of the window medians for evaluations a few steps apart (default on)."""
+        self._check(lib().guard_set_sliding(self._h, 1 if on else 0))
+
+    def sliding_rebuilds(self) -> int:
+        """Series the sliding evaluations rebuilt from their whole window (synchronises)."""
+        with torch.cuda.device(self.device):
+            n = int(lib().guard_sliding_rebuilds(self._h, _stream()))
+        if n < 0:
+            self._check(n)
+        return n
 
     def set_deferred(self, on: bool) -> None:
         """Deferred evaluations: score() does not make the current stream wait for its results; they

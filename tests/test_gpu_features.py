@@ -133,7 +133,7 @@ def test_state_export_import_resumes_bit_identically(R, M, W, B, cap, cap2, defe
         a.sync_status()
         compare_score(out, refs[i], "uninterrupted t=%d" % t)
         outs_a.append({k: to_np(v).copy() for k, v in out.items()})
-    fa, wa = a.fallback_steps(), a.window_fallbacks()
+    fa, wa, ra = a.fallback_steps(), a.window_fallbacks(), a.sliding_rebuilds()
     a.close()
     b = guard.Guard(R, M, W, max(1, W // 2), capacity=cap2, **kw)
     b.set_deferred(deferred)
@@ -149,7 +149,7 @@ def test_state_export_import_resumes_bit_identically(R, M, W, B, cap, cap2, defe
         for key, v in out.items():                       # and bit-identical to the run that never stopped
             assert np.array_equal(to_np(v).view(np.uint8), outs_a[i][key].view(np.uint8)), (key, t)
     # the resumed context took the same paths: its fallback counters continue the exported ones
-    assert b.fallback_steps() == fa and b.window_fallbacks() == wa
+    assert b.fallback_steps() == fa and b.window_fallbacks() == wa and b.sliding_rebuilds() == ra
     # rejects: another geometry, a buffer that is too small, garbage
     c = guard.Guard(R, M, W + 1, 1, capacity=cap2 + 1, dir=dirs)
     with pytest.raises(guard.GuardError) as ei:

@@ -2,9 +2,10 @@
 CPU oracle (slow: an oracle evaluation sorts every series of the fleet).
 
 * Streaming: 32 768 ranks x 8 metrics, one step per ingest into a 512-step ring that wraps, an
-  evaluation after EVERY step (consecutive windows share all but one step, which is what puts the
-  window kernel into its narrow-interval mode), default and deferred mode; a run of consecutive
-  evaluations after the wrap is compared in full, node-level fold included.
+  evaluation after EVERY step (consecutive windows share all but one step: the sliding update of the
+  window medians, and with that switched off the window kernel's narrow-interval mode), default
+  and deferred mode; a run of consecutive evaluations after the wrap is compared in full,
+  node-level fold included.
 * Large fleet: ten consecutive 200-step blocks around the onset of a fail-slow ramp, in the
   deferred in-place pipeline, every evaluation compared in full."""
 import numpy as np
@@ -49,9 +50,12 @@ def test_streaming_every_step_full_width_after_ring_wrap():
     stalled_now = [int(nrefs[i]["node_stall"].sum()) - int(nrefs[i - 1]["node_stall"].sum()) for i in range(1, ncmp)]
     assert any(d > 0 for d in stalled_now)         # a stall entered the window inside the compared run
 
-    for deferred in (False, True):
+    # sliding evaluations (the default: per-series state updated from the step that entered and the one that
+    # left) in default and deferred mode, and whole-window evaluations (the narrow-interval thread kernel)
+    for deferred, sliding in ((False, True), (True, True), (True, False)):
         g = guard.Guard(R, M, W, cfg.k, dir=dirs, capacity=cfg.ring_capacity, topk=cfg.topk)
         g.set_deferred(deferred)
+        g.set_sliding(sliding)
         out = g.alloc_outputs()
         nout = None
         bufs = [(g.alloc_outputs(), None) for _ in range(ncmp)]
@@ -71,12 +75,17 @@ def test_streaming_every_step_full_width_after_ring_wrap():
         g.join()
         assert g.sync_status() == 0
         assert g.steps_seen == T
-        wf = g.window_fallbacks()
-        # the narrow interval misses now and then (its whole-warp fallback is exact), but only for a small
-        # part of the 262 144 series x 547 thread-path evaluations
-        assert 0 < wf["total"] < 0.05 * R * M * T, wf
+        wf, rb = g.window_fallbacks(), g.sliding_rebuilds()
+        if sliding:
+            # every series builds its state at the first evaluation; afterwards a series rebuilds only when its
+            # median has left its interval: a small part of the 262 144 series x 547 later evaluations
+            assert wf["total"] == 0 and R * M < rb < R * M + 0.05 * R * M * T, (wf, rb)
+        else:
+            # the narrow interval misses now and then (its whole-warp fallback is exact), but only for a small
+            # part of the 262 144 series x 547 thread-path evaluations
+            assert rb == 0 and 0 < wf["total"] < 0.05 * R * M * T, (wf, rb)
         for i in range(ncmp):
-            what = "deferred=%s t=%d" % (deferred, first_cmp + i)
+            what = "deferred=%s sliding=%s t=%d" % (deferred, sliding, first_cmp + i)
             assert_bit_equal(to_np(smed[i]), irefs[i]["step_med"][0], what + " step_med")
             assert_bit_equal(to_np(smad[i]), irefs[i]["step_mad"][0], what + " step_mad")
             compare_score(bufs[i][0], refs[i], what)

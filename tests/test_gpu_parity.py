@@ -306,6 +306,44 @@ def test_long_window_paths():
         run_both(X, W, W // 2, 2, dirs, [W, 7], capacity=W + 16, score_every=1)
 
 
+@pytest.mark.parametrize("R,M,W,cap,gaps,quant", [
+    (300, 4, 50, 64, [1], None),                # an evaluation every step: one step enters, one leaves
+    (300, 4, 50, 60, [1, 3, 8, 2], None),       # several steps between evaluations, up to the sliding limit
+    (64, 8, 200, 256, [1], None),               # window of the streaming configuration (8 keys per lane when rebuilding)
+    (40, 3, 7, 9, [1, 2], None),                # tiny odd window, ring barely longer than it
+    (96, 4, 33, 40, [1, 9, 1, 1, 20, 1], None), # gaps beyond the limit fall back to whole-window kernels in between
+    (128, 4, 40, 64, [1], 25),                  # quantised: ties at the interval ends, lists that overflow
+    (50, 2, 30, 32, [1], 3),                    # very coarse: most series cannot hold their ties and rebuild every time
+])
+def test_sliding_evaluations_match_oracle(R, M, W, cap, gaps, quant):
+    from paper_2605_17879_b200 import guard
+    T = 3 * W + 20
+    X, dirs = _rand_fleet(T, R, M, seed=R + W, quant=quant)
+    X[W + 3:W + 9, 5] *= 1.5                     # a level shift: medians leave their intervals
+    Xd = torch.from_numpy(X).cuda()
+    k = max(1, W // 2)
+    for sliding in (True, False):
+        g = guard.Guard(R, M, W, k, dir=dirs, capacity=cap, topk=min(8, R), min_signals=min(2, M))
+        g.set_sliding(sliding)
+        o = go.Oracle(R, M, W, k, min(8, R), dir=dirs, min_signals=min(2, M))
+        t, i = 0, 0
+        while t < T:
+            b = min(gaps[i % len(gaps)], T - t)
+            g.ingest(Xd[t:t + b])
+            o.ingest(X[t:t + b])
+            t += b
+            i += 1
+            out = g.score()
+            assert g.sync_status() == 0
+            compare_score(out, o.score(), "sliding=%s t=%d" % (sliding, t))
+        rb = g.sliding_rebuilds()
+        if sliding and quant is None and max(gaps) <= 8:
+            assert R * M <= rb < 0.5 * R * M * i, rb      # state built once, then mostly slid
+        if not sliding:
+            assert rb == 0
+        g.close()
+
+
 def test_consecutive_evaluations_state():
     X, dirs = _rand_fleet(80, 32, 4, seed=9)
     run_both(X, 10, 6, 4, dirs, [10], n_consec=3)
