@@ -193,7 +193,8 @@ def run_streaming(dev, steps, warm):
     res = {"workload": "streaming: 32768 ranks x 8 metrics, ring 512, W=200 k=120 top-64, evaluation every step",
            "steps": steps, "latency_us": {"p50": pick(0.50), "p99": pick(0.99), "max": lat[-1] * 1e6},
            "sustained_cells_per_s": sustained, "us_per_step_sustained": e0.elapsed_time(e1) * 1e3 / steps,
-           "cells_per_step": R * M, "fallback_rows": g.fallback_steps()}
+           "cells_per_step": R * M, "fallback_rows": g.fallback_steps(),
+           "sliding_rebuilds_per_step": g.sliding_rebuilds() / float(warm + 2 * steps)}
     g.close()
     return res
 

@@ -99,13 +99,13 @@ cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st);
 // around its median, the number of window values below lo and the values inside the interval; the
 // median is then a rank among those.  A series whose median leaves the interval (or whose interval
 // overflows) rebuilds its state from the whole window.
-constexpr int kIncSlots = 24;     // values a series' interval can hold
-constexpr int kIncHalf = 6;       // ranks the interval reaches beyond the middle ranks when it is (re)built
+constexpr int kIncSlots = 40;     // values a series' interval can hold
+constexpr int kIncHalf = 12;      // ranks the interval reaches beyond the middle ranks when it is (re)built
 constexpr int kIncMaxNew = 8;     // most steps between two evaluations the sliding update is used for
 struct IncArgs {
     float *lo, *hi;               // [series] interval ends (inclusive)
     uint32_t *cnt;                // [series] bit 31: state valid; bits 16..23: values inside; bits 0..15: values below lo
-    float *val;                   // [kIncSlots][series] the values inside the interval, in no particular order
+    float *val;                   // [kIncSlots][series] the values inside the interval, ascending (total order)
     int rebuild_all;              // ignore the stored state: every series rebuilds
     int entering;                 // steps that entered the window since the state was current (the newest ones)
     int leaving;                  // steps that left it (those right before the window's oldest step)

@@ -623,8 +623,8 @@ cudaError_t launch_thread_path(const WindowArgs &a, cudaStream_t st) {
 // values below lo, and the handful of values inside the interval (global memory, one array per
 // slot so that a warp's accesses are contiguous).  An evaluation reads only the steps that
 // entered and left the window: a value below lo moves the count, a value inside the interval is
-// appended to / removed from the series' list; the median is then the rank (middle - count) among
-// the listed values, found by counting (the list holds a dozen values).  One thread per series.
+// inserted into / removed from the series' sorted list (fetched only in that case); the median is
+// then position (middle - count) of the list.  One thread per series.
 // A series whose median has left its interval, whose list is full, or that has no state yet is
 // rebuilt by its whole warp: the lanes fetch the window, sort it (bitonic network over registers
 // and shuffles) and take the median, the interval ends kIncHalf ranks beyond the middle ranks, and
@@ -648,27 +648,33 @@ __global__ void __launch_bounds__(kIncThreads) window_inc_kernel(const WindowArg
     bool ok = active && (w >> 31) && !s.rebuild_all;
     int cb = (int)(w & 0xFFFFu), nin = (int)((w >> 16) & 0xFFu);
     const float lo = s.lo[cc], hi = s.hi[cc];
-    bool dirty = false;
     if (ok) {
-        for (int j = 0; j < nin; ++j) sv[j][tid] = s.val[(size_t)j * a.series + c];
-        // steps that left the window: the ones right before its oldest step
-        for (int i = 0; i < s.leaving; ++i) {
+        // The steps that left the window (the ones right before its oldest step) and the steps that entered it
+        // (the newest ones).  A value below lo moves the count; a value inside the interval changes the list,
+        // which is kept sorted and fetched only then (seldom: the interval holds a few percent of the window).
+        bool listed = false, dirty = false;
+        auto fetch_list = [&]() {
+            if (!listed)
+                for (int j = 0; j < nin; ++j) sv[j][tid] = s.val[(size_t)j * a.series + c];
+            listed = true;
+        };
+        for (int i = 0; ok && i < s.leaving; ++i) {
             int slot = first - s.leaving + i;
             if (slot < 0) slot += a.capacity;
             const float x = __ldg(a.ring + (size_t)slot * a.row_stride + c);
             if (x < lo) {
                 --cb;
             } else if (x <= hi) {
+                fetch_list();
                 int at = -1;
                 for (int j = 0; j < nin; ++j)
                     if (__float_as_uint(sv[j][tid]) == __float_as_uint(x)) at = j;
                 if (at < 0) { ok = false; break; }      // the books do not balance: rebuild
-                sv[at][tid] = sv[nin - 1][tid];
+                for (int j = at; j + 1 < nin; ++j) sv[j][tid] = sv[j + 1][tid];
                 --nin;
                 dirty = true;
             }
         }
-        // steps that entered it: the newest ones
         for (int i = 0; ok && i < s.entering; ++i) {
             int slot = a.last_slot - (s.entering - 1 - i);
             if (slot < 0) slot += a.capacity;
@@ -677,33 +683,28 @@ __global__ void __launch_bounds__(kIncThreads) window_inc_kernel(const WindowArg
                 ++cb;
             } else if (x <= hi) {
                 if (nin >= kIncSlots) { ok = false; break; }
-                sv[nin][tid] = x;
+                fetch_list();
+                const uint32_t kx = f2key(x);
+                int at = nin;                            // behind the listed values whose key is not above x's
+                while (at > 0 && f2key(sv[at - 1][tid]) > kx) { sv[at][tid] = sv[at - 1][tid]; --at; }
+                sv[at][tid] = x;
                 ++nin;
                 dirty = true;
             }
         }
         ok = ok && cb >= 0 && cb <= k1 && k2 < cb + nin;
-    }
-    if (ok) {
-        // ranks j1, j2 among the listed values (total order: keys; equal keys by position)
-        const int j1 = k1 - cb, j2 = k2 - cb;
-        uint32_t v1 = 0, v2 = 0;
-        for (int i = 0; i < nin; ++i) {
-            const uint32_t ki = f2key(sv[i][tid]);
-            int rank = 0;
-            for (int j = 0; j < nin; ++j) {
-                const uint32_t kj = f2key(sv[j][tid]);
-                rank += (kj < ki) || (kj == ki && j < i);
-            }
-            if (rank == j1) v1 = ki;
-            if (rank == j2) v2 = ki;
+        if (ok) {
+            // the list is sorted: the middle ranks of the window are positions k1 - cb and k2 - cb of it
+            const int j1 = k1 - cb, j2 = k2 - cb;
+            const float f1 = listed ? sv[j1][tid] : s.val[(size_t)j1 * a.series + c];
+            const float f2 = listed ? sv[j2][tid] : s.val[(size_t)j2 * a.series + c];
+            const float med = median_from_keys(f2key(f1), f2key(f2), even);
+            a.wmed[c] = med;
+            if (a.wmed_user) a.wmed_user[c] = med;
+            s.cnt[c] = 0x80000000u | ((uint32_t)nin << 16) | (uint32_t)cb;
+            if (dirty)
+                for (int j = 0; j < nin; ++j) s.val[(size_t)j * a.series + c] = sv[j][tid];
         }
-        const float med = median_from_keys(v1, v2, even);
-        a.wmed[c] = med;
-        if (a.wmed_user) a.wmed_user[c] = med;
-        s.cnt[c] = 0x80000000u | ((uint32_t)nin << 16) | (uint32_t)cb;
-        if (dirty)
-            for (int j = 0; j < nin; ++j) s.val[(size_t)j * a.series + c] = sv[j][tid];
     }
     // ---- series without a usable state: the whole warp rebuilds them one by one ------------------
     unsigned todo = __ballot_sync(0xFFFFFFFFu, active && !ok);
