@@ -139,6 +139,117 @@ def oracle_sample_rate(cfg, block_host, sample_steps):
     return x.size / dt, dt
 
 
+def _oracle_block_worker(job):
+    """One 200-step block of the workload through the oracle (as it stands, one thread): generated on the
+    CPU by the same seeded generator, then ingest + one evaluation are timed.  Runs in a spawned process."""
+    t0_step, = job
+    import torch
+    torch.set_num_threads(1)
+    from oracle import guard_oracle as go
+    from paper_2605_17879_b200 import synth
+    cfg = synth.paper_configs()["large"]
+    blk = synth.fleet_block(cfg, t0_step, t0_step + cfg.block, device="cpu").numpy()
+    o = go.Oracle(cfg.ranks, cfg.metrics, cfg.W, cfg.k, cfg.topk, dir=synth.fleet_dir(cfg.metrics))
+    t0 = time.perf_counter()
+    o.ingest(blk)
+    o.score()
+    return blk.size, time.perf_counter() - t0
+
+
+def oracle_all_cores(cfg):
+    """The oracle on all host cores: the workload's outermost independent loop (its 200-step blocks: windows are
+    tumbling, so blocks do not depend on one another) split over one spawned process per core, one block
+    each.  The oracle's source is untouched.  Returns the cpu_baseline sub-object."""
+    import multiprocessing as mp
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    workers = max(1, min(cores, cfg.steps // cfg.block, 32))
+    model = "unknown"
+    try:
+        for ln in open("/proc/cpuinfo"):
+            if ln.startswith("model name"):
+                model = ln.split(":", 1)[1].strip()
+                break
+    except Exception:
+        pass
+    ctx = mp.get_context("spawn")
+    wall0 = time.perf_counter()
+    with ctx.Pool(workers) as pool:
+        res = pool.map(_oracle_block_worker, [(j * cfg.block,) for j in range(workers)])
+    wall = time.perf_counter() - wall0
+    cells = sum(r[0] for r in res)
+    slowest = max(r[1] for r in res)
+    return {"value": cells / slowest, "unit": UNIT, "cores": workers, "host_cores": cores, "cpu_model": model, "kind": "oracle",
+            "seconds": slowest, "wall_seconds_with_generation": wall,
+            "sample": "%d blocks of 200 steps at full width, one per spawned process, each ingest + one evaluation; "
+                      "rate = cells of all blocks / slowest process" % workers}
+
+
+def run_sweep(dev, reps=10):
+    """Offline node-sweep qualification (2 048 nodes x 8 GPUs x 200 repetitions x 6 metrics, 78.6 MB), timed with
+    CUDA events; algorithmic traffic is one 4-byte read per cell."""
+    import torch
+    from paper_2605_17879_b200 import guard, synth
+    cfg = synth.SweepConfig()
+    S = synth.sweep_tensor(cfg, device=dev)
+    kw = dict(dir=synth.sweep_dir(cfg.metrics), thr=3.5, floor_rel=1e-4, floor_abs=synth.sweep_floor_abs(cfg.metrics),
+              pct_ppm=cfg.pct_ppm)
+    out = guard.sweep_qualify(S, cfg.nodes, cfg.gpus_per_node, **kw)
+    ws = torch.empty(int(guard.lib().guard_sweep_workspace_bytes(cfg.gpus, cfg.reps, cfg.metrics)), dtype=torch.uint8, device=dev)
+    flush = torch.empty(L2_BYTES * 2, dtype=torch.uint8, device=dev)
+    times = []
+    for _ in range(3 + reps):
+        flush.zero_()                                # the 78.6 MB input would otherwise sit in L2 between repetitions
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        guard.sweep_qualify(S, cfg.nodes, cfg.gpus_per_node, workspace=ws, out=out, **kw)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / 1e3)
+    t = statistics.median(times[3:])
+    peak, _ = measured_hbm_peak()
+    cells = S.numel()
+    return {"workload": "node sweep: %d nodes x %d GPUs x %d repetitions x %d metrics (%.1f MB), L2 flushed between repetitions"
+                        % (cfg.nodes, cfg.gpus_per_node, cfg.reps, cfg.metrics, cells * 4 / 1e6),
+            "ms": t * 1e3, "cells_per_s": cells / t, "algorithmic_GBps": cells * 4 / t / 1e9,
+            "frac_of_peak": cells * 4 / t / 1e9 / peak, "gpus_failed": int((out["gpu_pass"] == 0).sum().item()),
+            "status": int(out["status"].item())}
+
+
+def run_small_config(dev, name, passes=5):
+    """Whole-path throughput of one of the smaller fleet configurations (resident telemetry, deferred mode)."""
+    import torch
+    from paper_2605_17879_b200 import guard, synth
+    cfg = synth.paper_configs()[name]
+    R, M, T, B = cfg.ranks, cfg.metrics, cfg.steps, cfg.block
+    g = guard.Guard(R, M, cfg.W, cfg.k, dir=synth.fleet_dir(M), capacity=T, topk=cfg.topk, device=dev)
+    ring = g.ring_reserve(T)
+    ring.copy_(synth.fleet_tensor(cfg, device=dev))
+    out = g.alloc_outputs()
+    g.set_deferred(True)
+
+    def one_pass():
+        g.reset()
+        for j in range(T // B):
+            g.ingest(ring[j * B:(j + 1) * B])
+            g.score(out)
+        g.join()
+
+    for _ in range(2):
+        one_pass()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(passes):
+        one_pass()
+    e1.record()
+    torch.cuda.synchronize()
+    g.sync_status()
+    secs = e0.elapsed_time(e1) / 1e3 / passes
+    g.close()
+    return {"workload": "%s fleet: %d ranks x %d steps x %d metrics, W=%d, blocks of %d (launch-bound at this size)"
+                        % (name, R, T, M, cfg.W, B), "ms_per_pass": secs * 1e3, "cells_per_s": R * M * T / secs}
+
+
 def run_streaming(dev, steps, warm):
     """Streaming configuration: 32 768 ranks x 8 metrics, one step per ingest into a 512-step
     ring, an evaluation after every step, flags and top-k read back to pinned host memory.
@@ -242,6 +353,7 @@ def main():
     ap.add_argument("--impl", default="guard", choices=["guard", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-all-cores", action="store_true", help="skip the all-core leg of the CPU baseline")
     ap.add_argument("--streaming-steps", type=int, default=500)
     ap.add_argument("--blocks", type=int, default=0,
                     help="profile-sized run: only this many 200-step blocks of the workload (0 = all 100); not a bench value")
@@ -397,13 +509,18 @@ def main():
         cpu_baseline = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
                         "sample": "ingest + one evaluation of the first %d steps at full width (%d ranks x %d metrics)"
                                   % (sample_steps, R, M)}
+        if not args.no_all_cores:
+            cpu_baseline["all_cores"] = oracle_all_cores(cfg)
 
     streaming = None
+    other = None
     if rank == 0 and world == 1 and args.streaming_steps > 0:
         del ring, out
         g.close()
         torch.cuda.empty_cache()
-        streaming = run_streaming(dev, args.streaming_steps, 50)
+        # 250 warm-up steps: the 200-step window is full and the sliding state settled before anything is timed
+        streaming = run_streaming(dev, args.streaming_steps, 250)
+        other = {"sweep": run_sweep(dev), "tiny": run_small_config(dev, "tiny"), "medium": run_small_config(dev, "medium")}
 
     if rank == 0:
         line = {
@@ -419,7 +536,7 @@ def main():
                        "l2": "inputs (10.49 GB) larger than L2", "parallelism": "replicas only",
                        "flagged_last_evaluation": flagged, "direct_path_fallback_rows_last_pass": fallback_rows},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
-            "streaming": streaming,
+            "streaming": streaming, "other_configs": other,
         }
         print(json.dumps(line), flush=True)
     g.close()

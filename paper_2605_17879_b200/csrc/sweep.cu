@@ -2,6 +2,7 @@
 // pass / fail verdicts against the fleet distribution (GPU level, then node level).
 #include "colselect.cuh"
 #include "kernels.h"
+#include "warpselect.cuh"
 
 namespace guard {
 
@@ -35,6 +36,69 @@ __global__ void __launch_bounds__(kSweepCols) sweep_median_kernel(const SweepMed
     const size_t o = (size_t)g0 * M + tid;
     a.gmed[o] = med;
     if (a.gmed_user) a.gmed_user[o] = med;
+}
+
+// Warp-per-GPU path (up to 256 repetitions): the benchmark results of one GPU are one contiguous
+// [reps][M] block, so a warp fetches its GPU's block with whole-line 128-bit loads into its slice
+// of shared memory; then, metric by metric, the lanes pick the metric's column out of the block
+// (VPL keys per lane), sort their own keys and run the warp selection.  Eight warps per CTA, a
+// few kilobytes of shared memory per warp: every SM holds dozens of GPUs at once.
+constexpr int kSweepWarps = 8;
+
+template <int VPL>
+__global__ void __launch_bounds__(kSweepWarps * 32) sweep_median_warp_kernel(const SweepMedArgs a) {
+    extern __shared__ __align__(16) float sbuf[];      // [kSweepWarps][per], per rounded up to a multiple of 4
+    const int lane = lane_id(), w = warp_id(), M = a.M, reps = a.reps;
+    const int per = reps * M, per4 = (per + 3) & ~3;
+    const int g = blockIdx.x * kSweepWarps + w;
+    if (g >= a.G) return;                               // warps are independent: no CTA barrier below
+    float *buf = sbuf + (size_t)w * per4;
+    const float *src = a.S + (size_t)g * per;
+    bool bad = false;
+    if ((per & 3) == 0 && ((uintptr_t)a.S & 15) == 0) {
+        for (int i = 4 * lane; i < per; i += 128) {
+            const float4 v = __ldg(reinterpret_cast<const float4 *>(src + i));
+            bad |= nonfinite_bits(__float_as_uint(v.x)) | nonfinite_bits(__float_as_uint(v.y)) |
+                   nonfinite_bits(__float_as_uint(v.z)) | nonfinite_bits(__float_as_uint(v.w));
+            *reinterpret_cast<float4 *>(buf + i) = v;
+        }
+    } else {
+        for (int i = lane; i < per; i += 32) {
+            const float v = __ldg(src + i);
+            bad |= nonfinite_bits(__float_as_uint(v));
+            buf[i] = v;
+        }
+    }
+    if (a.status && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(a.status, kStatNonFinite);
+    __syncwarp();
+    for (int m = 0; m < M; ++m) {
+        uint32_t kv[VPL];
+        int nreal = 0;
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int rep = lane + 32 * j;
+            const bool real = rep < reps;
+            kv[j] = real ? f2key(buf[rep * M + m]) : 0xFFFFFFFFu;
+            nreal += real;
+        }
+        lane_sort<VPL>(kv);
+        float med = 0.0f;
+        const bool ok = warp_median<VPL>(kv, nreal, reps, 0u, med);
+        if (lane == 0) {
+            if (!ok && a.status) atomicOr(a.status, kStatInternal);
+            const size_t o = (size_t)g * M + m;
+            a.gmed[o] = med;
+            if (a.gmed_user) a.gmed_user[o] = med;
+        }
+    }
+}
+
+template <int VPL>
+cudaError_t launch_sweep_warp(const SweepMedArgs &a, size_t smem, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(sweep_median_warp_kernel<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    sweep_median_warp_kernel<VPL><<<(a.G + kSweepWarps - 1) / kSweepWarps, kSweepWarps * 32, smem, st>>>(a);
+    return cudaGetLastError();
 }
 
 // Fallback when the repetitions of one GPU do not fit a tile: bit-by-bit counting
@@ -106,6 +170,12 @@ __global__ void sweep_verdict_kernel(const SweepVerdictArgs a, const MetricParam
 }  // namespace
 
 cudaError_t launch_sweep_medians(const SweepMedArgs &a, cudaStream_t st) {
+    const size_t wsmem = (size_t)kSweepWarps * (((size_t)a.reps * a.M + 3) & ~(size_t)3) * sizeof(float);
+    if (a.reps <= 256 && wsmem <= 96 * 1024) {
+        if (a.reps <= 64) return launch_sweep_warp<2>(a, wsmem, st);
+        if (a.reps <= 128) return launch_sweep_warp<4>(a, wsmem, st);
+        return launch_sweep_warp<8>(a, wsmem, st);
+    }
     const size_t smem = (size_t)a.reps * kSweepCols * 4;
     if (smem <= 200 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(sweep_median_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -466,7 +466,11 @@ def test_runtime_argument_errors():
 
 
 @pytest.mark.parametrize("nodes,gpn,N,M,seed", [(1, 1, 1, 1, 0), (3, 2, 5, 3, 1), (16, 8, 20, 6, 2), (5, 4, 33, 7, 3),
-                                               (2, 8, 600, 6, 4)])
+                                               (40, 8, 200, 6, 5),      # warp per GPU, 8 keys per lane, 128-bit loads
+                                               (9, 3, 100, 5, 6),       # warp per GPU, blocks not 16-byte aligned
+                                               (3, 8, 256, 32, 7),      # widest block a warp stages
+                                               (2, 8, 300, 6, 8),       # staged tile of a CTA
+                                               (2, 8, 600, 6, 4)])      # too long to stage: selection from global memory
 def test_sweep_small_matches_oracle(nodes, gpn, N, M, seed):
     from paper_2605_17879_b200 import guard
     rng = np.random.default_rng(300 + seed)
