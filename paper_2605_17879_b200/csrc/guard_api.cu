@@ -24,7 +24,7 @@ constexpr int kIngestStreams = GUARD_INGEST_STREAMS;   // internal streams the c
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, lastflag, lasttier, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, inc_lo, inc_hi, inc_cnt, inc_val, xr_big, xr_big_stride, mask, ring, total;
+    size_t status, consec, lastflag, lasttier, topk_idx, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, inc_lo, inc_hi, inc_cnt, inc_val, xr_big, xr_big_stride, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
@@ -40,6 +40,7 @@ Layout make_layout(int R, int M, int C, int K) {
     L.consec = off;    off = align_up(off + (size_t)R);
     L.lastflag = off;  off = align_up(off + (size_t)R);
     L.lasttier = off;  off = align_up(off + (size_t)R);
+    L.topk_idx = off;  off = align_up(off + (size_t)(K > 0 ? K : 1) * sizeof(int32_t));
     L.xr_split = xrank_split_supported(R, M) ? 1 : 0;
     L.xr_cluster = (!L.xr_split && xrank_cluster_supported(R, M)) ? 1 : 0;
     L.xr_steps = (!L.xr_split && !L.xr_cluster && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
@@ -148,7 +149,7 @@ struct guard_ctx {
     bool overlap = true;
     bool fork_fresh = false;          // ev_fork was recorded by an ingest not yet followed by an evaluation
     cudaStream_t side = nullptr;
-    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_topk = nullptr;
     bool ensure_side() {
         if (side) return true;
         // the evaluation's streams get the highest priority: flags should not queue behind the next blocks' sweeps
@@ -156,7 +157,8 @@ struct guard_ctx {
         cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
         if (cudaStreamCreateWithPriority(&side, cudaStreamNonBlocking, GUARD_EVAL_PRIO ? prio_hi : 0) != cudaSuccess) { side = nullptr; return false; }
         if (cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-            cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming) != cudaSuccess) {
+            cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ev_topk, cudaEventDisableTiming) != cudaSuccess) {
             cudaStreamDestroy(side);
             side = nullptr;
             return false;
@@ -262,6 +264,7 @@ struct guard_ctx {
     uint8_t *consec() const { return (uint8_t *)(ws + L.consec); }
     uint8_t *lastflag() const { return (uint8_t *)(ws + L.lastflag); }
     uint8_t *lasttier() const { return (uint8_t *)(ws + L.lasttier); }
+    int32_t *topk_idx() const { return (int32_t *)(ws + L.topk_idx); }
     float *wmed() const { return (float *)(ws + L.wmed); }
     float *step_med() const { return (float *)(ws + L.stepstat); }
     float *step_mad() const { return step_med() + (size_t)C * M; }
@@ -561,6 +564,39 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     c->inc_now = nullptr;
     if (e != cudaSuccess) return c->cuda_fail(e, "window_select launch");
 
+    // The top-k selection needs only the windowed medians: it runs beside the fleet baseline (on the
+    // internal stream, behind the window medians); its scores, which need the baseline, are filled in by
+    // the score pass.
+    const bool want_topk = c->K > 0 && (d_topk_idx || d_topk_score);
+    bool topk_side = false;
+    if (want_topk) {
+        TopkArgs t{};
+        t.R = c->R;
+        t.M = c->M;
+        t.K = c->K;
+        t.wmed = c->wmed();
+        t.fleet_med = c->fleet_med();
+        t.fleet_mad = c->fleet_mad();
+        t.cand = c->topk_cand();
+        t.ticket = c->ticket();
+        t.idx = d_topk_idx;
+        t.idx_keep = c->topk_idx();
+        t.score = nullptr;
+        if (c->overlap && c->ensure_side()) {
+            if (!(defer || forked)) {   // the window medians ran on `st`: order the internal stream behind them
+                e = cudaEventRecord(c->ev_fork, st);
+                if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
+            }
+            if (e == cudaSuccess) e = launch_topk(t, c->p, c->side);
+            if (e == cudaSuccess) e = cudaEventRecord(c->ev_topk, c->side);
+            topk_side = true;
+        } else {
+            e = launch_topk(t, c->p, ts);
+        }
+        if (e != cudaSuccess) return c->cuda_fail(e, "topk launch");
+        c->launches += 1;
+    }
+
     XrankArgs x{};
     x.base = c->wmed();
     x.row_stride = (long long)row;
@@ -595,43 +631,17 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     s.tier = d_tier;
     s.flags_keep = c->lastflag();
     s.tier_keep = c->lasttier();
-    // top-k and the score pass are independent of each other: top-k goes to the internal stream
-    const bool want_topk = c->K > 0 && (d_topk_idx || d_topk_score);
-    bool topk_forked = false;
-    TopkArgs t{};
-    if (want_topk) {
-        t.R = c->R;
-        t.M = c->M;
-        t.K = c->K;
-        t.wmed = c->wmed();
-        t.fleet_med = c->fleet_med();
-        t.fleet_mad = c->fleet_mad();
-        t.cand = c->topk_cand();
-        t.ticket = c->ticket();
-        t.idx = d_topk_idx;
-        t.score = d_topk_score;
-        if (c->overlap && c->ensure_side()) {
-            e = cudaEventRecord(c->ev_fork, ts);
-            if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
-            if (e == cudaSuccess) e = launch_topk(t, c->p, c->side);
-            if (e == cudaSuccess) e = cudaEventRecord(c->ev_join, c->side);
-            if (e != cudaSuccess) return c->cuda_fail(e, "topk launch");
-            topk_forked = true;
-            c->launches += 1;
-        }
+    s.topk_idx = want_topk ? c->topk_idx() : nullptr;
+    s.topk_score = want_topk ? d_topk_score : nullptr;
+    s.K = c->K;
+    if (topk_side) {
+        e = cudaStreamWaitEvent(ts, c->ev_topk, 0);
+        if (e != cudaSuccess) return c->cuda_fail(e, "topk join");
     }
     e = launch_score_flag(s, c->p, ts);
     if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
     c->evals += 1;
     c->launches += 1 + window_launch_count(w);
-    if (topk_forked) {
-        e = cudaStreamWaitEvent(ts, c->ev_join, 0);
-        if (e != cudaSuccess) return c->cuda_fail(e, "topk join");
-    } else if (want_topk) {
-        e = launch_topk(t, c->p, ts);
-        if (e != cudaSuccess) return c->cuda_fail(e, "topk launch");
-        c->launches += 1;
-    }
     if (defer) {
         e = cudaEventRecord(c->ev_e, c->tail);
         if (e != cudaSuccess) return c->cuda_fail(e, "event record");
@@ -1059,6 +1069,7 @@ void guard_destroy(guard_ctx *c) {
             cudaStreamDestroy(c->side);
             cudaEventDestroy(c->ev_fork);
             cudaEventDestroy(c->ev_join);
+            if (c->ev_topk) cudaEventDestroy(c->ev_topk);
         }
     }
     delete c;

@@ -135,6 +135,11 @@ struct ScoreArgs {
     uint8_t *tier;           // [R] or NULL
     uint8_t *flags_keep;     // [R] the context's own copy (input of the node-level fold), never NULL
     uint8_t *tier_keep;      // [R] likewise
+    // scores of an already selected top-k list (the selection itself needs no fleet statistics and runs
+    // beside the fleet baseline): topk_score[i] = primary score of rank topk_idx[i]; NULL / 0 to skip
+    const int32_t *topk_idx;
+    float *topk_score;
+    int K;
 };
 cudaError_t launch_score_flag(const ScoreArgs &a, const MetricParams &p, cudaStream_t st);
 
@@ -160,7 +165,8 @@ struct TopkArgs {
     unsigned long long *cand;   // scratch [topk_blocks(R)][K]
     unsigned int *ticket;       // scratch, zero before first use (self-resetting)
     int32_t *idx;               // [K] or NULL
-    float *score;               // [K] or NULL
+    int32_t *idx_keep;          // [K] second copy of the indices (the context's own), or NULL
+    float *score;               // [K] or NULL: needs fleet_med / fleet_mad to be final when the kernel runs
 };
 int topk_blocks(int R);
 // Records the text guard_last_error(NULL) returns (defined next to the C ABI).

@@ -9,6 +9,19 @@ namespace {
 
 constexpr int kScoreThreads = 128;
 
+// Scores of the ranks a top-k selection has already picked (first CTA only): the same float32
+// arithmetic as the per-rank scores.
+__device__ __forceinline__ void topk_scores(const ScoreArgs &a, const MetricParams &p, const float *s_B, const float *s_Ds) {
+    if (blockIdx.x != 0 || !a.topk_score || !a.topk_idx) return;
+    const int pm = p.primary;
+    for (int i = threadIdx.x; i < a.K; i += blockDim.x) {
+        const int r = a.topk_idx[i];
+        float dev = __fsub_rn(a.wmed[(size_t)r * a.M + pm], s_B[pm]);
+        if (p.dir[pm] < 0) dev = -dev;
+        a.topk_score[i] = (dev == 0.0f) ? 0.0f : __fdiv_rn(__fmul_rn(0.6745f, dev), s_Ds[pm]);
+    }
+}
+
 template <typename MaskT, int NM>
 __global__ void __launch_bounds__(kScoreThreads) score_flag_kernel(const ScoreArgs a, const MetricParams p) {
     __shared__ float s_B[kMaxMetrics], s_rhs[kMaxMetrics], s_Ds[kMaxMetrics];
@@ -22,6 +35,7 @@ __global__ void __launch_bounds__(kScoreThreads) score_flag_kernel(const ScoreAr
         s_rhs[m] = __fmul_rn(p.thrp[m], Ds);
     }
     __syncthreads();
+    topk_scores(a, p, s_B, s_Ds);
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= a.R) return;
 
@@ -93,6 +107,8 @@ __global__ void __launch_bounds__(kFastWarps * 32) score_flag_bytes_kernel(const
         s_Ds[tid] = Ds;
         s_rhs[tid] = __fmul_rn(p.thrp[tid], Ds);
     }
+    __syncthreads();
+    topk_scores(a, p, s_B, s_Ds);
     const int r0 = blockIdx.x * kFastRanks;
     const uint8_t *mask_base = (const uint8_t *)a.mask_base;
     const int first = ((a.last_slot - (a.n - 1)) % a.capacity + a.capacity) % a.capacity;

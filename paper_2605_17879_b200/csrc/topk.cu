@@ -129,11 +129,13 @@ __global__ void __launch_bounds__(kTopThreads) topk_kernel(const TopkArgs a, con
             fold_topk(e, K, list, run, sh, &s_n);
         }
     }
-    const float B = a.fleet_med[pm];
-    const float Ds = scale_of(a.fleet_mad[pm], B, p.floor_rel[pm], p.floor_abs[pm]);
+    // scores only where the caller asked for them here (then the fleet statistics are final already)
+    const float B = a.score ? a.fleet_med[pm] : 0.0f;
+    const float Ds = a.score ? scale_of(a.fleet_mad[pm], B, p.floor_rel[pm], p.floor_abs[pm]) : 1.0f;
     for (int i = tid; i < K; i += blockDim.x) {
         const int r = (int)(0xFFFFFFFFu - (uint32_t)(run[i] & 0xFFFFFFFFull));
         if (a.idx) a.idx[i] = r;
+        if (a.idx_keep) a.idx_keep[i] = r;
         if (a.score) {
             float dev = __fsub_rn(a.wmed[(size_t)r * a.M + pm], B);
             if (dirp < 0) dev = -dev;
@@ -150,7 +152,7 @@ int topk_blocks(int R) {
 }
 
 cudaError_t launch_topk(const TopkArgs &a, const MetricParams &p, cudaStream_t st) {
-    if (a.K <= 0 || (!a.idx && !a.score)) return cudaSuccess;
+    if (a.K <= 0 || (!a.idx && !a.score && !a.idx_keep)) return cudaSuccess;
     const int nb = topk_blocks(a.R);
     topk_kernel<<<nb, kTopThreads, 0, st>>>(a, p, nb);
     return cudaGetLastError();
