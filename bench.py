@@ -37,7 +37,7 @@ UNIT = "cells/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this workload, from
 # the ncu capture summarised under profiles/ (None once the kernel has changed since the capture)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 116.14e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 118.60e6
 # which kernel the roofline object describes: 2 = window_thread_kernel (guard_score), 1 = the MAD sweep (guard_ingest)
 PROFILE_MODE = 2
 PROFILE_KERNEL = ("window_thread_kernel (windowed per-rank medians of one evaluation)" if PROFILE_MODE == 2 else
@@ -355,11 +355,23 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-all-cores", action="store_true", help="skip the all-core leg of the CPU baseline")
     ap.add_argument("--streaming-steps", type=int, default=500)
+    ap.add_argument("--only", default="", choices=["", "streaming", "sweep"],
+                    help="run only this secondary leg and print its object (for profiling; not a bench line)")
     ap.add_argument("--blocks", type=int, default=0,
                     help="profile-sized run: only this many 200-step blocks of the workload (0 = all 100); not a bench value")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.only:
+        # profile-sized runs of one secondary leg (not a bench line): prints that leg's object only
+        import torch
+        from paper_2605_17879_b200 import guard
+        guard.lib()
+        dev = torch.device("cuda", 0)
+        torch.cuda.set_device(dev)
+        res = run_streaming(dev, args.streaming_steps, 250) if args.only == "streaming" else run_sweep(dev)
+        print(json.dumps({"only": args.only, "result": res}), flush=True)
+        return 0
 
     import torch
     from paper_2605_17879_b200 import dist as gd, guard, synth

@@ -98,6 +98,96 @@ __global__ void __launch_bounds__(kColThreads) xrank_column_kernel(const XrankAr
     }
 }
 
+// The same with every column spread over a cluster of NC CTAs (wide fleets: one CTA per column is
+// bound by instruction issue on its SM; four SMs per column share the histogram rounds through
+// distributed shared memory).  CTA c of the cluster holds ranks (i * NC + c) * 1024 + tid.
+template <int VPT, int NC, typename MaskT>
+__global__ void __cluster_dims__(NC, 1, 1) __launch_bounds__(kColThreads)
+    xrank_column_cluster_kernel(const XrankArgs a, const MetricParams p) {
+    __shared__ ColShared sh;
+    const int m = blockIdx.x / NC, t = blockIdx.y, tid = threadIdx.x, lane = lane_id();
+    const int crank = (int)cl_rank();
+    const int R = a.R, M = a.M;
+    const int slot = (int)(((long long)a.first_slot + t) % a.capacity);
+    const float *row = a.base + (size_t)slot * a.row_stride;
+    const size_t col = (size_t)t * M + m;
+    const bool even = (R & 1) == 0;
+    const uint32_t k1 = (uint32_t)((R - 1) / 2);
+
+    float x[VPT];
+    uint32_t key[VPT];
+    uint32_t valid = 0;
+    bool bad = false;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int r = (i * NC + crank) * kColThreads + tid;
+        x[i] = 0.0f;
+        if (r < R) {
+            x[i] = __ldg(row + (size_t)r * M + m);
+            valid |= 1u << i;
+            bad |= nonfinite_bits(__float_as_uint(x[i]));
+        }
+        key[i] = f2key(x[i]);
+    }
+    if (a.check_finite && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(a.status, kStatNonFinite);
+
+    uint32_t v1, v2;
+    bool ok = colc_select_regs<VPT, NC>(key, valid, k1, even, sh, v1, v2);
+    const float med = median_from_keys(v1, v2, even);
+    if (a.cut) {
+        uint32_t c1, c2;
+        ok = colc_select_regs<VPT, NC>(key, valid, (uint32_t)a.cut_rank[m], false, sh, c1, c2) && ok;
+        if (tid == 0 && crank == 0) a.cut[col] = key2f(c1);
+    }
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) key[i] = f2key(fabsf(__fsub_rn(x[i], med)));
+    ok = colc_select_regs<VPT, NC>(key, valid, k1, even, sh, v1, v2) && ok;
+    const float mad = median_from_keys(v1, v2, even);
+    if (tid == 0 && crank == 0) {
+        if (!ok) atomicOr(a.status, kStatInternal);
+        a.med[col] = med;
+        a.mad[col] = mad;
+        if (a.med_user) a.med_user[col] = med;
+        if (a.mad_user) a.mad_user[col] = mad;
+    }
+    if (a.mask_base) {
+        // the mask row was zeroed before the launch; the CTAs of a row OR their bits in
+        const float rhs = __fmul_rn(p.thrp[m], scale_of(mad, med, p.floor_rel[m], p.floor_abs[m]));
+        const int dir = p.dir[m];
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int r = (i * NC + crank) * kColThreads + tid;
+            const uint32_t e = (((valid >> i) & 1u) && exceeds(x[i], med, dir, rhs)) ? 1u : 0u;
+            if (sizeof(MaskT) == 1 && (R & 3) == 0) {
+                // four adjacent ranks share a 32-bit word: combine their bits, one atomic per word
+                uint32_t b = (e << m) << (8 * (tid & 3));
+                b |= __shfl_xor_sync(0xFFFFFFFFu, b, 1);
+                b |= __shfl_xor_sync(0xFFFFFFFFu, b, 2);
+                if ((tid & 3) == 0 && b)
+                    atomicOr(reinterpret_cast<unsigned int *>(reinterpret_cast<uintptr_t>(a.mask_base) + (size_t)slot * R + (size_t)r), b);
+            } else if (e) {
+                if (sizeof(MaskT) == 1) {
+                    const size_t bi = (size_t)slot * R + (size_t)r;
+                    unsigned int *w = reinterpret_cast<unsigned int *>(reinterpret_cast<uintptr_t>(a.mask_base) + (bi & ~(size_t)3));
+                    atomicOr(w, (1u << m) << (8 * (bi & 3)));
+                } else {
+                    atomicOr(reinterpret_cast<unsigned int *>(a.mask_base) + (size_t)slot * R + r, 1u << m);
+                }
+            }
+        }
+    }
+}
+
+constexpr int kColCluster = 4;
+
+template <int VPT>
+cudaError_t launch_cluster_vpt(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st) {
+    const dim3 grid(a.M * kColCluster, S);
+    if (a.mask_bytes == 4) xrank_column_cluster_kernel<VPT, kColCluster, uint32_t><<<grid, kColThreads, 0, st>>>(a, p);
+    else xrank_column_cluster_kernel<VPT, kColCluster, uint8_t><<<grid, kColThreads, 0, st>>>(a, p);
+    return cudaGetLastError();
+}
+
 template <int VPT>
 cudaError_t launch_vpt(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st) {
     const dim3 grid(a.M, S);
@@ -123,6 +213,10 @@ cudaError_t launch_xrank_column(const XrankArgs &a, const MetricParams &p, int S
         if (e != cudaSuccess) return e;
     }
     const int vpt = (a.R + kColThreads - 1) / kColThreads;
+    // the widest columns (more than 16 keys per thread of a single CTA) take a cluster of four CTAs each:
+    // measured 45 -> 35 us per launch at 32 768 ranks; at 16 384 ranks the cluster barriers cost more than
+    // the shared work saves (node sweep 0.13 -> 0.18 ms), so narrower columns stay with one CTA
+    if (vpt > 16) return launch_cluster_vpt<8>(a, p, S, st);
     if (vpt <= 4) return launch_vpt<4>(a, p, S, st);
     if (vpt <= 8) return launch_vpt<8>(a, p, S, st);
     if (vpt <= 16) return launch_vpt<16>(a, p, S, st);

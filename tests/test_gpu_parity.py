@@ -61,6 +61,9 @@ def test_small_fleets_match_oracle(R, M, W, k, K, T, blocks, cap):
     (4100, 16, 4, 8, None),
     (4096, 32, 3, 6, None),
     (6001, 8, 4, 8, None),         # odd rank count: a single middle element
+    (20001, 3, 4, 8, None),        # few columns at a time, wide: a cluster of four CTAs per column; odd rank count (byte-wise mask atomics)
+    (17000, 9, 3, 6, None),        # the same with 32-bit exceedance masks
+    (32768, 2, 3, 6, 40),          # widest column the clusters hold (8 keys per thread), quantised values (ties)
     (4096, 8, 4, 8, 50),           # quantised: intervals collapse onto tied values, some steps fall back
     (8192, 4, 4, 8, 4),            # very coarse: candidate lists overflow, every step falls back
 ])
