@@ -269,7 +269,9 @@ int guard_set_overlap(guard_ctx *ctx, int on);
  * steps (the online monitor of Sec. 4.2 / 7.1 re-evaluates every step or poll), consecutive
  * windows share almost all their steps; guard_score then updates a small per-series state (an
  * interval around the series' median, the count of window values below it, the values inside)
- * from the few steps that entered and left the window instead of reading the whole window again.
+ * from the few steps that entered and left the window instead of reading the whole window again
+ * (the steps that left must still be in the ring: capacity_steps >= W + the steps between two
+ * evaluations, else every evaluation reads its whole window).
  * Series whose median has left their interval are rebuilt from the window.  Results are identical
  * either way; guard_set_sliding(ctx, 0) makes every evaluation read its whole window. */
 int guard_set_sliding(guard_ctx *ctx, int on);

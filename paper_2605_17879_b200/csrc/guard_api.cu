@@ -24,7 +24,7 @@ constexpr int kIngestStreams = GUARD_INGEST_STREAMS;   // internal streams the c
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, lastflag, lasttier, topk_idx, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, inc_lo, inc_hi, inc_cnt, inc_val, xr_big, xr_big_stride, mask, ring, total;
+    size_t status, consec, lastflag, lasttier, topk_idx, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, kcnt, inc_lo, inc_hi, inc_cnt, inc_val, xr_big, xr_big_stride, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
@@ -50,6 +50,7 @@ Layout make_layout(int R, int M, int C, int K) {
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
     L.wspread = off;   off = align_up(off + (size_t)R * M * sizeof(float));
     L.wcentre = off;   off = align_up(off + (size_t)R * M * sizeof(float));
+    L.kcnt = off;      off = align_up(off + (size_t)R * M * sizeof(uint16_t));   // k-of-W counts of the last evaluation's window
     // sliding-window state: interval ends, packed counts, listed values
     L.inc_lo = off;    off = align_up(off + window_inc_bytes(R * M));
     L.inc_hi = off;    off = align_up(off + window_inc_bytes(R * M));
@@ -142,6 +143,8 @@ struct guard_ctx {
     // (-1: none).  hints_ready: a whole-window kernel has seeded the per-series search intervals.
     long long inc_seen = -1;
     int inc_n = 0;
+    long long cnt_seen = -1;      // the k-of-W counts kept in the workspace hold for the window of cnt_n steps ending here
+    int cnt_n = 0;
     bool sliding = true;          // guard_set_sliding
     bool hints_ready = false;
     // overlap of the window medians (which need only the ring) with the cross-rank kernels of the
@@ -492,8 +495,11 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     // Evaluations that follow one another by a few steps: the sliding update reads only the steps that
     // entered and left the window since its per-series state was current (or rebuilds that state).
     IncArgs ia{};
-    const bool close = c->evals > 0 ? (c->seen - c->seen_at_eval) <= kIncMaxNew : c->seen <= kIncMaxNew;
-    const bool use_inc = c->sliding && close && window_inc_supported(w);
+    const long long gap = c->evals > 0 ? c->seen - c->seen_at_eval : c->seen;   // steps since the previous evaluation
+    // the steps that leave the window must still be in the ring when the next evaluation slides: a ring of
+    // exactly W steps has overwritten them, and rebuilding every series every time would cost more than the
+    // whole-window kernels
+    const bool use_inc = c->sliding && gap <= kIncMaxNew && window_inc_supported(w) && (long long)c->C >= n + (gap > 0 ? gap : 1);
     if (use_inc) {
         ia.lo = (float *)(c->ws + c->L.inc_lo);
         ia.hi = (float *)(c->ws + c->L.inc_hi);
@@ -631,6 +637,19 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     s.tier = d_tier;
     s.flags_keep = c->lastflag();
     s.tier_keep = c->lasttier();
+    // k-of-W counts slide like the window medians: the previous evaluation's counts plus / minus the exceedance
+    // rows of the steps that entered / left (the rows that left must still be in the exceedance ring)
+    s.kcnt = (uint16_t *)(c->ws + c->L.kcnt);
+    {
+        const long long p1 = c->cnt_seen, p0 = p1 - c->cnt_n, q1 = c->seen, q0 = q1 - n;
+        if (c->sliding && p1 >= 0 && q0 < p1 && q1 - p1 <= kIncMaxNew && q0 - p0 <= kIncMaxNew && q1 - p0 <= c->C) {
+            s.slide = 1;
+            s.entering = (int)(q1 - p1);
+            s.leaving = (int)(q0 - p0);
+        }
+        c->cnt_seen = c->seen;
+        c->cnt_n = n;
+    }
     s.topk_idx = want_topk ? c->topk_idx() : nullptr;
     s.topk_score = want_topk ? d_topk_score : nullptr;
     s.K = c->K;
@@ -646,7 +665,8 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         e = cudaEventRecord(c->ev_e, c->tail);
         if (e != cudaSuccess) return c->cuda_fail(e, "event record");
         c->pending = true;
-        c->pending_n = n + (use_inc ? ia.leaving : 0);   // the sliding update also reads the steps that just left the window
+        // the sliding updates also read the steps that just left the window
+        c->pending_n = n + ((use_inc ? ia.leaving : 0) > s.leaving ? (use_inc ? ia.leaving : 0) : s.leaving);
         c->pending_seen = c->seen;
     }
     return GUARD_OK;
@@ -909,6 +929,7 @@ int guard_state_import(guard_ctx *c, const void *d_state, size_t state_bytes, vo
     c->seen_at_eval = h.seen_at_eval;
     c->inc_seen = h.inc_seen;
     c->inc_n = h.inc_n;
+    c->cnt_seen = -1;   // the kept counts are not part of the state: the next evaluation recounts
     c->hints_ready = h.hints_ready != 0;
     c->fork_fresh = false;
     return GUARD_OK;
@@ -943,6 +964,7 @@ int guard_reset(guard_ctx *c, void *stream) {
     c->evals = 0;
     c->seen_at_eval = 0;
     c->inc_seen = -1;
+    c->cnt_seen = -1;
     c->hints_ready = false;
     return GUARD_OK;
 }

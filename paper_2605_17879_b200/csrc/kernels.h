@@ -140,6 +140,11 @@ struct ScoreArgs {
     const int32_t *topk_idx;
     float *topk_score;
     int K;
+    // k-of-W counts kept across evaluations: kcnt [R][M] is rewritten by every evaluation; with slide != 0
+    // it holds the counts of the previous evaluation's window and only the exceedance rows of the
+    // `entering` newest steps and of the `leaving` steps right before the window's oldest step are read
+    uint16_t *kcnt;
+    int slide, entering, leaving;
 };
 cudaError_t launch_score_flag(const ScoreArgs &a, const MetricParams &p, cudaStream_t st);
 

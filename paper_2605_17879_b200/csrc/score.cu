@@ -45,11 +45,37 @@ __global__ void __launch_bounds__(kScoreThreads) score_flag_kernel(const ScoreAr
     for (int m = 0; m < NM; ++m) cnt[m] = 0;
     const MaskT *mask_base = (const MaskT *)a.mask_base;
     int slot = ((a.last_slot - (a.n - 1)) % a.capacity + a.capacity) % a.capacity;
-    for (int j = 0; j < a.n; ++j) {
-        const uint32_t e = mask_base[(size_t)slot * a.R + r];
+    if (a.slide) {
+        // the previous window's counts, minus the steps that left, plus the steps that entered
 #pragma unroll
-        for (int m = 0; m < NM; ++m) cnt[m] += (e >> m) & 1u;
-        if (++slot == a.capacity) slot = 0;
+        for (int m = 0; m < NM; ++m)
+            if (m < M) cnt[m] = a.kcnt[(size_t)r * M + m];
+        for (int i = 0; i < a.leaving; ++i) {
+            int sl = slot - a.leaving + i;
+            if (sl < 0) sl += a.capacity;
+            const uint32_t e = mask_base[(size_t)sl * a.R + r];
+#pragma unroll
+            for (int m = 0; m < NM; ++m) cnt[m] -= (e >> m) & 1u;
+        }
+        for (int i = 0; i < a.entering; ++i) {
+            int sl = a.last_slot - i;
+            if (sl < 0) sl += a.capacity;
+            const uint32_t e = mask_base[(size_t)sl * a.R + r];
+#pragma unroll
+            for (int m = 0; m < NM; ++m) cnt[m] += (e >> m) & 1u;
+        }
+    } else {
+        for (int j = 0; j < a.n; ++j) {
+            const uint32_t e = mask_base[(size_t)slot * a.R + r];
+#pragma unroll
+            for (int m = 0; m < NM; ++m) cnt[m] += (e >> m) & 1u;
+            if (++slot == a.capacity) slot = 0;
+        }
+    }
+    if (a.kcnt) {
+#pragma unroll
+        for (int m = 0; m < NM; ++m)
+            if (m < M) a.kcnt[(size_t)r * M + m] = (uint16_t)cnt[m];
     }
 
     uint32_t mask = 0;
@@ -124,7 +150,7 @@ __global__ void __launch_bounds__(kFastWarps * 32) score_flag_bytes_kernel(const
         for (int m = 0; m < 8; ++m) sums[q][m] = 0;
     int pending = 0;
     constexpr int KU = 5;   // window steps whose loads are in flight together
-    for (int j0 = w; j0 < a.n; j0 += kFastWarps * KU) {
+    for (int j0 = w; !a.slide && j0 < a.n; j0 += kFastWarps * KU) {
         uint32_t word[KU];
 #pragma unroll
         for (int u = 0; u < KU; ++u) {
@@ -175,12 +201,32 @@ __global__ void __launch_bounds__(kFastWarps * 32) score_flag_bytes_kernel(const
     if (tid >= kFastRanks) return;
     const int r = r0 + tid;
     if (r >= a.R) return;
+    // sliding counts: the exceedance bytes of the few steps that left and entered the window, for this rank
+    int slide_delta[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (a.slide) {
+        for (int i = 0; i < a.leaving; ++i) {
+            int sl = first - a.leaving + i;
+            if (sl < 0) sl += a.capacity;
+            const uint32_t e = mask_base[(size_t)sl * a.R + r];
+#pragma unroll
+            for (int m = 0; m < 8; ++m) slide_delta[m] -= (int)((e >> m) & 1u);
+        }
+        for (int i = 0; i < a.entering; ++i) {
+            int sl = a.last_slot - i;
+            if (sl < 0) sl += a.capacity;
+            const uint32_t e = mask_base[(size_t)sl * a.R + r];
+#pragma unroll
+            for (int m = 0; m < 8; ++m) slide_delta[m] += (int)((e >> m) & 1u);
+        }
+    }
     uint32_t mask = 0;
     const float *wv = a.wmed + (size_t)r * M;
 #pragma unroll
     for (int m = 0; m < 8; ++m) {
         if (m < M) {
-            const int cnt = (int)s_cnt[tid][m];
+            int cnt = (int)s_cnt[tid][m];
+            if (a.slide) cnt = (int)a.kcnt[(size_t)r * M + m] + slide_delta[m];
+            if (a.kcnt) a.kcnt[(size_t)r * M + m] = (uint16_t)cnt;
             float dev = __fsub_rn(wv[m], s_B[m]);
             if (p.dir[m] < 0) dev = -dev;
             if (dev > s_rhs[m] && cnt >= p.k) mask |= 1u << m;
