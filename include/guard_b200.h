@@ -21,7 +21,7 @@
  *   - `stream` is a cudaStream_t passed as void*.  All work is ordered on it.  The calls that
  *     synchronise `stream` with the host are the ones that hand a value back from the device:
  *     guard_sync_status, guard_fallback_steps, guard_fallback_reasons, guard_window_fallbacks,
- *     guard_sliding_rebuilds and guard_state_import;
+ *     guard_sliding_rebuilds, guard_row_hints and guard_state_import;
  *     guard_profile_read waits for the events it recorded.  No other call synchronises.
  *     (guard_score may run the window medians on an internal stream forked from and joined back
  *     into `stream` with events, so that they overlap the preceding guard_ingest; to the caller
@@ -275,6 +275,23 @@ int guard_set_overlap(guard_ctx *ctx, int on);
  * Series whose median has left their interval are rebuilt from the window.  Results are identical
  * either way; guard_set_sliding(ctx, 0) makes every evaluation read its whole window. */
 int guard_set_sliding(guard_ctx *ctx, int on);
+
+/* Single rows of wide fleets (on by default).  The cross-rank statistics of a one-step ingest and
+ * the fleet baseline of an evaluation (Sec. 4.2: median and MAD over all ranks) are each ONE row; from
+ * 8 192 ranks on, a call site keeps its previous median and MAD and a tuned width per metric, which
+ * bracket the next row's: the selection then counts the values below the bracket, bins the few inside
+ * and ranks the wanted bin's values directly.  The counts prove the bracket; a row they do not prove
+ * (the first one, a jump, ties) takes the general selection inside the same kernel.  Results are
+ * identical either way; guard_set_row_hints(ctx, 0) always takes the general selection. */
+int guard_set_row_hints(guard_ctx *ctx, int on);
+
+/* Diagnostic: synchronises `stream` and fills out[6] (HOST): single rows seen and (row, metric)
+ * columns whose median and MAD both came out of their brackets, 0-1 for ingested steps, 2-3 for
+ * fleet baselines (zero where hints do not apply); 4-5: evaluations whose top-k list (Sec. 4.2: the
+ * slowest ranks) came from the candidates above the previous evaluation's threshold, and
+ * evaluations that had to rank all ranks instead (evaluations at most 8 steps apart try the
+ * threshold first; the list is identical either way).  Since creation / reset / state import. */
+int guard_row_hints(guard_ctx *ctx, uint32_t out[6], void *stream);
 
 /* Deferred evaluations (off by default).  While on, guard_score enqueues the evaluation on
  * streams of the library's own, ordered after everything enqueued on `stream` so far, and

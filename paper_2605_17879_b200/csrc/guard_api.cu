@@ -1,6 +1,7 @@
 // C ABI of the library: context object, workspace carving, argument checks and the
 // stream-ordered kernel sequences behind guard_ingest / guard_score / guard_sweep_qualify.
 #include <cstdarg>
+#include <cstddef>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -24,10 +25,11 @@ constexpr int kIngestStreams = GUARD_INGEST_STREAMS;   // internal streams the c
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, lastflag, lasttier, topk_idx, ticket, fleet, xr_small, wmed, stepstat, topk_cand, wspread, wcentre, kcnt, inc_lo, inc_hi, inc_cnt, inc_val, xr_big, xr_big_stride, mask, ring, total;
+    size_t status, consec, lastflag, lasttier, topk_idx, topk_hint, ticket, fleet, xr_small, xr_grid, wmed, stepstat, topk_cand, wspread, wcentre, kcnt, inc_lo, inc_hi, inc_cnt, inc_val, xr_big, xr_big_stride, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
+    int xr_gridp;   // single rows keep brackets between calls (two ColHintState at xr_grid: ingest, fleet baseline)
 };
 
 // State and scratch first, the two rings last (the telemetry ring is by far the largest).
@@ -41,10 +43,13 @@ Layout make_layout(int R, int M, int C, int K) {
     L.lastflag = off;  off = align_up(off + (size_t)R);
     L.lasttier = off;  off = align_up(off + (size_t)R);
     L.topk_idx = off;  off = align_up(off + (size_t)(K > 0 ? K : 1) * sizeof(int32_t));
+    L.topk_hint = off; off = align_up(off + 256 + 1024 * sizeof(unsigned long long));   // TopkHint, then the hinted pass's list
     L.xr_split = xrank_split_supported(R, M) ? 1 : 0;
     L.xr_cluster = (!L.xr_split && xrank_cluster_supported(R, M)) ? 1 : 0;
     L.xr_steps = (!L.xr_split && !L.xr_cluster && xrank_bracket_supported(R, M)) ? xrank_scratch_steps(R, M, C) : 0;
     L.xr_small = off;  off = align_up(off + (L.xr_steps ? xrank_scratch_small_bytes(M, L.xr_steps) : 0));
+    L.xr_gridp = (xrank_column_supported(R) && R >= 8192) ? 1 : 0;
+    L.xr_grid = off;   off = align_up(off + 2 * align_up(sizeof(ColHintState)));
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
@@ -211,8 +216,13 @@ struct guard_ctx {
     // steps that ended where `seen` stood when it was enqueued; an internal ingest stream reads the
     // blocks enqueued on it since it was last joined.  Everything from that step on is protected.
     // Work whose end event has already completed (a host-side query, no waiting) reads nothing any more.
-    long long protected_steps() {
+    long long protected_steps(int need) {
         long long first = seen;
+        if (pending && pending_seen - pending_n < first) first = pending_seen - pending_n;
+        for (int k = 0; k < kIngestStreams; ++k)
+            if (xs_busy[k] && xs_first[k] < first) first = xs_first[k];
+        if (need + (seen - first) <= C) return seen - first;   // no conflict even if all of it is still running: nothing to query
+        first = seen;
         if (pending && pending_seen - pending_n < first && cudaEventQuery(ev_e) != cudaSuccess) first = pending_seen - pending_n;
         for (int k = 0; k < kIngestStreams; ++k)
             if (xs_busy[k] && xs_first[k] < first) {
@@ -279,9 +289,14 @@ struct guard_ctx {
     // own_scratch = false: the call may run beside another cross-rank call of this context (the fleet
     // baseline of a deferred evaluation beside the next ingest), so it must not touch the one
     // scratch of the bracketed path: such rows take the direct selection.
-    cudaError_t xrank(XrankArgs a, int S, cudaStream_t st, bool own_scratch = true) {
+    // site: 0 the ingested step, 1 the fleet baseline, -1 neither.  A site keeps the brackets of its single rows.
+    bool row_hints = true;   // guard_set_row_hints
+    ColHintState *hint_state(int site) const { return (ColHintState *)(ws + L.xr_grid + (size_t)site * align_up(sizeof(ColHintState))); }
+    cudaError_t xrank(XrankArgs a, int S, cudaStream_t st, bool own_scratch = true, int site = -1) {
         // a few rows at a time: one CTA per column keeps the whole GPU busy
         if (xrank_column_supported(R) && (long long)S * M <= 64 && !a.cut) {
+            // one row of a wide fleet: bracketed by the call site's previous result
+            if (S == 1 && site >= 0 && L.xr_gridp && row_hints) a.hint = hint_state(site);
             launches += 1;
             return launch_xrank_column(a, p, S, st);
         }
@@ -396,7 +411,7 @@ int guard_ring_reserve(guard_ctx *c, int steps, float **d_slot) {
     if (!d_slot || steps < 1 || steps > c->C) return c->fail(GUARD_ERR_ARG, "steps must be in 1..capacity and d_slot non-NULL");
     const int slot = (int)(c->seen % c->C);
     if (slot + steps > c->C) return c->fail(GUARD_ERR_ARG, "reserved span would wrap around the ring (slot %d + %d > %d)", slot, steps, c->C);
-    if (steps + c->protected_steps() > c->C)
+    if (steps + c->protected_steps(steps) > c->C)
         return c->fail(GUARD_ERR_NOT_READY, "the reserved slots are still read by deferred work: call guard_join first");
     *d_slot = c->ring() + (size_t)slot * c->R * c->M;
     return GUARD_OK;
@@ -410,7 +425,7 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
     const size_t row = (size_t)c->R * c->M;
     const int slot = (int)(c->seen % c->C);
     const bool in_place = (d_block == c->ring() + (size_t)slot * row) && (slot + B <= c->C);
-    if (B + c->protected_steps() > c->C) {   // this block's slots are still read by deferred work
+    if (B + c->protected_steps(B) > c->C) {   // this block's slots are still read by deferred work
         cudaError_t e = c->join(st);
         if (e == cudaSuccess) e = c->join_xs(st);
         if (e != cudaSuccess) return c->cuda_fail(e, "join of deferred work");
@@ -460,7 +475,7 @@ int guard_ingest(guard_ctx *c, const float *d_block, int B, float *d_step_med, f
         c->xs_busy[k] = true;
     } else {
         e = c->join_xs(st);   // earlier blocks still on the internal streams come first
-        if (e == cudaSuccess) e = c->xrank(a, B, st);
+        if (e == cudaSuccess) e = c->xrank(a, B, st, true, 0);
     }
     if (e != cudaSuccess) return c->cuda_fail(e, "xrank launch");
     c->seen += B;
@@ -588,6 +603,11 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         t.idx = d_topk_idx;
         t.idx_keep = c->topk_idx();
         t.score = nullptr;
+        // evaluations a few steps apart: the previous evaluation's threshold pre-selects the candidates
+        if (c->sliding && gap <= kIncMaxNew) {
+            t.hint = (TopkHint *)(c->ws + c->L.topk_hint);
+            t.hcand = (unsigned long long *)(c->ws + c->L.topk_hint + 256);
+        }
         if (c->overlap && c->ensure_side()) {
             if (!(defer || forked)) {   // the window medians ran on `st`: order the internal stream behind them
                 e = cudaEventRecord(c->ev_fork, st);
@@ -600,7 +620,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
             e = launch_topk(t, c->p, ts);
         }
         if (e != cudaSuccess) return c->cuda_fail(e, "topk launch");
-        c->launches += 1;
+        c->launches += t.hint ? 2 : 1;
     }
 
     XrankArgs x{};
@@ -615,7 +635,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     x.med_user = d_fleet_med;
     x.mad_user = d_fleet_mad;
     x.status = c->status();
-    e = c->xrank(x, 1, ts, !defer);
+    e = c->xrank(x, 1, ts, !defer, 1);
     if (e != cudaSuccess) return c->cuda_fail(e, "fleet baseline launch");
 
     ScoreArgs s{};
@@ -1046,6 +1066,27 @@ int64_t guard_fallback_steps(guard_ctx *c, void *stream) {
 int guard_set_sliding(guard_ctx *c, int on) {
     if (!c) return GUARD_ERR_ARG;
     c->sliding = on != 0;
+    return GUARD_OK;
+}
+
+int guard_set_row_hints(guard_ctx *c, int on) {
+    if (!c) return GUARD_ERR_ARG;
+    c->row_hints = on != 0;
+    return GUARD_OK;
+}
+
+int guard_row_hints(guard_ctx *c, uint32_t out[6], void *stream) {
+    if (!c || !out) return GUARD_ERR_ARG;
+    for (int i = 0; i < 6; ++i) out[i] = 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = c->join(st);
+    if (e == cudaSuccess) e = c->join_xs(st);
+    for (int site = 0; site < 2 && e == cudaSuccess && c->L.xr_gridp; ++site)   // rows and settled are the first two words
+        e = cudaMemcpyAsync(&out[2 * site], c->hint_state(site), 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess)   // hits and misses of the hinted top-k pass
+        e = cudaMemcpyAsync(&out[4], (char *)(c->ws + c->L.topk_hint) + offsetof(TopkHint, hits), 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return c->cuda_fail(e, "guard_row_hints");
     return GUARD_OK;
 }
 

@@ -27,6 +27,7 @@ struct XrankArgs {
     uint32_t *status;
     uint32_t *only_flagged; // [S] or NULL: direct kernel processes step s only if nonzero, then clears it
     uint32_t *fallbacks;    // or NULL: counts the steps the direct kernel redid for the bracketed path
+    void *hint;             // ColHintState of the call site (one row per call), or NULL: column kernels only
 };
 
 // Scratch of the bracketed path for up to S_max steps per launch.
@@ -44,6 +45,18 @@ struct XrankScratch {
     int cap, amb_cap, S_max;
 };
 enum { kWhyCtaList = 0, kWhyStepList = 1, kWhyAmbList = 2, kWhyMedianMiss = 3, kWhySelect = 4, kWhyMadMiss = 5 };
+// State a call site of the column kernels keeps between its rows (zero before first use): the previous
+// median / MAD in the output arrays bracket the next ones; hw holds the tuned half-widths of the two
+// brackets per metric (0: derive from the MAD; negative: rows left before the hint is tried again).
+struct ColHintState {
+    uint32_t rows;       // diagnostic: rows seen
+    uint32_t settled;    // diagnostic: columns whose median and MAD both came out of their brackets
+    uint32_t pad[2];
+    uint32_t valid[kMaxMetrics];   // the output arrays hold a previous result of this call site for metric m
+    float hw[2][kMaxMetrics];
+    // every entry of metric m is written only by the leader of the cluster that handles column m, after all
+    // CTAs of that cluster have read it: the CTAs of a cluster always decide alike
+};
 // One CTA per (row, metric) column with the column in registers: for a few rows at a time.
 bool xrank_column_supported(int R);
 cudaError_t launch_xrank_column(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st);
@@ -161,6 +174,12 @@ struct NodeArgs {
 };
 cudaError_t launch_node_verdict(const NodeArgs &a, cudaStream_t st);
 
+// State the top-k of consecutive evaluations keeps (zero before first use): the threshold key the
+// previous evaluation left (about three times K ranks lie at or above it), the list counter and
+// ticket of the hinted pass, whether the full pass has to run, and diagnostic counters.
+struct TopkHint {
+    uint32_t valid, tau, count, ticket, need_full, hits, misses, pad;
+};
 // Block-then-grid top-k of dir * wmed[:, primary].
 struct TopkArgs {
     int R, M, K;
@@ -172,6 +191,8 @@ struct TopkArgs {
     int32_t *idx;               // [K] or NULL
     int32_t *idx_keep;          // [K] second copy of the indices (the context's own), or NULL
     float *score;               // [K] or NULL: needs fleet_med / fleet_mad to be final when the kernel runs
+    TopkHint *hint;             // or NULL: state of the hinted pass (evaluations a few steps apart; used when score is NULL)
+    unsigned long long *hcand;  // scratch [1024] of the hinted pass
 };
 int topk_blocks(int R);
 // Records the text guard_last_error(NULL) returns (defined next to the C ABI).

@@ -80,11 +80,12 @@ __device__ void fold_topk(const unsigned long long (&e)[2], int K, unsigned long
 
 __global__ void __launch_bounds__(kTopThreads) topk_kernel(const TopkArgs a, const MetricParams p, const int nblocks) {
     __shared__ unsigned long long list[kTopList];
-    __shared__ unsigned long long run[GUARD_MAX_TOPK];
+    __shared__ unsigned long long run[2 * GUARD_MAX_TOPK];
     __shared__ ColShared sh;
     __shared__ uint32_t s_n;
     __shared__ int is_last;
     const int tid = threadIdx.x, b = blockIdx.x;
+    if (a.hint && __ldcg(&a.hint->need_full) == 0) return;   // the hinted kernel in front has produced the list
     const int pm = p.primary, dirp = p.dir[pm];
     const int per = (a.R + nblocks - 1) / nblocks;
     const int lo = b * per, hi = min(a.R, lo + per);
@@ -118,16 +119,27 @@ __global__ void __launch_bounds__(kTopThreads) topk_kernel(const TopkArgs a, con
         if (!is_last) return;
         __threadfence();
         const int total = nblocks * K;
-        for (int i = tid; i < K; i += blockDim.x) run[i] = 0ull;
+        // with a hint state the fold keeps up to three times K entries: the last of them bounds the next
+        // evaluation's threshold from below (at least that many ranks lie at or above it)
+        const int K2 = a.hint ? min(3 * K, 2 * GUARD_MAX_TOPK) : K;
+        for (int i = tid; i < K2; i += blockDim.x) run[i] = 0ull;
         __syncthreads();
         for (int c0 = 0; c0 < total; c0 += kTopChunk) {
             unsigned long long e[2];
             const int j = c0 + tid;
             e[0] = j < total ? __ldcg(a.cand + j) : 0ull;
-            e[1] = tid < K ? run[tid] : 0ull;
+            e[1] = tid < K2 ? run[tid] : 0ull;
             __syncthreads();
-            fold_topk(e, K, list, run, sh, &s_n);
+            fold_topk(e, K2, list, run, sh, &s_n);
         }
+        if (a.hint && tid == 0) {
+            int last = K2 - 1;
+            while (last > 0 && run[last] == 0ull) --last;
+            a.hint->tau = (uint32_t)(run[last] >> 32);
+            a.hint->valid = run[last] != 0ull ? 1u : 0u;
+        }
+    } else if (a.hint && tid == 0) {
+        a.hint->valid = 0u;
     }
     // scores only where the caller asked for them here (then the fleet statistics are final already)
     const float B = a.score ? a.fleet_med[pm] : 0.0f;
@@ -144,6 +156,76 @@ __global__ void __launch_bounds__(kTopThreads) topk_kernel(const TopkArgs a, con
     }
 }
 
+
+// Hinted pass (evaluations that follow one another closely: the set of slowest ranks hardly changes): every
+// CTA appends the entries at or above the threshold the previous evaluation left (about three times K of
+// them) to one global list; the CTA that takes the last ticket sorts the list, takes the K best and leaves the
+// next threshold.  Fewer than K entries, or more than the list holds, leaves the evaluation to topk_kernel,
+// which is launched right behind and returns at once otherwise.
+__global__ void __launch_bounds__(kTopThreads) topk_hint_kernel(const TopkArgs a, const MetricParams p, const int nblocks) {
+    __shared__ unsigned long long list[kTopChunk];
+    __shared__ int is_last;
+    TopkHint *h = a.hint;
+    const int tid = threadIdx.x, b = blockIdx.x, lane = lane_id();
+    if (!h->valid) {   // nobody writes the state in a launch that starts like this: every CTA sees the same
+        if (b == 0 && tid == 0) { h->need_full = 1u; h->misses += 1u; }
+        return;
+    }
+    const uint32_t tau = h->tau;
+    const int pm = p.primary, dirp = p.dir[pm];
+    const int K = a.K;
+    for (int r0 = b * kTopThreads; r0 < a.R; r0 += nblocks * kTopThreads) {   // uniform trip count: the ballots below need whole warps
+        const int r = r0 + tid;
+        unsigned long long e = 0ull;
+        bool pass = false;
+        if (r < a.R) {
+            float v = a.wmed[(size_t)r * a.M + pm];
+            if (dirp < 0) v = -v;
+            const uint32_t key = f2key(v);
+            pass = key >= tau;
+            e = ((unsigned long long)key << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)r);
+        }
+        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, pass);
+        if (bal) {
+            uint32_t base = 0;
+            if (lane == __ffs(bal) - 1) base = atomicAdd(&h->count, (uint32_t)__popc(bal));
+            base = __shfl_sync(0xFFFFFFFFu, base, __ffs(bal) - 1);
+            const uint32_t pos = base + __popc(bal & ((1u << lane) - 1u));
+            if (pass && pos < (uint32_t)kTopChunk) a.hcand[pos] = e;
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) is_last = (atomicAdd(&h->ticket, 1u) == (unsigned)nblocks - 1u) ? 1 : 0;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int n = (int)__ldcg(&h->count);
+    const bool ok = n >= K && n <= kTopChunk;
+    if (ok) {
+        int n2 = 2;
+        while (n2 < n) n2 <<= 1;
+        for (int i = tid; i < n2; i += blockDim.x) list[i] = i < n ? __ldcg(a.hcand + i) : 0ull;
+        bitonic_desc(list, n2);
+        for (int i = tid; i < K; i += blockDim.x) {
+            const int r = (int)(0xFFFFFFFFu - (uint32_t)(list[i] & 0xFFFFFFFFull));
+            if (a.idx) a.idx[i] = r;
+            if (a.idx_keep) a.idx_keep[i] = r;
+        }
+    }
+    if (tid == 0) {
+        h->count = 0u;
+        h->ticket = 0u;
+        h->need_full = ok ? 0u : 1u;
+        if (ok) {
+            h->tau = (uint32_t)(list[min(n, 3 * K) - 1] >> 32);
+            h->hits += 1u;
+        } else {
+            h->misses += 1u;
+        }
+    }
+}
+
 }  // namespace
 
 int topk_blocks(int R) {
@@ -154,6 +236,12 @@ int topk_blocks(int R) {
 cudaError_t launch_topk(const TopkArgs &a, const MetricParams &p, cudaStream_t st) {
     if (a.K <= 0 || (!a.idx && !a.score && !a.idx_keep)) return cudaSuccess;
     const int nb = topk_blocks(a.R);
+    if (a.hint && !a.score) {
+        const int hb = (a.R + kTopThreads - 1) / kTopThreads;
+        topk_hint_kernel<<<hb < 64 ? hb : 64, kTopThreads, 0, st>>>(a, p, hb < 64 ? hb : 64);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     topk_kernel<<<nb, kTopThreads, 0, st>>>(a, p, nb);
     return cudaGetLastError();
 }

@@ -131,8 +131,35 @@ __global__ void __cluster_dims__(NC, 1, 1) __launch_bounds__(kColThreads)
     }
     if (a.check_finite && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(a.status, kStatNonFinite);
 
-    uint32_t v1, v2;
-    bool ok = colc_select_regs<VPT, NC>(key, valid, k1, even, sh, v1, v2);
+    // brackets from the previous result of this call site (read before anything of this row is written)
+    __shared__ HintShared hs;
+    ColHintState *hst = reinterpret_cast<ColHintState *>(a.hint);
+    float hc[2] = {0.0f, 0.0f}, hh[2] = {0.0f, 0.0f};
+    bool hinted[2] = {false, false};
+    if (hst) {
+        hint_clear(hs);
+        // (every CTA of the cluster reads the same state: only this cluster's own leader writes it, at the end)
+        if (hst->valid[m]) {
+            hc[0] = a.med[col];
+            hc[1] = a.mad[col];
+            // no tuned width yet: one standard error of a sample median of normal data is 1.25 x 1.4826 MAD / sqrt(R);
+            // five of them for the median, three for the MAD (whose neighbourhood is 1.6 times denser)
+            const float se = hc[1] * rsqrtf((float)R);
+            hh[0] = hst->hw[0][m];
+            hh[1] = hst->hw[1][m];
+            if (hh[0] == 0.0f) hh[0] = 9.0f * se;
+            if (hh[1] == 0.0f) hh[1] = 5.5f * se;
+#pragma unroll
+            for (int ph = 0; ph < 2; ++ph) hinted[ph] = hh[ph] >= 0.0f && hc[ph] - hh[ph] <= hc[ph] + hh[ph] && fabsf(hc[ph]) + hh[ph] < 3.0e38f;
+        }
+        __syncthreads();
+    }
+    uint32_t v1, v2, nin[2] = {0u, 0u};
+    int side[2] = {0, 0};
+    bool hit[2] = {false, false};
+    bool ok = true;
+    if (hinted[0]) hit[0] = colc_select_hinted<VPT, NC>(key, valid, k1, even, f2key(hc[0] - hh[0]), f2key(hc[0] + hh[0]), hs, 0, v1, v2, nin[0], side[0]);
+    if (!hit[0]) ok = colc_select_regs<VPT, NC>(key, valid, k1, even, sh, v1, v2);
     const float med = median_from_keys(v1, v2, even);
     if (a.cut) {
         uint32_t c1, c2;
@@ -141,7 +168,8 @@ __global__ void __cluster_dims__(NC, 1, 1) __launch_bounds__(kColThreads)
     }
 #pragma unroll
     for (int i = 0; i < VPT; ++i) key[i] = f2key(fabsf(__fsub_rn(x[i], med)));
-    ok = colc_select_regs<VPT, NC>(key, valid, k1, even, sh, v1, v2) && ok;
+    if (hinted[1]) hit[1] = colc_select_hinted<VPT, NC>(key, valid, k1, even, f2key(fmaxf(hc[1] - hh[1], 0.0f)), f2key(hc[1] + hh[1]), hs, 1, v1, v2, nin[1], side[1]);
+    if (!hit[1]) ok = colc_select_regs<VPT, NC>(key, valid, k1, even, sh, v1, v2) && ok;
     const float mad = median_from_keys(v1, v2, even);
     if (tid == 0 && crank == 0) {
         if (!ok) atomicOr(a.status, kStatInternal);
@@ -149,6 +177,24 @@ __global__ void __cluster_dims__(NC, 1, 1) __launch_bounds__(kColThreads)
         a.mad[col] = mad;
         if (a.med_user) a.med_user[col] = med;
         if (a.mad_user) a.mad_user[col] = mad;
+        if (hst) {
+            // keep about 4.5 sqrt(R) keys inside a bracket (four to five standard errors of a sample median to
+            // either side for normal data); a bracket that missed is widened; one whose bins held more keys
+            // than the gather lists (ties) rests for sixteen rows (negative values count up to zero)
+            const float target = fminf(fmaxf(4.5f * sqrtf((float)R), 64.0f), 1500.0f);
+#pragma unroll
+            for (int ph = 0; ph < 2; ++ph) {
+                float h = hst->hw[ph][m];
+                if (hit[ph]) h = hh[ph] * fminf(fmaxf(target / (float)max(nin[ph], 1u), 0.7f), 1.5f);
+                else if (hinted[ph]) h = side[ph] != 0 ? hh[ph] * 4.0f : -16.0f;
+                else if (h < 0.0f) h = fminf(h + 1.0f, 0.0f);
+                else h = 0.0f;
+                hst->hw[ph][m] = h;
+            }
+            hst->valid[m] = 1;
+            if (m == 0) atomicAdd(&hst->rows, 1u);
+            if (hit[0] && hit[1]) atomicAdd(&hst->settled, 1u);
+        }
     }
     if (a.mask_base) {
         // the mask row was zeroed before the launch; the CTAs of a row OR their bits in
@@ -176,6 +222,7 @@ __global__ void __cluster_dims__(NC, 1, 1) __launch_bounds__(kColThreads)
             }
         }
     }
+    if (hst) cl_sync();   // the hinted selection reads the other CTAs' lists last: none may exit before all have
 }
 
 constexpr int kColCluster = 4;
@@ -201,7 +248,8 @@ cudaError_t launch_vpt(const XrankArgs &a, const MetricParams &p, int S, cudaStr
 bool xrank_column_supported(int R) { return R >= 1024 && R <= 32 * kColThreads; }
 
 // Zeroes the exceedance rows of the S steps (at most two memsets when the span wraps), then
-// runs one CTA per column.
+// runs one CTA per column (or one cluster per column: the widest columns, and single rows whose call
+// site keeps a bracket from its previous result).
 cudaError_t launch_xrank_column(const XrankArgs &a, const MetricParams &p, int S, cudaStream_t st) {
     if (S <= 0) return cudaSuccess;
     if (a.mask_base) {
@@ -217,6 +265,12 @@ cudaError_t launch_xrank_column(const XrankArgs &a, const MetricParams &p, int S
     // measured 45 -> 35 us per launch at 32 768 ranks; at 16 384 ranks the cluster barriers cost more than
     // the shared work saves (node sweep 0.13 -> 0.18 ms), so narrower columns stay with one CTA
     if (vpt > 16) return launch_cluster_vpt<8>(a, p, S, st);
+    // a single row with a bracket from the previous result of its call site: the hinted selection of the cluster
+    // kernel needs two cluster barriers per statistic, which pays from 8 192 ranks on
+    if (a.hint && S == 1 && a.R >= 8192) {
+        const int cv = (a.R + kColCluster * kColThreads - 1) / (kColCluster * kColThreads);
+        return cv <= 2 ? launch_cluster_vpt<2>(a, p, S, st) : launch_cluster_vpt<4>(a, p, S, st);
+    }
     if (vpt <= 4) return launch_vpt<4>(a, p, S, st);
     if (vpt <= 8) return launch_vpt<8>(a, p, S, st);
     if (vpt <= 16) return launch_vpt<16>(a, p, S, st);

@@ -101,6 +101,10 @@ def lib():
         L.guard_set_sliding.argtypes = [vp, C.c_int]
         L.guard_sliding_rebuilds.restype = C.c_int64
         L.guard_sliding_rebuilds.argtypes = [vp, vp]
+        L.guard_set_row_hints.restype = C.c_int
+        L.guard_set_row_hints.argtypes = [vp, C.c_int]
+        L.guard_row_hints.restype = C.c_int
+        L.guard_row_hints.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.guard_set_deferred.restype = C.c_int
         L.guard_set_deferred.argtypes = [vp, C.c_int]
         L.guard_join.restype = C.c_int
@@ -123,6 +127,19 @@ def lib():
 
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
+
+
+class _Here:
+    """Stands in for torch.cuda.device(...) when the wanted device is already current."""
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        return False
+
+
+_HERE_CTX = _Here()
 
 
 def _ptr(t: Optional[torch.Tensor], dtype=None, numel: Optional[int] = None) -> Optional[int]:
@@ -159,6 +176,9 @@ def workspace_bytes(ranks: int, metrics: int, W: int, capacity: int, topk: int) 
     return int(lib().guard_workspace_bytes(ranks, metrics, W, capacity, topk))
 
 
+_OUT_NAMES = ("wmed", "fleet_med", "fleet_mad", "scores", "counts", "mask", "flags", "tier", "topk_idx", "topk_score")
+
+
 class Guard:
     """Online scorer: `ingest` blocks of steps, `score` the current window."""
 
@@ -170,6 +190,9 @@ class Guard:
         self.ranks_per_node = ranks_per_node
         self.C = capacity if capacity is not None else W
         self.device = torch.device(device)
+        self._devidx = self.device.index if self.device.index is not None else torch.cuda.current_device()
+        self._views = {}        # ring views handed out by ring_reserve, by (byte offset, steps)
+        self._out_cache = None  # (dict, tensors, marshalled pointers) of the last score() outputs
         self._h = C.c_void_p()
         self._params = _Params(metrics, dir, thr, floor_rel, floor_abs, primary, min_signals, n_consec,
                                ranks_per_node, tier_moderate, tier_severe)
@@ -179,7 +202,7 @@ class Guard:
         if workspace is None:
             workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
         self.workspace = workspace
-        with torch.cuda.device(self.device):
+        with self._dev():
             rc = lib().guard_create(C.byref(self._h), ranks, metrics, W, k, C.byref(self._params.struct), self.C, topk,
                                     _ptr(workspace, torch.uint8), workspace.numel(), _stream())
         if rc != GUARD_OK:
@@ -196,6 +219,10 @@ class Guard:
         except Exception:
             pass
 
+    def _dev(self):
+        """Context that makes the context's device current (nothing to do when it already is)."""
+        return _HERE_CTX if torch.cuda.current_device() == self._devidx else torch.cuda.device(self.device)
+
     def _check(self, rc: int):
         if rc != GUARD_OK:
             raise GuardError(rc, lib().guard_last_error(self._h).decode())
@@ -210,7 +237,7 @@ class Guard:
 
     def fallback_steps(self) -> int:
         """Rows the fast cross-rank path handed to the direct selection (synchronises)."""
-        with torch.cuda.device(self.device):
+        with self._dev():
             n = int(lib().guard_fallback_steps(self._h, _stream()))
         if n < 0:
             self._check(n)
@@ -219,7 +246,7 @@ class Guard:
     def fallback_reasons(self):
         """Counts of the events that send rows to the direct selection (synchronises)."""
         out = (C.c_uint32 * 6)()
-        with torch.cuda.device(self.device):
+        with self._dev():
             self._check(lib().guard_fallback_reasons(self._h, out, _stream()))
         names = ("cta_list", "step_list", "deferred_list", "median_miss", "select", "mad_miss")
         return dict(zip(names, [int(v) for v in out]))
@@ -227,7 +254,7 @@ class Guard:
     def window_fallbacks(self):
         """Series the thread-per-series window kernel handed to its whole-warp fallback (synchronises)."""
         out = (C.c_uint32 * 6)()
-        with torch.cuda.device(self.device):
+        with self._dev():
             self._check(lib().guard_window_fallbacks(self._h, out, _stream()))
         names = ("total", "no_interval", "overflow", "below", "above", "no_convergence")
         return dict(zip(names, [int(v) for v in out]))
@@ -242,11 +269,23 @@ class Guard:
 
     def sliding_rebuilds(self) -> int:
         """Series the sliding evaluations rebuilt from their whole window (synchronises)."""
-        with torch.cuda.device(self.device):
+        with self._dev():
             n = int(lib().guard_sliding_rebuilds(self._h, _stream()))
         if n < 0:
             self._check(n)
         return n
+
+    def set_row_hints(self, on: bool) -> None:
+        """Single rows of wide fleets bracketed by the call site's previous result (default on)."""
+        self._check(lib().guard_set_row_hints(self._h, 1 if on else 0))
+
+    def row_hints(self):
+        """Single rows seen and columns settled inside their brackets, per call site (synchronises)."""
+        out = (C.c_uint32 * 6)()
+        with self._dev():
+            self._check(lib().guard_row_hints(self._h, out, _stream()))
+        names = ("ingest_rows", "ingest_settled", "baseline_rows", "baseline_settled", "topk_hinted", "topk_full")
+        return dict(zip(names, [int(v) for v in out]))
 
     def set_deferred(self, on: bool) -> None:
         """Deferred evaluations: score() does not make the current stream wait for its results; they
@@ -255,7 +294,7 @@ class Guard:
 
     def join(self) -> None:
         """Makes the current stream wait for the pending deferred evaluation, if any."""
-        with torch.cuda.device(self.device):
+        with self._dev():
             self._check(lib().guard_join(self._h, _stream()))
 
     def profile_enable(self, on=True) -> None:
@@ -273,15 +312,20 @@ class Guard:
         p = C.c_void_p()
         self._check(lib().guard_ring_reserve(self._h, steps, C.byref(p)))
         off = p.value - self.workspace.data_ptr()
-        nbytes = steps * self.R * self.M * 4
-        return self.workspace[off:off + nbytes].view(torch.float32).view(steps, self.R, self.M)
+        view = self._views.get((off, steps))
+        if view is None:
+            nbytes = steps * self.R * self.M * 4
+            view = self.workspace[off:off + nbytes].view(torch.float32).view(steps, self.R, self.M)
+            if len(self._views) < 4096:
+                self._views[(off, steps)] = view
+        return view
 
     def ingest(self, block: torch.Tensor, step_med: Optional[torch.Tensor] = None,
                step_mad: Optional[torch.Tensor] = None) -> None:
         if block.dim() != 3 or block.shape[1] != self.R or block.shape[2] != self.M:
             raise ValueError("block must be [B, %d, %d]" % (self.R, self.M))
         B = block.shape[0]
-        with torch.cuda.device(self.device):
+        with self._dev():
             self._check(lib().guard_ingest(self._h, _ptr(block, torch.float32), B,
                                            _ptr(step_med, torch.float32, B * self.M),
                                            _ptr(step_mad, torch.float32, B * self.M), _stream()))
@@ -307,14 +351,22 @@ class Guard:
             out = self.alloc_outputs()
         g = out.get
         R, M, K = self.R, self.M, self.K
-        with torch.cuda.device(self.device):
-            self._check(lib().guard_score(
-                self._h, _ptr(g("wmed"), torch.float32, R * M), _ptr(g("fleet_med"), torch.float32, M),
-                _ptr(g("fleet_mad"), torch.float32, M), _ptr(g("scores"), torch.float32, R * M),
-                _ptr(g("counts"), torch.uint16, R * M), _ptr(g("mask"), torch.uint32, R),
-                _ptr(g("flags"), torch.uint8, R), _ptr(g("tier"), torch.uint8, R),
-                _ptr(g("topk_idx"), torch.int32, K) if K else None,
-                _ptr(g("topk_score"), torch.float32, K) if K else None, _stream()))
+        # the same output tensors as last time (a monitor scores into the same buffers every step): reuse
+        # the checked pointers
+        cached = self._out_cache
+        if cached is not None and cached[0] is out and all(
+                g(n) is t and (t is None or t.data_ptr() == q) for (n, t), q in zip(cached[1], cached[2])):
+            ptrs = cached[2]
+        else:
+            ptrs = (_ptr(g("wmed"), torch.float32, R * M), _ptr(g("fleet_med"), torch.float32, M),
+                    _ptr(g("fleet_mad"), torch.float32, M), _ptr(g("scores"), torch.float32, R * M),
+                    _ptr(g("counts"), torch.uint16, R * M), _ptr(g("mask"), torch.uint32, R),
+                    _ptr(g("flags"), torch.uint8, R), _ptr(g("tier"), torch.uint8, R),
+                    _ptr(g("topk_idx"), torch.int32, K) if K else None,
+                    _ptr(g("topk_score"), torch.float32, K) if K else None)
+            self._out_cache = (out, tuple((n, g(n)) for n in _OUT_NAMES), ptrs)
+        with self._dev():
+            self._check(lib().guard_score(self._h, *ptrs, _stream()))
         return out
 
     def node_verdict(self, out: Optional[Dict[str, Optional[torch.Tensor]]] = None) -> Dict[str, Optional[torch.Tensor]]:
@@ -325,7 +377,7 @@ class Guard:
                    "node_tier": torch.empty(N, dtype=torch.uint8, device=self.device),
                    "node_stall": torch.empty(N, dtype=torch.uint16, device=self.device)}
         g = out.get
-        with torch.cuda.device(self.device):
+        with self._dev():
             self._check(lib().guard_node_verdict(self._h, _ptr(g("node_flag"), torch.uint8, N),
                                                  _ptr(g("node_tier"), torch.uint8, N),
                                                  _ptr(g("node_stall"), torch.uint16, N), _stream()))
@@ -338,13 +390,13 @@ class Guard:
         """Copies the context's state into `state` (a uint8 CUDA tensor of state_bytes(), allocated if None)."""
         if state is None:
             state = torch.empty(self.state_bytes(), dtype=torch.uint8, device=self.device)
-        with torch.cuda.device(self.device):
+        with self._dev():
             self._check(lib().guard_state_export(self._h, _ptr(state, torch.uint8), state.numel(), _stream()))
         return state
 
     def state_import(self, state: torch.Tensor) -> None:
         """Loads a state written by state_export of a context of the same sizes (synchronises)."""
-        with torch.cuda.device(self.device):
+        with self._dev():
             self._check(lib().guard_state_import(self._h, _ptr(state, torch.uint8), state.numel(), _stream()))
 
     def debug_set_wait_limit(self, cycles: int) -> None:
@@ -352,13 +404,13 @@ class Guard:
 
     def sync_status(self) -> int:
         """Synchronises the current stream; raises GuardError on a sticky device error."""
-        with torch.cuda.device(self.device):
+        with self._dev():
             rc = lib().guard_sync_status(self._h, _stream())
         self._check(rc)
         return rc
 
     def reset(self) -> None:
-        with torch.cuda.device(self.device):
+        with self._dev():
             self._check(lib().guard_reset(self._h, _stream()))
 
 
