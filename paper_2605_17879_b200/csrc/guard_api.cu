@@ -25,7 +25,7 @@ constexpr int kIngestStreams = GUARD_INGEST_STREAMS;   // internal streams the c
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t status, consec, lastflag, lasttier, topk_idx, topk_hint, ticket, fleet, xr_small, xr_grid, wmed, stepstat, topk_cand, wspread, wcentre, kcnt, inc_lo, inc_hi, inc_cnt, inc_val, xr_big, xr_big_stride, mask, ring, total;
+    size_t status, consec, lastflag, lasttier, topk_idx, topk_hint, ticket, fleet, xr_small, xr_grid, inc_rbc, wmed, wmed_stride, stepstat, topk_cand, wspread, wcentre, kcnt, inc_lo, inc_hi, inc_cnt, inc_val, inc_rbl, xr_big, xr_big_stride, mask, ring, total;
     int xr_steps;   // steps per launch of the multi-kernel bracketed cross-rank path (0: not used)
     int xr_cluster; // the cluster-per-step cross-rank path applies
     int xr_split;   // the six-kernel split cross-rank path applies
@@ -42,7 +42,7 @@ Layout make_layout(int R, int M, int C, int K) {
     L.consec = off;    off = align_up(off + (size_t)R);
     L.lastflag = off;  off = align_up(off + (size_t)R);
     L.lasttier = off;  off = align_up(off + (size_t)R);
-    L.topk_idx = off;  off = align_up(off + (size_t)(K > 0 ? K : 1) * sizeof(int32_t));
+    L.topk_idx = off;  off = align_up(off + 2 * align_up((size_t)(K > 0 ? K : 1) * sizeof(int32_t)));
     L.topk_hint = off; off = align_up(off + 256 + 1024 * sizeof(unsigned long long));   // TopkHint, then the hinted pass's list
     L.xr_split = xrank_split_supported(R, M) ? 1 : 0;
     L.xr_cluster = (!L.xr_split && xrank_cluster_supported(R, M)) ? 1 : 0;
@@ -50,7 +50,12 @@ Layout make_layout(int R, int M, int C, int K) {
     L.xr_small = off;  off = align_up(off + (L.xr_steps ? xrank_scratch_small_bytes(M, L.xr_steps) : 0));
     L.xr_gridp = (xrank_column_supported(R) && R >= 8192) ? 1 : 0;
     L.xr_grid = off;   off = align_up(off + 2 * align_up(sizeof(ColHintState)));
+    L.inc_rbc = off;   off = align_up(off + 64);   // rebuild list counter and ticket (zero before first use)
+    // the windowed medians and the kept top-k indices exist twice: consecutive evaluations alternate, so that a
+    // deferred evaluation's tail may still read its medians while the next evaluation's window kernels write theirs
     L.wmed = off;      off = align_up(off + (size_t)R * M * sizeof(float));
+    L.wmed_stride = off - L.wmed;
+    off = align_up(off + (size_t)R * M * sizeof(float));
     L.stepstat = off;  off = align_up(off + 2 * (size_t)C * M * sizeof(float));
     L.topk_cand = off; off = align_up(off + (size_t)topk_blocks(R) * (K > 0 ? K : 1) * sizeof(unsigned long long));
     L.wspread = off;   off = align_up(off + (size_t)R * M * sizeof(float));
@@ -61,6 +66,7 @@ Layout make_layout(int R, int M, int C, int K) {
     L.inc_hi = off;    off = align_up(off + window_inc_bytes(R * M));
     L.inc_cnt = off;   off = align_up(off + window_inc_bytes(R * M));
     L.inc_val = off;   off = align_up(off + (size_t)kIncSlots * window_inc_bytes(R * M));
+    L.inc_rbl = off;   off = align_up(off + window_inc_bytes(R * M));   // series a sliding launch has to rebuild
     L.xr_big = off;    off = align_up(off + (L.xr_split ? xrank_split_scratch_bytes(R, M, C < kSplitMaxSteps ? C : kSplitMaxSteps)
                                              : L.xr_steps ? xrank_scratch_big_bytes(R, M, L.xr_steps) : 0));
     // in deferred mode consecutive blocks run their cross-rank kernels on streams of their own
@@ -191,7 +197,12 @@ struct guard_ctx {
     int xs_next = 0;
     int scratch_sel = 0;                // which split scratch the next launch uses
     cudaStream_t tail = nullptr;
-    cudaEvent_t ev_x = nullptr, ev_w = nullptr, ev_e = nullptr;
+    cudaEvent_t ev_x = nullptr, ev_w = nullptr;
+    // end of the deferred evaluations, by parity of the evaluation count: up to two may be in flight (the tail of
+    // one beside the window medians of the next); each keeps its window for the ring protection
+    cudaEvent_t ev_e[2] = {nullptr, nullptr};
+    struct Inflight { bool on = false; long long seen = 0; int n = 0; } infl[2];
+    int last_q = 0;                   // parity of the pending evaluation
     bool ensure_xs() {
         if (xs[0]) return true;
         if (!ensure_tail()) return false;
@@ -218,12 +229,17 @@ struct guard_ctx {
     // Work whose end event has already completed (a host-side query, no waiting) reads nothing any more.
     long long protected_steps(int need) {
         long long first = seen;
-        if (pending && pending_seen - pending_n < first) first = pending_seen - pending_n;
+        for (int q = 0; q < 2; ++q)
+            if (infl[q].on && infl[q].seen - infl[q].n < first) first = infl[q].seen - infl[q].n;
         for (int k = 0; k < kIngestStreams; ++k)
             if (xs_busy[k] && xs_first[k] < first) first = xs_first[k];
         if (need + (seen - first) <= C) return seen - first;   // no conflict even if all of it is still running: nothing to query
         first = seen;
-        if (pending && pending_seen - pending_n < first && cudaEventQuery(ev_e) != cudaSuccess) first = pending_seen - pending_n;
+        for (int q = 0; q < 2; ++q)
+            if (infl[q].on) {
+                if (cudaEventQuery(ev_e[q]) == cudaSuccess) { infl[q].on = false; continue; }   // finished: reads nothing any more
+                if (infl[q].seen - infl[q].n < first) first = infl[q].seen - infl[q].n;
+            }
         for (int k = 0; k < kIngestStreams; ++k)
             if (xs_busy[k] && xs_first[k] < first) {
                 if (cudaEventQuery(ev_xs[k]) == cudaSuccess) { xs_busy[k] = false; continue; }   // finished: nothing left to wait for
@@ -240,7 +256,8 @@ struct guard_ctx {
         if (cudaStreamCreateWithPriority(&tail, cudaStreamNonBlocking, GUARD_EVAL_PRIO ? prio_hi : 0) != cudaSuccess) { tail = nullptr; return false; }
         if (cudaEventCreateWithFlags(&ev_x, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&ev_w, cudaEventDisableTiming) != cudaSuccess ||
-            cudaEventCreateWithFlags(&ev_e, cudaEventDisableTiming) != cudaSuccess) {
+            cudaEventCreateWithFlags(&ev_e[0], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ev_e[1], cudaEventDisableTiming) != cudaSuccess) {
             cudaStreamDestroy(tail);
             tail = nullptr;
             return false;
@@ -250,9 +267,9 @@ struct guard_ctx {
     // Makes `st` wait for the pending evaluation, if any.
     cudaError_t join(cudaStream_t st) {
         cudaError_t e = cudaSuccess;
-        if (pending) {
-            e = cudaStreamWaitEvent(st, ev_e, 0);
-            if (e == cudaSuccess) pending = false;
+        if (pending) {   // the tail stream runs the evaluations in order: the latest one's end covers the one before
+            e = cudaStreamWaitEvent(st, ev_e[last_q], 0);
+            if (e == cudaSuccess) { pending = false; infl[0].on = false; infl[1].on = false; }
         }
         return e;
     }
@@ -277,8 +294,10 @@ struct guard_ctx {
     uint8_t *consec() const { return (uint8_t *)(ws + L.consec); }
     uint8_t *lastflag() const { return (uint8_t *)(ws + L.lastflag); }
     uint8_t *lasttier() const { return (uint8_t *)(ws + L.lasttier); }
-    int32_t *topk_idx() const { return (int32_t *)(ws + L.topk_idx); }
-    float *wmed() const { return (float *)(ws + L.wmed); }
+    int32_t *topk_idx(int q) const { return (int32_t *)(ws + L.topk_idx + (size_t)q * align_up((size_t)(K > 0 ? K : 1) * sizeof(int32_t))); }
+    float *wmed(int q) const { return (float *)(ws + L.wmed + (size_t)q * L.wmed_stride); }
+    int eval_q() const { return (int)(evals & 1); }        // buffers of the evaluation about to be made
+    int prev_q() const { return (int)((evals + 1) & 1); }  // ... and of the one made last
     float *step_med() const { return (float *)(ws + L.stepstat); }
     float *step_mad() const { return step_med() + (size_t)C * M; }
     unsigned long long *topk_cand() const { return (unsigned long long *)(ws + L.topk_cand); }
@@ -499,7 +518,9 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     w.last_slot = last;
     w.n = n;
     w.series = (int)row;
-    w.wmed = c->wmed();
+    const int q = c->eval_q();
+    w.wmed = c->wmed(q);
+    w.wmed_prev = c->wmed(q ^ 1);
     w.wmed_user = d_wmed;
     w.use_hint = c->hints_ready ? 1 : 0;
     w.spread = (float *)(c->ws + c->L.wspread);
@@ -521,6 +542,8 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         ia.cnt = (uint32_t *)(c->ws + c->L.inc_cnt);
         ia.val = (float *)(c->ws + c->L.inc_val);
         ia.rebuilds = c->status() + 14;
+        ia.rb_list = (uint32_t *)(c->ws + c->L.inc_rbl);
+        ia.rb_count = (uint32_t *)(c->ws + c->L.inc_rbc);
         const long long p1 = c->inc_seen, p0 = p1 - c->inc_n, q1 = c->seen, q0 = q1 - n;
         // the windows overlap, few steps entered / left, and the steps that left are still in the ring
         if (p1 >= 0 && q0 < p1 && q1 - p1 <= kIncMaxNew && q0 - p0 <= kIncMaxNew && q1 - p0 <= c->C) {
@@ -565,7 +588,8 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
             if (e != cudaSuccess) return c->cuda_fail(e, "event record");
         }
         e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
-        if (e == cudaSuccess && had_pending) e = cudaStreamWaitEvent(c->side, c->ev_e, 0);
+        // the evaluation before the previous one used the same buffers: its tail must have read them
+        if (e == cudaSuccess && c->infl[q].on) e = cudaStreamWaitEvent(c->side, c->ev_e[q], 0);
         if (e == cudaSuccess) e = c->window(w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_x, st);
@@ -595,13 +619,13 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         t.R = c->R;
         t.M = c->M;
         t.K = c->K;
-        t.wmed = c->wmed();
+        t.wmed = c->wmed(q);
         t.fleet_med = c->fleet_med();
         t.fleet_mad = c->fleet_mad();
         t.cand = c->topk_cand();
         t.ticket = c->ticket();
         t.idx = d_topk_idx;
-        t.idx_keep = c->topk_idx();
+        t.idx_keep = c->topk_idx(q);
         t.score = nullptr;
         // evaluations a few steps apart: the previous evaluation's threshold pre-selects the candidates
         if (c->sliding && gap <= kIncMaxNew) {
@@ -624,7 +648,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     }
 
     XrankArgs x{};
-    x.base = c->wmed();
+    x.base = c->wmed(q);
     x.row_stride = (long long)row;
     x.first_slot = 0;
     x.capacity = 1;
@@ -641,7 +665,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     ScoreArgs s{};
     s.R = c->R;
     s.M = c->M;
-    s.wmed = c->wmed();
+    s.wmed = c->wmed(q);
     s.fleet_med = c->fleet_med();
     s.fleet_mad = c->fleet_mad();
     s.mask_base = c->mask();
@@ -670,7 +694,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         c->cnt_seen = c->seen;
         c->cnt_n = n;
     }
-    s.topk_idx = want_topk ? c->topk_idx() : nullptr;
+    s.topk_idx = want_topk ? c->topk_idx(q) : nullptr;
     s.topk_score = want_topk ? d_topk_score : nullptr;
     s.K = c->K;
     if (topk_side) {
@@ -680,14 +704,18 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     e = launch_score_flag(s, c->p, ts);
     if (e != cudaSuccess) return c->cuda_fail(e, "score_flag launch");
     c->evals += 1;
-    c->launches += 1 + window_launch_count(w);
+    c->launches += 1 + window_launch_count(w) + (use_inc ? 1 : 0);
     if (defer) {
-        e = cudaEventRecord(c->ev_e, c->tail);
+        e = cudaEventRecord(c->ev_e[q], c->tail);
         if (e != cudaSuccess) return c->cuda_fail(e, "event record");
         c->pending = true;
         // the sliding updates also read the steps that just left the window
         c->pending_n = n + ((use_inc ? ia.leaving : 0) > s.leaving ? (use_inc ? ia.leaving : 0) : s.leaving);
         c->pending_seen = c->seen;
+        c->last_q = q;
+        c->infl[q].on = true;
+        c->infl[q].seen = c->seen;
+        c->infl[q].n = c->pending_n;
     }
     return GUARD_OK;
 }
@@ -797,7 +825,7 @@ int guard_node_verdict(guard_ctx *c, uint8_t *d_node_flag, uint8_t *d_node_tier,
     const bool on_tail = c->pending && c->tail;
     cudaStream_t ts = on_tail ? c->tail : (cudaStream_t)stream;
     cudaError_t e = launch_node_verdict(a, ts);
-    if (e == cudaSuccess && on_tail) e = cudaEventRecord(c->ev_e, c->tail);
+    if (e == cudaSuccess && on_tail) e = cudaEventRecord(c->ev_e[c->last_q], c->tail);
     if (e != cudaSuccess) return c->cuda_fail(e, "node verdict launch");
     c->launches += 1;
     return GUARD_OK;
@@ -884,7 +912,7 @@ int guard_state_export(guard_ctx *c, void *d_state, size_t state_bytes, void *st
     dd(sl.consec, c->consec(), (size_t)c->R);
     dd(sl.lastflag, c->lastflag(), (size_t)c->R);
     dd(sl.lasttier, c->lasttier(), (size_t)c->R);
-    dd(sl.wmed, c->wmed(), RM);
+    dd(sl.wmed, c->wmed(c->prev_q()), RM);   // the medians of the evaluation made last
     dd(sl.wspread, c->ws + c->L.wspread, RM);
     dd(sl.wcentre, c->ws + c->L.wcentre, RM);
     {   // sliding-window state: four arrays, stored back to back
@@ -931,7 +959,7 @@ int guard_state_import(guard_ctx *c, const void *d_state, size_t state_bytes, vo
     dd(c->consec(), sl.consec, (size_t)c->R);
     dd(c->lastflag(), sl.lastflag, (size_t)c->R);
     dd(c->lasttier(), sl.lasttier, (size_t)c->R);
-    dd(c->wmed(), sl.wmed, RM);
+    dd(c->wmed((int)((h.evals + 1) & 1)), sl.wmed, RM);   // where the next evaluation looks for the previous medians
     dd(c->ws + c->L.wspread, sl.wspread, RM);
     dd(c->ws + c->L.wcentre, sl.wcentre, RM);
     {
@@ -1126,7 +1154,8 @@ void guard_destroy(guard_ctx *c) {
             cudaStreamDestroy(c->tail);
             cudaEventDestroy(c->ev_x);
             cudaEventDestroy(c->ev_w);
-            cudaEventDestroy(c->ev_e);
+            cudaEventDestroy(c->ev_e[0]);
+            cudaEventDestroy(c->ev_e[1]);
         }
         if (c->side) {
             cudaStreamDestroy(c->side);

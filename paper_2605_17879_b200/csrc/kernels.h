@@ -94,7 +94,8 @@ struct WindowArgs {
     int n;                  // window length in steps
     int series;             // R * M
     float *wmed;            // [series] (never NULL)
-    int use_hint;           // wmed holds the previous evaluation's medians: use them as first pivots
+    const float *wmed_prev; // [series] the previous evaluation's medians (another buffer than wmed), or NULL
+    int use_hint;           // wmed_prev holds the previous evaluation's medians: use them as first pivots
     float *wmed_user;       // or NULL
     float *spread;          // [series] tuned half-width of the thread path's interval (state), or NULL
     float *centre;          // [series] smoothed median: the centre of the thread path's interval (state), or NULL
@@ -113,16 +114,18 @@ cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st);
 // median is then a rank among those.  A series whose median leaves the interval (or whose interval
 // overflows) rebuilds its state from the whole window.
 constexpr int kIncSlots = 40;     // values a series' interval can hold
-constexpr int kIncHalf = 12;      // ranks the interval reaches beyond the middle ranks when it is (re)built
+constexpr int kIncHalf = 8;      // ranks the interval reaches beyond the middle ranks when it is (re)built
 constexpr int kIncMaxNew = 8;     // most steps between two evaluations the sliding update is used for
 struct IncArgs {
     float *lo, *hi;               // [series] interval ends (inclusive)
     uint32_t *cnt;                // [series] bit 31: state valid; bits 16..23: values inside; bits 0..15: values below lo
-    float *val;                   // [kIncSlots][series] the values inside the interval, ascending (total order)
+    float *val;                   // [series][kIncSlots] the values inside the interval, ascending (total order)
     int rebuild_all;              // ignore the stored state: every series rebuilds
     int entering;                 // steps that entered the window since the state was current (the newest ones)
     int leaving;                  // steps that left it (those right before the window's oldest step)
     uint32_t *rebuilds;           // diagnostic counter or NULL
+    uint32_t *rb_list;            // [series] scratch: the series this launch has to rebuild
+    uint32_t *rb_count;           // [2] their number and the rebuild kernel's ticket: zero before first use, self-resetting
 };
 size_t window_inc_bytes(int series);   // per array: lo, hi, cnt take series * 4 bytes, val kIncSlots * series * 4
 bool window_inc_supported(const WindowArgs &a);

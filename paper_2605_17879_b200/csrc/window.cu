@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(1024, 2) window_warp_kernel(const WindowArgs a
             }
             lane_sort<VPL>(kv);
             float med = 0.0f;
-            const uint32_t hint = a.use_hint ? f2key(a.wmed[series]) : 0u;   // last evaluation's median
+            const uint32_t hint = (a.use_hint && a.wmed_prev) ? f2key(a.wmed_prev[series]) : 0u;   // last evaluation's median
             const bool ok = warp_median<VPL>(kv, nreal, n, hint, med);
             const float h0 = warp_spread_guess<VPL>(kv, n, med);
             if (lane == 0) {
@@ -477,11 +477,12 @@ cudaError_t launch_thread_path(const WindowArgs &a, cudaStream_t st) {
 // Sliding-window path: evaluations that follow one another by a few steps (streaming: one step)
 // share all but a few steps of their windows, so a series' median moves by a rank or two.  Each
 // series keeps, across evaluations, an interval [lo, hi] around its median, the number of window
-// values below lo, and the handful of values inside the interval (global memory, one array per
-// slot so that a warp's accesses are contiguous).  An evaluation reads only the steps that
-// entered and left the window: a value below lo moves the count, a value inside the interval is
-// inserted into / removed from the series' sorted list (fetched only in that case); the median is
-// then position (middle - count) of the list.  One thread per series.
+// values below lo, and the handful of values inside the interval (global memory, each series' sorted
+// list contiguous).  An evaluation reads only the steps that entered and left the window, one thread
+// per series: a value below lo moves the count; a value inside the interval is inserted into /
+// removed from the series' list by the whole warp (lane j holds list slots j and j + 32: the position
+// comes from a ballot, the shift from one shuffle), series after series; the median is then
+// position (middle - count) of the list.
 // A series whose median has left its interval, whose list is full, or that has no state yet is
 // rebuilt by its whole warp: the lanes fetch the window, sort it (bitonic network over registers
 // and shuffles) and take the median, the interval ends kIncHalf ranks beyond the middle ranks, and
@@ -489,12 +490,14 @@ cudaError_t launch_thread_path(const WindowArgs &a, cudaStream_t st) {
 // ---------------------------------------------------------------------------------------
 constexpr int kIncThreads = 128;
 
-template <int VPL>
-__global__ void __launch_bounds__(kIncThreads) window_inc_kernel(const WindowArgs a, const IncArgs s) {
-    __shared__ float sv[kIncSlots][kIncThreads];   // this thread's listed values: column tid
-    const int tid = threadIdx.x, lane = lane_id();
+// NEW: the most steps that entered / left (1 for an evaluation after every step, else kIncMaxNew).
+template <int NEW>
+__global__ void __launch_bounds__(kIncThreads, 8) window_inc_kernel(const WindowArgs a, const IncArgs s) {
+    static_assert(kIncSlots > 32 && kIncSlots <= 64, "a lane holds list slots lane and lane + 32");
+    __shared__ float sl[kIncThreads / 32][32][kIncSlots];   // per warp: the lists of the series it updates, staged asynchronously
+    const int lane = lane_id(), wid = warp_id();
     const int n = a.n;
-    const int c = blockIdx.x * kIncThreads + tid;
+    const int c = blockIdx.x * kIncThreads + threadIdx.x;
     const bool active = c < a.series;
     const int cc = active ? c : a.series - 1;
     const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;   // slot of the window's oldest step
@@ -505,70 +508,163 @@ __global__ void __launch_bounds__(kIncThreads) window_inc_kernel(const WindowArg
     bool ok = active && (w >> 31) && !s.rebuild_all;
     int cb = (int)(w & 0xFFFFu), nin = (int)((w >> 16) & 0xFFu);
     const float lo = s.lo[cc], hi = s.hi[cc];
-    if (ok) {
-        // The steps that left the window (the ones right before its oldest step) and the steps that entered it
-        // (the newest ones).  A value below lo moves the count; a value inside the interval changes the list,
-        // which is kept sorted and fetched only then (seldom: the interval holds a few percent of the window).
-        bool listed = false, dirty = false;
-        auto fetch_list = [&]() {
-            if (!listed)
-                for (int j = 0; j < nin; ++j) sv[j][tid] = s.val[(size_t)j * a.series + c];
-            listed = true;
-        };
-        for (int i = 0; ok && i < s.leaving; ++i) {
+    // The steps that left the window (the ones right before its oldest step) and the steps that entered it (the
+    // newest ones), all fetched up front.  A value below lo moves the count; a value inside the interval
+    // changes the series' sorted list, which the whole warp then updates (below).
+    float xl[NEW], xe[NEW];
+    uint32_t in_l = 0, in_e = 0;   // which of them lie inside the interval
+#pragma unroll
+    for (int i = 0; i < NEW; ++i) {
+        xl[i] = 0.0f;
+        xe[i] = 0.0f;
+        if (i < s.leaving) {
             int slot = first - s.leaving + i;
             if (slot < 0) slot += a.capacity;
-            const float x = __ldg(a.ring + (size_t)slot * a.row_stride + c);
-            if (x < lo) {
-                --cb;
-            } else if (x <= hi) {
-                fetch_list();
-                int at = -1;
-                for (int j = 0; j < nin; ++j)
-                    if (__float_as_uint(sv[j][tid]) == __float_as_uint(x)) at = j;
-                if (at < 0) { ok = false; break; }      // the books do not balance: rebuild
-                for (int j = at; j + 1 < nin; ++j) sv[j][tid] = sv[j + 1][tid];
-                --nin;
-                dirty = true;
-            }
+            xl[i] = __ldg(a.ring + (size_t)slot * a.row_stride + cc);
         }
-        for (int i = 0; ok && i < s.entering; ++i) {
+        if (i < s.entering) {
             int slot = a.last_slot - (s.entering - 1 - i);
             if (slot < 0) slot += a.capacity;
-            const float x = __ldg(a.ring + (size_t)slot * a.row_stride + c);
-            if (x < lo) {
-                ++cb;
-            } else if (x <= hi) {
-                if (nin >= kIncSlots) { ok = false; break; }
-                fetch_list();
-                const uint32_t kx = f2key(x);
-                int at = nin;                            // behind the listed values whose key is not above x's
-                while (at > 0 && f2key(sv[at - 1][tid]) > kx) { sv[at][tid] = sv[at - 1][tid]; --at; }
-                sv[at][tid] = x;
-                ++nin;
-                dirty = true;
-            }
-        }
-        ok = ok && cb >= 0 && cb <= k1 && k2 < cb + nin;
-        if (ok) {
-            // the list is sorted: the middle ranks of the window are positions k1 - cb and k2 - cb of it
-            const int j1 = k1 - cb, j2 = k2 - cb;
-            const float f1 = listed ? sv[j1][tid] : s.val[(size_t)j1 * a.series + c];
-            const float f2 = listed ? sv[j2][tid] : s.val[(size_t)j2 * a.series + c];
-            const float med = median_from_keys(f2key(f1), f2key(f2), even);
-            a.wmed[c] = med;
-            if (a.wmed_user) a.wmed_user[c] = med;
-            s.cnt[c] = 0x80000000u | ((uint32_t)nin << 16) | (uint32_t)cb;
-            if (dirty)
-                for (int j = 0; j < nin; ++j) s.val[(size_t)j * a.series + c] = sv[j][tid];
+            xe[i] = __ldg(a.ring + (size_t)slot * a.row_stride + cc);
         }
     }
-    // ---- series without a usable state: the whole warp rebuilds them one by one ------------------
-    unsigned todo = __ballot_sync(0xFFFFFFFFu, active && !ok);
-    while (todo) {
-        const int src = __ffs(todo) - 1;
-        todo &= todo - 1;
-        const int series = __shfl_sync(0xFFFFFFFFu, c, src);
+#pragma unroll
+    for (int i = 0; i < NEW; ++i) {
+        if (i < s.leaving) {
+            if (xl[i] < lo) --cb;
+            else if (xl[i] <= hi) in_l |= 1u << i;
+        }
+        if (i < s.entering) {
+            if (xe[i] < lo) ++cb;
+            else if (xe[i] <= hi) in_e |= 1u << i;
+        }
+    }
+    // ---- list updates, one series at a time by the whole warp: lane j holds list slots j and j + 32 ----
+    float f1 = 0.0f, f2 = 0.0f;
+    bool have = false;             // f1 / f2 hold the list values at the middle ranks
+    unsigned upd = __ballot_sync(0xFFFFFFFFu, ok && (in_l | in_e) != 0u);
+    {   // all lists this warp needs are fetched at once (asynchronous copies into shared memory: one round trip)
+        unsigned m = upd;
+        int k = 0;
+        while (m) {
+            const int src = __ffs(m) - 1;
+            m &= m - 1;
+            const int cs = __shfl_sync(0xFFFFFFFFu, c, src);
+            const int ns = __shfl_sync(0xFFFFFFFFu, nin, src);
+            const float *g = s.val + (size_t)cs * kIncSlots;   // a series' list is contiguous
+            if (lane < ns) cp_async4(&sl[wid][k][lane], g + lane);
+            if (lane + 32 < ns) cp_async4(&sl[wid][k][lane + 32], g + lane + 32);
+            ++k;
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncwarp();
+    }
+    int kk = 0;
+    while (upd) {
+        const int src = __ffs(upd) - 1;
+        upd &= upd - 1;
+        const int cs = __shfl_sync(0xFFFFFFFFu, c, src);
+        int ns = __shfl_sync(0xFFFFFFFFu, nin, src);
+        const uint32_t ml = __shfl_sync(0xFFFFFFFFu, in_l, src), me = __shfl_sync(0xFFFFFFFFu, in_e, src);
+        const size_t lbase = (size_t)cs * kIncSlots;
+        const float v0s = sl[wid][kk][lane], v1s = sl[wid][kk][(lane + 32) % kIncSlots];
+        float v0 = lane < ns ? v0s : 0.0f, v1 = lane + 32 < ns ? v1s : 0.0f;
+        ++kk;
+        bool good = true;
+        int dirty_from = kIncSlots;
+#pragma unroll
+        for (int i = 0; i < NEW; ++i) {
+            const float x = __shfl_sync(0xFFFFFFFFu, xl[i], src);
+            if (!((ml >> i) & 1u) || !good) continue;    // uniform: ml and good are the same in every lane
+            const uint32_t m0 = __ballot_sync(0xFFFFFFFFu, lane < ns && __float_as_uint(v0) == __float_as_uint(x));
+            const uint32_t m1 = __ballot_sync(0xFFFFFFFFu, lane + 32 < ns && __float_as_uint(v1) == __float_as_uint(x));
+            if ((m0 | m1) == 0u) { good = false; continue; }   // the books do not balance: rebuild
+            const int pos = m0 ? __ffs(m0) - 1 : 32 + __ffs(m1) - 1;
+            // positions above pos move down by one
+            const float d0 = __shfl_down_sync(0xFFFFFFFFu, v0, 1), h1 = __shfl_sync(0xFFFFFFFFu, v1, 0);
+            const float d1 = __shfl_down_sync(0xFFFFFFFFu, v1, 1);
+            if (lane >= pos) v0 = (lane == 31) ? h1 : d0;
+            if (lane + 32 >= pos) v1 = d1;
+            --ns;
+            dirty_from = min(dirty_from, pos);
+        }
+#pragma unroll
+        for (int i = 0; i < NEW; ++i) {
+            const float x = __shfl_sync(0xFFFFFFFFu, xe[i], src);
+            if (!((me >> i) & 1u) || !good) continue;
+            if (ns >= kIncSlots) { good = false; continue; }
+            const uint32_t kx = f2key(x);
+            // behind the listed values whose key is not above x's
+            const int at = __popc(__ballot_sync(0xFFFFFFFFu, lane < ns && f2key(v0) <= kx)) +
+                           __popc(__ballot_sync(0xFFFFFFFFu, lane + 32 < ns && f2key(v1) <= kx));
+            const float u0 = __shfl_up_sync(0xFFFFFFFFu, v0, 1), t0 = __shfl_sync(0xFFFFFFFFu, v0, 31);
+            const float u1 = __shfl_up_sync(0xFFFFFFFFu, v1, 1);
+            if (lane + 32 > at) v1 = (lane == 0) ? t0 : u1;
+            else if (lane + 32 == at) v1 = x;
+            if (lane > at) v0 = u0;
+            else if (lane == at) v0 = x;
+            ++ns;
+            dirty_from = min(dirty_from, at);
+        }
+        const int cbs = __shfl_sync(0xFFFFFFFFu, cb, src);
+        good = good && cbs >= 0 && cbs <= k1 && k2 < cbs + ns;
+        if (good) {   // write back the part that moved; hand the middle ranks' values to the series' own lane
+            if (lane >= dirty_from && lane < ns) s.val[lbase + lane] = v0;
+            if (lane + 32 >= dirty_from && lane + 32 < ns) s.val[lbase + lane + 32] = v1;
+        }
+        const int j1 = good ? k1 - cbs : 0, j2 = good ? k2 - cbs : 0;
+        const float g10 = __shfl_sync(0xFFFFFFFFu, v0, j1 & 31), g11 = __shfl_sync(0xFFFFFFFFu, v1, j1 & 31);
+        const float g20 = __shfl_sync(0xFFFFFFFFu, v0, j2 & 31), g21 = __shfl_sync(0xFFFFFFFFu, v1, j2 & 31);
+        if (lane == src) {
+            ok = good;
+            nin = ns;
+            f1 = (j1 >> 5) ? g11 : g10;
+            f2 = (j2 >> 5) ? g21 : g20;
+            have = true;
+        }
+    }
+    ok = ok && cb >= 0 && cb <= k1 && k2 < cb + nin;
+    if (ok) {
+        // the list is sorted: the middle ranks of the window are positions k1 - cb and k2 - cb of it
+        if (!have) {
+            f1 = s.val[(size_t)c * kIncSlots + (k1 - cb)];
+            f2 = s.val[(size_t)c * kIncSlots + (k2 - cb)];
+        }
+        const float med = median_from_keys(f2key(f1), f2key(f2), even);
+        a.wmed[c] = med;
+        if (a.wmed_user) a.wmed_user[c] = med;
+        s.cnt[c] = 0x80000000u | ((uint32_t)nin << 16) | (uint32_t)cb;
+    }
+    // ---- series without a usable state go on the launch's rebuild list (window_rebuild_kernel follows) ----
+    const unsigned todo = __ballot_sync(0xFFFFFFFFu, active && !ok);
+    if (todo) {
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(s.rb_count, (uint32_t)__popc(todo));
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        if ((todo >> lane) & 1u) s.rb_list[base + __popc(todo & ((1u << lane) - 1u))] = (uint32_t)c;
+    }
+}
+
+// The rebuilds of a launch, one warp per listed series (a few per thousand series in steady state, all of them
+// when sliding starts): the lanes fetch the window, sort it (bitonic network over registers and shuffles), take
+// the median, the interval ends kIncHalf ranks beyond the middle ranks, and the values inside.  A kernel of its
+// own so that the rebuilds spread over the whole GPU instead of queueing inside the warps that found them.
+constexpr int kRbThreads = 128;
+constexpr int kRbCtas = 148 * 8;
+
+template <int VPL>
+__global__ void __launch_bounds__(kRbThreads) window_rebuild_kernel(const WindowArgs a, const IncArgs s) {
+    __shared__ int is_last;
+    const int lane = lane_id();
+    const int n = a.n;
+    const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;
+    const bool even = !(n & 1);
+    const int k1 = (n - 1) >> 1, k2 = n >> 1;
+    const uint32_t count = min(__ldcg(s.rb_count), (uint32_t)a.series);
+    const uint32_t nwarps = gridDim.x * (kRbThreads / 32);
+    for (uint32_t i = blockIdx.x * (kRbThreads / 32) + warp_id(); i < count; i += nwarps) {
+        const int series = (int)__ldcg(s.rb_list + i);
         uint32_t kv[VPL];
 #pragma unroll
         for (int j = 0; j < VPL; ++j) {
@@ -613,7 +709,7 @@ __global__ void __launch_bounds__(kIncThreads) window_inc_kernel(const WindowArg
             for (int j = 0; j < VPL; ++j) {
                 const bool real = lane * VPL + j < n;
                 const float x = key2f(kv[j]);
-                if (real && !(x < flo) && (x <= fhi)) { s.val[(size_t)pos * a.series + series] = x; ++pos; }
+                if (real && !(x < flo) && (x <= fhi)) { s.val[(size_t)series * kIncSlots + pos] = x; ++pos; }
             }
         }
         if (lane == 0) {
@@ -625,6 +721,14 @@ __global__ void __launch_bounds__(kIncThreads) window_inc_kernel(const WindowArg
             s.cnt[series] = fits ? (0x80000000u | ((uint32_t)nin2 << 16) | (uint32_t)cb2) : 0u;
             if (s.rebuilds) atomicAdd(s.rebuilds, 1u);
         }
+    }
+    // the CTA that finishes last clears the list for the next launch
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(s.rb_count + 1, 1u) == gridDim.x - 1u) ? 1 : 0;
+    __syncthreads();
+    if (is_last && threadIdx.x == 0) {
+        s.rb_count[0] = 0u;
+        s.rb_count[1] = 0u;
     }
 }
 
@@ -694,9 +798,12 @@ bool window_inc_supported(const WindowArgs &a) { return a.n >= 1 && a.n <= 256; 
 
 cudaError_t launch_window_incremental(const WindowArgs &a, const IncArgs &inc, cudaStream_t st) {
     const int grid = (a.series + kIncThreads - 1) / kIncThreads;
-    if (a.n <= 64) window_inc_kernel<2><<<grid, kIncThreads, 0, st>>>(a, inc);
-    else if (a.n <= 128) window_inc_kernel<4><<<grid, kIncThreads, 0, st>>>(a, inc);
-    else window_inc_kernel<8><<<grid, kIncThreads, 0, st>>>(a, inc);
+    const int rgrid = min(kRbCtas, (a.series + kRbThreads / 32 - 1) / (kRbThreads / 32));
+    if (inc.entering <= 1 && inc.leaving <= 1) window_inc_kernel<1><<<grid, kIncThreads, 0, st>>>(a, inc);
+    else window_inc_kernel<kIncMaxNew><<<grid, kIncThreads, 0, st>>>(a, inc);
+    if (a.n <= 64) window_rebuild_kernel<2><<<rgrid, kRbThreads, 0, st>>>(a, inc);
+    else if (a.n <= 128) window_rebuild_kernel<4><<<rgrid, kRbThreads, 0, st>>>(a, inc);
+    else window_rebuild_kernel<8><<<rgrid, kRbThreads, 0, st>>>(a, inc);
     return cudaGetLastError();
 }
 
