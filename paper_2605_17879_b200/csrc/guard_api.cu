@@ -632,7 +632,9 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
             t.hint = (TopkHint *)(c->ws + c->L.topk_hint);
             t.hcand = (unsigned long long *)(c->ws + c->L.topk_hint + 256);
         }
-        if (c->overlap && c->ensure_side()) {
+        // a deferred evaluation with a hinted (short) selection keeps it on the tail stream: two event calls less, and
+        // the internal stream is free for the next evaluation's window medians
+        if (c->overlap && !(defer && t.hint) && c->ensure_side()) {
             if (!(defer || forked)) {   // the window medians ran on `st`: order the internal stream behind them
                 e = cudaEventRecord(c->ev_fork, st);
                 if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
