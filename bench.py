@@ -253,6 +253,9 @@ def run_small_config(dev, name, passes=5):
 def run_streaming(dev, steps, warm):
     """Streaming configuration: 32 768 ranks x 8 metrics, one step per ingest into a 512-step
     ring, an evaluation after every step, flags and top-k read back to pinned host memory.
+    Latency leg: the step is landed in its ring slot before the clock starts (in-place ingest).
+    Sustained leg: guard_ingest copies each step from a staging buffer into the ring (one call
+    per step), deferred evaluations, joined before the clock stops.
     Returns per-step ingest-to-flag latency percentiles (host clock) and sustained cells/s."""
     import torch
     from paper_2605_17879_b200 import guard, synth
