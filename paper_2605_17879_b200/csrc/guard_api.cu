@@ -560,6 +560,8 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     c->inc_now = use_inc ? &ia : nullptr;
     c->seen_at_eval = c->seen;
     w.fb_count = c->status() + 8;
+    w.fb_list = (uint32_t *)(c->ws + c->L.inc_rbl);          // shared with the sliding path's rebuild list: an evaluation takes one path
+    w.fb_list_count = (uint32_t *)(c->ws + c->L.inc_rbc);
     w.status = c->status();
     w.first_wait_cycles = c->wait_limit;
     // The window medians read only the ring: run them on the internal stream, forked where the

@@ -101,6 +101,8 @@ struct WindowArgs {
     float *centre;          // [series] smoothed median: the centre of the thread path's interval (state), or NULL
     int target;             // number of keys the thread path's interval is tuned to catch (0: default)
     float smooth;           // weight of the newest median in the interval's centre (0: default)
+    uint32_t *fb_list;      // [series] scratch: series the thread path leaves to its finishing kernel (why << 28 | series)
+    uint32_t *fb_list_count;// [2] their number and the finishing kernel's ticket: zero before first use, self-resetting
     uint32_t *fb_count;     // [6] series the thread path's interval did not serve, in total and by reason (diagnostic), or NULL
     uint32_t *status;
     long long first_wait_cycles;   // limit of the warp path's wait for a staged tile (0: the default of about a second)

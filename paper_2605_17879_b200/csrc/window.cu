@@ -419,16 +419,37 @@ __global__ void __launch_bounds__(kThCols, 9) window_thread_kernel(const WindowA
         a.spread[c] = h * (0.5f + 0.5f * f);
         a.centre[c] = hint + (a.smooth > 0.0f ? a.smooth : kThSmooth) * (med - hint);
     }
-    // ---- series the interval did not serve: the whole warp finishes them one by one ------------
-    unsigned todo = __ballot_sync(0xFFFFFFFFu, active && !ok);
+    // ---- series the interval did not serve go on the launch's list (window_finish_kernel follows) ------
     // why (diagnostic): 0 no usable interval, 1 more keys than slots, 2 median below the interval,
     // 3 above it, 4 selection did not converge
     const int why = !usable ? 0 : (nk > kThSlots ? 1 : ((int)clt > k1 ? 2 : (k2 >= (int)clt + nk ? 3 : 4)));
-    while (todo) {
-        const int src = __ffs(todo) - 1;
-        todo &= todo - 1;
-        const int series = __shfl_sync(0xFFFFFFFFu, c, src);
-        const int why_src = __shfl_sync(0xFFFFFFFFu, why, src);
+    const unsigned todo = __ballot_sync(0xFFFFFFFFu, active && !ok);
+    if (todo) {
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(a.fb_list_count, (uint32_t)__popc(todo));
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        if ((todo >> lane) & 1u) a.fb_list[base + __popc(todo & ((1u << lane) - 1u))] = ((uint32_t)why << 28) | (uint32_t)c;
+    }
+}
+
+// The series the thread path's interval did not serve (a few per thousand), one warp per listed series: the lanes
+// fetch the window, sort their own keys and run the warp selection; the series' interval state starts afresh.
+// A kernel of its own, so that these series spread over the GPU instead of queueing behind one another at the end
+// of the warp that found them.
+constexpr int kFinThreads = 128;
+constexpr int kFinCtas = 148 * 4;
+
+template <int VPL>
+__global__ void __launch_bounds__(kFinThreads) window_finish_kernel(const WindowArgs a) {
+    __shared__ int is_last;
+    const int lane = lane_id();
+    const int n = a.n;
+    const int first = ((a.last_slot - (n - 1)) % a.capacity + a.capacity) % a.capacity;
+    const uint32_t count = min(__ldcg(a.fb_list_count), (uint32_t)a.series);
+    const uint32_t nwarps = gridDim.x * (kFinThreads / 32);
+    for (uint32_t i = blockIdx.x * (kFinThreads / 32) + warp_id(); i < count; i += nwarps) {
+        const uint32_t item = __ldcg(a.fb_list + i);
+        const int series = (int)(item & 0x0FFFFFFFu), why_src = (int)(item >> 28);
         uint32_t kv[VPL];
         int nreal = 0;
 #pragma unroll
@@ -455,6 +476,14 @@ __global__ void __launch_bounds__(kThCols, 9) window_thread_kernel(const WindowA
             if (a.fb_count) { atomicAdd(a.fb_count, 1u); atomicAdd(a.fb_count + 1 + why_src, 1u); }
         }
     }
+    // the CTA that finishes last clears the list for the next launch
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(a.fb_list_count + 1, 1u) == gridDim.x - 1u) ? 1 : 0;
+    __syncthreads();
+    if (is_last && threadIdx.x == 0) {
+        a.fb_list_count[0] = 0u;
+        a.fb_list_count[1] = 0u;
+    }
 }
 
 template <int VPL>
@@ -470,6 +499,8 @@ cudaError_t launch_thread_path(const WindowArgs &a, cudaStream_t st) {
     });
     if (e != cudaSuccess) return e;
     window_thread_kernel<VPL><<<(a.series + kThCols - 1) / kThCols, kThCols, smem, st>>>(a);
+    const int fgrid = min(kFinCtas, (a.series + kFinThreads / 32 - 1) / (kFinThreads / 32));
+    window_finish_kernel<VPL><<<fgrid, kFinThreads, 0, st>>>(a);
     return cudaGetLastError();
 }
 
@@ -790,7 +821,7 @@ cudaError_t launch_staged(const WindowArgs &a, int use_bulk, cudaStream_t st) {
 
 }  // namespace
 
-int window_launch_count(const WindowArgs &) { return 1; }
+int window_launch_count(const WindowArgs &a) { return (a.use_hint && a.spread && a.centre && a.fb_list && a.series < (1 << 28) && a.n <= 256) ? 2 : 1; }
 
 size_t window_inc_bytes(int series) { return (size_t)series * sizeof(float); }
 
@@ -812,7 +843,7 @@ cudaError_t launch_window_select(const WindowArgs &a, cudaStream_t st) {
     // bulk copies need 16-byte aligned sources and sizes
     const int use_bulk = (a.series % 4 == 0) && (((uintptr_t)a.ring & 15) == 0);
     const size_t n = (size_t)a.n;
-    if (a.use_hint && a.spread && a.centre && n <= 256) {
+    if (a.use_hint && a.spread && a.centre && a.fb_list && a.series < (1 << 28) && n <= 256) {
         if (n <= 64) return launch_thread_path<2>(a, st);
         if (n <= 128) return launch_thread_path<4>(a, st);
         return launch_thread_path<8>(a, st);
