@@ -310,6 +310,9 @@ struct guard_ctx {
     // scratch of the bracketed path: such rows take the direct selection.
     // site: 0 the ingested step, 1 the fleet baseline, -1 neither.  A site keeps the brackets of its single rows.
     bool row_hints = true;   // guard_set_row_hints
+    // stamp of the split path's column records: changed whenever the scratch stops describing this context's data
+    uint32_t split_epoch = 1;
+    void new_epoch() { split_epoch = split_epoch * 2654435761u + 12345u; if (split_epoch == 0) split_epoch = 1; }
     ColHintState *hint_state(int site) const { return (ColHintState *)(ws + L.xr_grid + (size_t)site * align_up(sizeof(ColHintState))); }
     cudaError_t xrank(XrankArgs a, int S, cudaStream_t st, bool own_scratch = true, int site = -1) {
         // a few rows at a time: one CTA per column keeps the whole GPU busy
@@ -321,6 +324,7 @@ struct guard_ctx {
         }
         if (L.xr_split && a.mask_bytes == 1) {
             a.fallbacks = status() + 1;
+            a.hint_epoch = row_hints ? split_epoch : 0u;
             const int first = a.first_slot;
             const int smax = C < kSplitMaxSteps ? C : kSplitMaxSteps;
             for (int s0 = 0; s0 < S; s0 += smax) {
@@ -414,6 +418,8 @@ int guard_create(guard_ctx **out, int ranks, int metrics, int W, int k, const gu
     c->R = ranks; c->M = metrics; c->W = W; c->k = k; c->C = capacity_steps; c->K = topk;
     c->p = p; c->L = L; c->ws = (char *)d_workspace; c->seen = 0; c->launches = 0; c->evals = 0; c->error[0] = 0;
     c->ranks_per_node = th->ranks_per_node;
+    c->split_epoch = (uint32_t)((uintptr_t)c >> 4) ^ (uint32_t)((uintptr_t)d_workspace >> 8);
+    c->new_epoch();
     // state: status word, ticket, fleet statistics, consecutive counters
     cudaError_t e = cudaMemsetAsync(c->ws, 0, L.wmed, (cudaStream_t)stream);
     if (e != cudaSuccess) {
@@ -983,6 +989,7 @@ int guard_state_import(guard_ctx *c, const void *d_state, size_t state_bytes, vo
     c->inc_n = h.inc_n;
     c->cnt_seen = -1;   // the kept counts are not part of the state: the next evaluation recounts
     c->hints_ready = h.hints_ready != 0;
+    c->new_epoch();   // the split scratch describes other data
     c->fork_fresh = false;
     return GUARD_OK;
 }
@@ -1018,6 +1025,7 @@ int guard_reset(guard_ctx *c, void *stream) {
     c->inc_seen = -1;
     c->cnt_seen = -1;
     c->hints_ready = false;
+    c->new_epoch();
     return GUARD_OK;
 }
 

@@ -28,6 +28,7 @@ struct XrankArgs {
     uint32_t *only_flagged; // [S] or NULL: direct kernel processes step s only if nonzero, then clears it
     uint32_t *fallbacks;    // or NULL: counts the steps the direct kernel redid for the bracketed path
     void *hint;             // ColHintState of the call site (one row per call), or NULL: column kernels only
+    uint32_t hint_epoch;    // split path: non-zero lets a block use the records the previous block left in its scratch
 };
 
 // Scratch of the bracketed path for up to S_max steps per launch.

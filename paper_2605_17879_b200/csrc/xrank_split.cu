@@ -63,7 +63,9 @@ struct SpCol {
     float lo, hi, dlo, dhi;   // intervals of the median and of the MAD
     float med, rlo, rhi, rhs; // median; range of the exceedance threshold over [dlo, dhi]; exact threshold
     uint32_t cnt;             // elements below the current interval
-    uint32_t pad[3];
+    float mad;                // the column's MAD (kept for the next use of this record)
+    uint32_t epoch;           // SpScratch::epoch of the launch that completed med / mad on the fast path (else 0)
+    uint32_t pad;
 };
 
 struct SpScratch {
@@ -73,6 +75,7 @@ struct SpScratch {
     uint32_t *amb;    // [S][kSpAmb] (rank << 5 | metric)
     uint32_t *nseg;   // [S][M][chunks] kept elements of each sweep CTA
     uint32_t *list;   // [S][M][chunks][cap] kept elements (raw bits), one segment per sweep CTA
+    uint32_t epoch;   // non-zero: records stamped with this value hold the previous results of the same step position
 };
 
 // ---- per-element operations of the sweeps, written out so that each is a fixed handful of
@@ -154,6 +157,36 @@ __global__ void __launch_bounds__(kSpSmpThreads, 3) xsplit_sample_kernel(const X
     const float *row = a.base + (size_t)slot * a.row_stride;
     const int period = 4 * g.stride, first = (period - 4) >> 1;
 
+    // The column records still hold what the previous block on this scratch found at the same step position:
+    // consecutive blocks of a fleet have almost the same per-step cross-rank median and MAD, so those bracket
+    // the new ones without sampling anything (five standard errors of the difference of two sample medians /
+    // MADs of normal data to either side; a miss is caught by the counts and the step redone).  Anything
+    // else (first use, a step that left the fast path, a zero MAD) samples.
+    __shared__ int s_hinted[4];
+    if (tid < 4) {
+        const SpCol &old = sc.col[(size_t)t * M + 4 * q + tid];
+        const float om = old.med, od = old.mad;
+        const bool v = sc.epoch != 0u && old.epoch == sc.epoch && od > 0.0f && od < kFltMax && fabsf(om) < kFltMax;
+        s_hinted[tid] = v ? 1 : 0;
+    }
+    __syncthreads();
+    if (s_hinted[0] && s_hinted[1] && s_hinted[2] && s_hinted[3]) {
+        if (tid < 4) {
+            SpCol &col = sc.col[(size_t)t * M + 4 * q + tid];
+            const float om = col.med, od = col.mad;
+            const float u = od * rsqrtf((float)R);
+            const float hm = 13.1f * u, hd = 8.25f * u;
+            col.lo = fmaxf(om - hm, -kFltMax);
+            col.hi = fminf(om + hm, kFltMax);
+            col.dlo = fmaxf(od - hd, 0.0f);
+            col.dhi = fminf(od + hd, kFltMax);
+            col.cnt = 0;
+            col.epoch = 0;   // stamped again when this block's median and MAD are complete
+        }
+        if (tid == 0 && q == 0) { sc.fail[t] = 0; sc.namb[t] = 0; }
+        return;
+    }
+
     // all loads first: the sampled ranks, and (warps 0..3) the 32 spread values that fix a metric's bin map
     float4 xs[kSpSmpLoads];
 #pragma unroll
@@ -168,6 +201,7 @@ __global__ void __launch_bounds__(kSpSmpThreads, 3) xsplit_sample_kernel(const X
     if (tid < 4) {
         SpCol &col = sc.col[(size_t)t * M + 4 * q + tid];
         col.cnt = 0;
+        col.epoch = 0;
     }
     if (tid == 0 && q == 0) { sc.fail[t] = 0; sc.namb[t] = 0; }
     if (tid == 0) {
@@ -649,6 +683,8 @@ __global__ void __launch_bounds__(kSpSelThreads, 12) xsplit_select_kernel(const 
                 a.mad[so + m] = val;
                 if (a.mad_user) a.mad_user[so + m] = val;
                 col.rhs = __fmul_rn(p.thrp[m], scale_of(val, col.med, p.floor_rel[m], p.floor_abs[m]));
+                col.mad = val;
+                col.epoch = sc.epoch;
             }
         } else {
             atomicOr(&sc.fail[t], 1u);
@@ -747,6 +783,7 @@ cudaError_t launch_xrank_split(const XrankArgs &a, const MetricParams &p, int S,
     sc.amb = (uint32_t *)b;   b += align256((size_t)S * kSpAmb * sizeof(uint32_t));
     sc.nseg = (uint32_t *)b;  b += align256((size_t)S * M * g.chunks * sizeof(uint32_t));
     sc.list = (uint32_t *)b;
+    sc.epoch = a.hint_epoch;
     const size_t smem = split_sweep_smem(g, M);
     static std::mutex attr_mutex;
     static bool attr_set_dev[64] = {};
