@@ -37,10 +37,10 @@ UNIT = "cells/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this workload, from
 # the ncu capture summarised under profiles/ (None once the kernel has changed since the capture)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 118.60e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 112.0e6   # window_thread_kernel 110.72e6 + its finishing kernel (~200 series x 6.4 KB)
 # which kernel the roofline object describes: 2 = window_thread_kernel (guard_score), 1 = the MAD sweep (guard_ingest)
 PROFILE_MODE = 2
-PROFILE_KERNEL = ("window_thread_kernel (windowed per-rank medians of one evaluation)" if PROFILE_MODE == 2 else
+PROFILE_KERNEL = ("window_thread_kernel + window_finish_kernel (windowed per-rank medians of one evaluation)" if PROFILE_MODE == 2 else
                   "xsplit_sweep_kernel<2,1> (cross-rank MAD / exceedance sweep of one ingested block)")
 FALLBACK_HBM_GBS = 6650.0   # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
 
