@@ -117,3 +117,36 @@ def test_rows_with_nonfinite_values_are_flagged():
         g.sync_status()
     assert ei.value.code == -4
     g.close()
+
+
+def test_block_brackets_of_the_split_path_survive_a_jump_between_blocks():
+    """Blocks of several steps on the split path: a block's column records bracket the next block's medians and
+    MADs.  After a jump of every rank between two blocks the counts do not prove the brackets: those steps are
+    redone by the direct selection, the next block samples again, and every result stays exact."""
+    from parity_util import run_both
+    from paper_2605_17879_b200 import guard
+    R, M, B, nb = 4096, 8, 16, 7
+    cfg = synth.FleetConfig("blocks", ranks=R, steps=B * nb, metrics=M, sigma=0.03, seed=77, W=B, k=10, topk=16, block=B,
+                            node_sigma=0.005, n_ramp=3, ramp_to=1.3, ramp_len=40, ramp_start_max=B * nb - 1, heavy_tail=0.01)
+    X = synth.fleet_block(cfg, 0, B * nb, device="cpu").numpy().copy()
+    X[3 * B:] *= np.float32(1.5)
+    dirs = synth.fleet_dir(M)
+    # stationary stretch first: no step leaves the fast path
+    run_both(X[:3 * B], B, 10, 16, dirs, [B], capacity=2 * B, max_fallback_steps=0)
+    # the jump: the sixteen steps of the first block after it are redone, nothing else
+    g = guard.Guard(R, M, B, 10, dir=dirs, capacity=2 * B, topk=16)
+    o = go.Oracle(R, M, B, 10, 16, dir=dirs)
+    Xd = torch.from_numpy(X).cuda()
+    for j in range(nb):
+        smed = torch.empty((B, M), dtype=torch.float32, device="cuda")
+        smad = torch.empty((B, M), dtype=torch.float32, device="cuda")
+        g.ingest(Xd[j * B:(j + 1) * B].contiguous(), smed, smad)
+        ir = o.ingest(X[j * B:(j + 1) * B])
+        assert_bit_equal(to_np(smed), ir["step_med"], "step_med block %d" % j)
+        assert_bit_equal(to_np(smad), ir["step_mad"], "step_mad block %d" % j)
+        out = g.score()
+        assert g.sync_status() == 0
+        compare_score(out, o.score(), "block %d" % j)
+        fb = g.fallback_steps()
+        assert fb == (0 if j < 3 else B), (j, fb)
+    g.close()
