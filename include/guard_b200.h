@@ -281,8 +281,12 @@ int guard_set_sliding(guard_ctx *ctx, int on);
  * 8 192 ranks on, a call site keeps its previous median and MAD and a tuned width per metric, which
  * bracket the next row's: the selection then counts the values below the bracket, bins the few inside
  * and ranks the wanted bin's values directly.  The counts prove the bracket; a row they do not prove
- * (the first one, a jump, ties) takes the general selection inside the same kernel.  Results are
- * identical either way; guard_set_row_hints(ctx, 0) always takes the general selection. */
+ * (the first one, a jump, ties) takes the general selection inside the same kernel.  Blocks of many
+ * steps (4 096 ranks and more, 4 or 8 metrics) use the same idea: the medians and MADs a block found
+ * stay in its scratch and bracket those of the next block at the same step position, so nothing is
+ * sampled; a step whose counts do not prove its bracket is redone exactly (it counts in
+ * guard_fallback_steps) and samples next time.  Results are identical either way;
+ * guard_set_row_hints(ctx, 0) always takes the general selection / sampled intervals. */
 int guard_set_row_hints(guard_ctx *ctx, int on);
 
 /* Diagnostic: synchronises `stream` and fills out[6] (HOST): single rows seen and (row, metric)

@@ -1,5 +1,7 @@
 // C ABI of the library: context object, workspace carving, argument checks and the
 // stream-ordered kernel sequences behind guard_ingest / guard_score / guard_sweep_qualify.
+#include <atomic>
+#include <chrono>
 #include <cstdarg>
 #include <cstddef>
 #include <cstdio>
@@ -312,7 +314,12 @@ struct guard_ctx {
     bool row_hints = true;   // guard_set_row_hints
     // stamp of the split path's column records: changed whenever the scratch stops describing this context's data
     uint32_t split_epoch = 1;
-    void new_epoch() { split_epoch = split_epoch * 2654435761u + 12345u; if (split_epoch == 0) split_epoch = 1; }
+    // never the same value twice in a process (device memory is handed out again with its old contents, at the
+    // same addresses: a stamp derived from addresses would take another context's leftovers for its own)
+    void new_epoch() {
+        static std::atomic<uint32_t> next{(uint32_t)std::chrono::steady_clock::now().time_since_epoch().count() | 1u};
+        do { split_epoch = next.fetch_add(1u); } while (split_epoch == 0u);
+    }
     ColHintState *hint_state(int site) const { return (ColHintState *)(ws + L.xr_grid + (size_t)site * align_up(sizeof(ColHintState))); }
     cudaError_t xrank(XrankArgs a, int S, cudaStream_t st, bool own_scratch = true, int site = -1) {
         // a few rows at a time: one CTA per column keeps the whole GPU busy
@@ -418,7 +425,6 @@ int guard_create(guard_ctx **out, int ranks, int metrics, int W, int k, const gu
     c->R = ranks; c->M = metrics; c->W = W; c->k = k; c->C = capacity_steps; c->K = topk;
     c->p = p; c->L = L; c->ws = (char *)d_workspace; c->seen = 0; c->launches = 0; c->evals = 0; c->error[0] = 0;
     c->ranks_per_node = th->ranks_per_node;
-    c->split_epoch = (uint32_t)((uintptr_t)c >> 4) ^ (uint32_t)((uintptr_t)d_workspace >> 8);
     c->new_epoch();
     // state: status word, ticket, fleet statistics, consecutive counters
     cudaError_t e = cudaMemsetAsync(c->ws, 0, L.wmed, (cudaStream_t)stream);
