@@ -740,7 +740,9 @@ size_t guard_sweep_workspace_bytes(int gpus, int reps, int metrics) {
     if (gpus < 1 || reps < 1 || reps > GUARD_MAX_WINDOW || metrics < 1 || metrics > GUARD_MAX_METRICS ||
         (long long)gpus * metrics > 0x7FFFFFFFLL)
         return 0;
-    return align_up(3 * kMaxMetrics * sizeof(float)) + align_up((size_t)gpus * metrics * sizeof(float));
+    // fleet statistics, per-GPU medians, then the thread path's list of unserved series and its counter
+    return align_up(3 * kMaxMetrics * sizeof(float)) + align_up((size_t)gpus * metrics * sizeof(float)) +
+           align_up((size_t)gpus * metrics * sizeof(uint32_t)) + align_up(64);
 }
 
 int guard_sweep_qualify(const float *d_S, int nodes, int gpus_per_node, int reps, int metrics, const guard_thresholds *th,
@@ -773,6 +775,8 @@ int guard_sweep_qualify(const float *d_S, int nodes, int gpus_per_node, int reps
     sm.gmed = gmed;
     sm.gmed_user = d_gpu_med;
     sm.status = d_status;
+    sm.list = (uint32_t *)((char *)gmed + align_up((size_t)G * metrics * sizeof(float)));
+    sm.list_count = (uint32_t *)((char *)sm.list + align_up((size_t)G * metrics * sizeof(uint32_t)));
     cudaError_t e = launch_sweep_medians(sm, st);
     if (e != cudaSuccess) { set_error(g_error, "sweep medians launch: %s", cudaGetErrorString(e)); return GUARD_ERR_CUDA; }
 

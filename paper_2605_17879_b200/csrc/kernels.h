@@ -212,6 +212,8 @@ struct SweepMedArgs {
     float *gmed;      // [G][M]
     float *gmed_user; // or NULL
     uint32_t *status; // or NULL
+    uint32_t *list;        // [G * M] scratch: series the thread path leaves to its finishing kernel, or NULL (then the warp path runs)
+    uint32_t *list_count;  // [1] their number (cleared by the launcher)
 };
 cudaError_t launch_sweep_medians(const SweepMedArgs &a, cudaStream_t st);
 

@@ -8,6 +8,7 @@
 
 #include "colselect.cuh"
 #include "kernels.h"
+#include "thselect.cuh"
 #include "warpselect.cuh"
 #include "xrank_common.cuh"
 
@@ -269,30 +270,6 @@ constexpr int kThRows = 8;       // rows in flight per thread
 constexpr int kThMaxPasses = 12;
 constexpr float kThSmooth = 0.3f;   // weight of the newest median in the interval's centre
 
-// cnt += (x < lo); if (lo <= x <= hi) { if (addr < lim) shared[addr] = x; addr += 4; }
-__device__ __forceinline__ void th_cell(const float x, const float lo, const float hi, const uint32_t lim, uint32_t &cnt,
-                                        uint32_t &addr) {
-    asm volatile(
-        "{\n\t.reg .pred p, q, r;\n\t"
-        "setp.lt.f32 p, %2, %3;\n\t"
-        "setp.le.and.f32 q, %2, %4, !p;\n\t"
-        "setp.lt.and.u32 r, %1, %5, q;\n\t"
-        "@p add.u32 %0, %0, 1;\n\t"
-        "@r st.shared.f32 [%1], %2;\n\t"
-        "@q add.u32 %1, %1, 4;\n\t}"
-        : "+r"(cnt), "+r"(addr)
-        : "f"(x), "f"(lo), "f"(hi), "r"(lim)
-        : "memory");
-}
-__device__ __forceinline__ uint4 th_lds4(const uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ void th_sts4(const uint32_t addr, const uint4 v) {
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
 template <int VPL>
 __global__ void __launch_bounds__(kThCols, 9) window_thread_kernel(const WindowArgs a) {
     extern __shared__ __align__(16) uint32_t tkept[];   // [kThCols][kThSlots]
@@ -337,79 +314,9 @@ __global__ void __launch_bounds__(kThCols, 9) window_thread_kernel(const WindowA
     const int t = k2 - (int)clt;     // rank of the upper middle among the kept keys (t >= 1 when n is even)
     float med = 0.0f;
     // ---- selection among the kept keys: the same instruction stream in every lane ---------------
-    const int nkmax = (int)__reduce_max_sync(0xFFFFFFFFu, ok ? (uint32_t)nk : 0u);
-    if (nkmax > 0) {
-        const int nkr = (nkmax + 3) & ~3;   // <= kThSlots (a multiple of 4)
-        for (int j = 0; j < nkr; j += 4) {  // raw bits -> keys; slots without a key compare above everything
-            uint4 v = th_lds4(kbase + 4u * j);
-            v.x = (ok && j + 0 < nk) ? key_of_bits(v.x) : 0xFFFFFFFFu;
-            v.y = (ok && j + 1 < nk) ? key_of_bits(v.y) : 0xFFFFFFFFu;
-            v.z = (ok && j + 2 < nk) ? key_of_bits(v.z) : 0xFFFFFFFFu;
-            v.w = (ok && j + 3 < nk) ? key_of_bits(v.w) : 0xFFFFFFFFu;
-            th_sts4(kbase + 4u * j, v);
-        }
-        // The pivot moves inside a key bracket (pl, ph) with below(pl) = al <= t - 2 and
-        // below(ph) = ah >= t + 2.
-        uint32_t pl = klo, ph = khi + 1u, pv = klo;
-        int al = 0, ah = nk, bsave = 0;
-        int done = 0;                 // 1: pv has bsave in {t - 1, t, t + 1} keys below it, 2: both ranks equal pl
-        if (!ok || t <= 1) { done = 1; pv = klo; bsave = 0; }
-        else if (t >= nk - 1) { done = 1; pv = khi + 1u; bsave = nk; }
-        for (int pass = 0; pass < kThMaxPasses; ++pass) {
-            if (__all_sync(0xFFFFFFFFu, done != 0)) break;
-            if (!done) {
-                if (ph - pl < 2u) {
-                    done = 2;
-                } else if (pass % 3 == 2) {
-                    pv = pl + ((ph - pl) >> 1);
-                } else {   // aim between the ends in proportion to the missing count
-                    const float fr = (float)(t - al) / (float)(ah - al);
-                    pv = pl + (uint32_t)((float)(ph - pl) * fr);
-                    pv = pv <= pl ? pl + 1u : (pv >= ph ? ph - 1u : pv);
-                }
-            }
-            // the loads of a third of the column are issued before their compares
-            int below = 0;
-#pragma unroll
-            for (int j0 = 0; j0 < kThSlots / 4; j0 += 5) {
-                uint4 kv4[5];
-#pragma unroll
-                for (int j = 0; j < 5; ++j)
-                    if (4 * (j0 + j) < nkr) kv4[j] = th_lds4(kbase + 16u * (j0 + j));
-#pragma unroll
-                for (int j = 0; j < 5; ++j)
-                    if (4 * (j0 + j) < nkr) below += (kv4[j].x < pv) + (kv4[j].y < pv) + (kv4[j].z < pv) + (kv4[j].w < pv);
-            }
-            if (!done) {
-                if (below >= t - 1 && below <= t + 1) { done = 1; bsave = below; }
-                else if (below < t) { pl = pv; al = below; }
-                else { ph = pv; ah = below; }
-            }
-        }
-        if (ok && !done) {
-            if (ph - pl < 2u) done = 2; else ok = false;
-        }
-        // the two largest keys below the pivot (b1 >= b2), the two smallest keys not below it (u1 <= u2)
-        uint32_t b1 = 0u, b2 = 0u, u1 = 0xFFFFFFFFu, u2 = 0xFFFFFFFFu;
-        for (int j = 0; j < nkr; j += 4) {
-            const uint4 v4 = th_lds4(kbase + 4u * j);
-            const uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const bool lt = v[u] < pv;
-                const uint32_t lo_v = lt ? v[u] : 0u, hi_v = lt ? 0xFFFFFFFFu : v[u];   // neutral on the other side
-                b2 = max(b2, min(b1, lo_v));
-                b1 = max(b1, lo_v);
-                u2 = min(u2, max(u1, hi_v));
-                u1 = min(u1, hi_v);
-            }
-        }
-        uint32_t vb = b1, vu = u1;                       // bsave == t
-        if (bsave == t + 1) { vb = b2; vu = b1; }
-        if (bsave == t - 1) { vb = u1; vu = u2; }
-        if (done == 2) { vb = pl; vu = pl; }
-        if (ok) med = median_from_keys(even ? vb : vu, vu, even);
-    }
+    uint32_t vb = 0, vu = 0;
+    th_select_pair<kThSlots, kThMaxPasses>(kbase, nk, ok, t, klo, khi, vb, vu);
+    if (ok) med = median_from_keys(even ? vb : vu, vu, even);
     if (active && ok) {
         a.wmed[c] = med;
         if (a.wmed_user) a.wmed_user[c] = med;
