@@ -581,7 +581,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
     // the caller's stream waits for them before anything that uses them.
     cudaError_t e;
     // a deferred evaluation still pending is complete, in the caller's stream order, from here on
-    const bool had_pending = c->pending;
+    const bool same_buffers_busy = c->infl[q].on;   // the evaluation before the previous one (join clears the records)
     e = c->join(st);
     if (e != cudaSuccess) return c->cuda_fail(e, "join of the deferred evaluation");
     const bool forked = c->overlap && c->fork_fresh && c->side;
@@ -603,7 +603,7 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
         }
         e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
         // the evaluation before the previous one used the same buffers: its tail must have read them
-        if (e == cudaSuccess && c->infl[q].on) e = cudaStreamWaitEvent(c->side, c->ev_e[q], 0);
+        if (e == cudaSuccess && same_buffers_busy) e = cudaStreamWaitEvent(c->side, c->ev_e[q], 0);
         if (e == cudaSuccess) e = c->window(w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_w, c->side);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_x, st);
