@@ -199,6 +199,7 @@ struct guard_ctx {
     int xs_next = 0;
     int scratch_sel = 0;                // which split scratch the next launch uses
     cudaStream_t tail = nullptr;
+    cudaStream_t aux = nullptr;       // deferred evaluations: the top-k selection, beside the fleet baseline and clear of the window medians' stream
     cudaEvent_t ev_x = nullptr, ev_w = nullptr;
     // end of the deferred evaluations, by parity of the evaluation count: up to two may be in flight (the tail of
     // one beside the window medians of the next); each keeps its window for the ring protection
@@ -256,6 +257,7 @@ struct guard_ctx {
         int prio_lo = 0, prio_hi = 0;
         cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
         if (cudaStreamCreateWithPriority(&tail, cudaStreamNonBlocking, GUARD_EVAL_PRIO ? prio_hi : 0) != cudaSuccess) { tail = nullptr; return false; }
+        if (cudaStreamCreateWithPriority(&aux, cudaStreamNonBlocking, GUARD_EVAL_PRIO ? prio_hi : 0) != cudaSuccess) aux = nullptr;
         if (cudaEventCreateWithFlags(&ev_x, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&ev_w, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&ev_e[0], cudaEventDisableTiming) != cudaSuccess ||
@@ -653,8 +655,12 @@ int guard_score(guard_ctx *c, float *d_wmed, float *d_fleet_med, float *d_fleet_
                 e = cudaEventRecord(c->ev_fork, st);
                 if (e == cudaSuccess) e = cudaStreamWaitEvent(c->side, c->ev_fork, 0);
             }
-            if (e == cudaSuccess) e = launch_topk(t, c->p, c->side);
-            if (e == cudaSuccess) e = cudaEventRecord(c->ev_topk, c->side);
+            // deferred: on a stream of its own behind the window medians (ev_w), so that the next evaluation's window
+            // medians need not queue behind it
+            cudaStream_t tk = (defer && c->aux) ? c->aux : c->side;
+            if (e == cudaSuccess && tk == c->aux) e = cudaStreamWaitEvent(c->aux, c->ev_w, 0);
+            if (e == cudaSuccess) e = launch_topk(t, c->p, tk);
+            if (e == cudaSuccess) e = cudaEventRecord(c->ev_topk, tk);
             topk_side = true;
         } else {
             e = launch_topk(t, c->p, ts);
@@ -1174,6 +1180,7 @@ void guard_destroy(guard_ctx *c) {
         if (c->tail) {
             cudaStreamSynchronize(c->tail);
             cudaStreamDestroy(c->tail);
+            if (c->aux) { cudaStreamSynchronize(c->aux); cudaStreamDestroy(c->aux); }
             cudaEventDestroy(c->ev_x);
             cudaEventDestroy(c->ev_w);
             cudaEventDestroy(c->ev_e[0]);
