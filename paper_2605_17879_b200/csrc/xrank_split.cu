@@ -44,6 +44,7 @@ constexpr int kSpSBins = 2048;      // sample histogram bins (16-bit counters, t
 constexpr int kSpBins = 1024;       // selection histogram bins
 constexpr int kSpSelThreads = 128;  // sample / select CTA
 constexpr int kSpJmax = 20;         // kept elements per thread the register selection can hold
+constexpr int kSpJsmall = 12;       // ... and of its variant for short lists
 constexpr int kSpSegs = 4;          // sweep CTAs per step the selection can gather from
 constexpr int kSpMaxM = 8;
 constexpr float kFltMax = 3.402823466e+38f;
@@ -665,8 +666,15 @@ __global__ void __launch_bounds__(kSpSelThreads, 12) xsplit_select_kernel(const 
     if (why < 0) {
         const uint32_t base = f2key((MODE == 0 && flo == 0.0f) ? -0.0f : flo);
         const uint32_t width = f2key((MODE == 0 && fhi == 0.0f) ? 0.0f : fhi) - base;
-        if (!sp_select_regs<kSpJmax>(sc.list + (so + m) * g.chunks * g.cap, g.cap, nseg, k1 - clt, even, base, width, sh, v1, v2))
-            why = kWhySelect;
+        // short lists (the brackets from the previous block's records keep about half as much as sampled ones)
+        // take the selection with fewer registers per thread: the same steps over fewer slots
+        bool small = true;
+#pragma unroll
+        for (int sg = 0; sg < kSpSegs; ++sg) small = small && nseg[sg] <= (uint32_t)((kSpJsmall / kSpSegs) * kSpSelThreads);
+        const uint32_t *lst = sc.list + (so + m) * g.chunks * g.cap;
+        const bool sel = small ? sp_select_regs<kSpJsmall>(lst, g.cap, nseg, k1 - clt, even, base, width, sh, v1, v2)
+                               : sp_select_regs<kSpJmax>(lst, g.cap, nseg, k1 - clt, even, base, width, sh, v1, v2);
+        if (!sel) why = kWhySelect;
     }
     if (tid == 0) {
         if (why < 0) {
